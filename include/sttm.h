@@ -1,0 +1,156 @@
+/*
+ * sttm.h - C ABI of the STTM token-merging library for NVIDIA B200 (sm_100a).
+ *
+ * STTM ("Multi-Granular Spatio-Temporal Token Merging", Section 3) reduces a video's
+ * visual tokens Z_V [T, H, W, D] to a packed multi-granular set Z_ST [N_ST, D]:
+ *   1. spatial stage (Section 3.2): per frame, 2x2 average pooling builds a quadtree up
+ *      to a coarsest map of at most lv1 x lv1 nodes; a coarse-to-fine search keeps the
+ *      coarsest node whose children all have cosine similarity > tau_s to it;
+ *   2. temporal stage (Section 3.3): every kept node of frame t is compared with the
+ *      kept nodes of frame t-1 that overlap its region and is linked to one whose
+ *      similarity is > tau_t (priority to the top-left one); links are followed to the
+ *      common root in the earliest frame and all nodes of a chain are averaged into it;
+ *   3. reordering (Section 3.4): surviving tokens are ordered by frame, then by their
+ *      top-left coordinate (row-major), and receive position ids.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says
+ *     "host".  The library never frees or keeps caller memory.
+ *   - Except sttm_merge / sttm_merge_host (which keep one cached workspace per device)
+ *     the library allocates nothing: the caller provides `ws` of at least
+ *     sttm_workspace_bytes(params) bytes, 256-byte aligned.
+ *   - Calls are asynchronous on `stream` and do not synchronise (sttm_merge_host does).
+ *   - Host-detectable errors are returned with no work enqueued.  Conditions found on
+ *     the device (output capacity exceeded, root search not converged) are OR-ed as
+ *     (1 << status) bits into *device_status; kernels never trap.
+ *   - Layout: feats is [B, T, H, W, D] contiguous, D fastest; D must be a multiple of 4
+ *     and the base pointer 16-byte aligned.  A token's cell id inside its video is
+ *     c = t*H*W + y*W + x.  A quadtree node is named by the cell id of its top-left
+ *     (anchor) cell.  Quadtrees deeper than 3 levels (coarsest node wider than 4 cells)
+ *     are reported as STTM_ERR_UNSUPPORTED.
+ */
+#ifndef STTM_H
+#define STTM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    STTM_OK = 0,
+    STTM_ERR_ARG = 1,            /* null pointer, non-positive size, misalignment      */
+    STTM_ERR_UNSUPPORTED = 2,    /* shape outside what the kernels cover                */
+    STTM_ERR_WORKSPACE = 3,      /* ws_bytes smaller than sttm_workspace_bytes()        */
+    STTM_ERR_CAPACITY = 4,       /* more output rows than out_capacity_rows (device)    */
+    STTM_ERR_NOT_CONVERGED = 5,  /* root search hit its round limit (device)            */
+    STTM_ERR_CUDA = 6            /* a CUDA runtime call failed                          */
+} sttm_status;
+
+typedef enum { STTM_BF16 = 0, STTM_F32 = 1 } sttm_dtype;
+/* Section 3.4: keep the surviving token's original position, or renumber 0..N_ST-1. */
+typedef enum { STTM_POS_SURVIVED = 0, STTM_POS_REASSIGNED = 1 } sttm_pos_mode;
+/* Averaging weights inside a chain (the paper does not fix them): one per node, or the
+ * number of grid cells the node covers. */
+typedef enum { STTM_W_NODE = 0, STTM_W_AREA = 1 } sttm_weight_mode;
+
+typedef struct sttm_params {
+    int B, T, H, W, D;            /* videos, frames, grid, channels                      */
+    sttm_dtype in_dtype;          /* dtype of feats                                       */
+    sttm_dtype out_dtype;         /* dtype of out_feats                                   */
+    int lv1;                      /* coarsest map is at most lv1 x lv1 (paper: 4, or 2)   */
+    float tau_s, tau_t;           /* thresholds, used when the per-video arrays are NULL  */
+    const float* tau_s_per_video; /* host, [B] or NULL                                    */
+    const float* tau_t_per_video; /* host, [B] or NULL                                    */
+    sttm_pos_mode pos;
+    sttm_weight_mode wt;
+    long long out_capacity_rows;  /* rows available in out_feats / out_pos (all videos)   */
+} sttm_params;
+
+/* Fills *p with defaults: B=1, bf16 in and out, lv1=4, survived ids, node weights,
+ * capacity B*T*H*W.  Host only. */
+void sttm_default_params(sttm_params* p, int T, int H, int W, int D, float tau_s, float tau_t);
+
+/* Bytes of device workspace the calls below need for these params (0 on bad params). */
+size_t sttm_workspace_bytes(const sttm_params* p);
+
+/* Number of parent-child similarities per frame, stored level by level (level 0 first,
+ * each level row-major); 0 when the grid has a single level. Host only. */
+int sttm_sims_per_frame(int H, int W, int lv1);
+
+/*
+ * Spatial stage alone (Section 3.2).
+ *   cover_level  [B, T, H, W] int8   out: quadtree level (0 = single cell) of the kept
+ *                                    node covering each cell
+ *   frame_counts [B, T] int32        out: kept nodes per frame
+ *   spatial_sims [B, T, sttm_sims_per_frame] float32, out, may be NULL:
+ *                                    cos(node, its parent) of every non-root node
+ */
+sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
+                         int8_t* cover_level, int32_t* frame_counts, float* spatial_sims,
+                         void* stream);
+
+/*
+ * Temporal stage alone (Section 3.3), given the spatial stage's cover map.
+ *   link [B, T*H*W] int32  out, per cell: anchor id of the node (frame t-1) that the
+ *                          cell's covering node is linked to, or -1
+ *   root [B, T*H*W] int32  out, per cell: anchor id of the chain's root
+ *   temporal_sims [B, T*H*W] float32, out, may be NULL: cosine of each compared pair,
+ *                          stored at the anchor cell of the finer node of the pair
+ *                          (frame t's index), NaN elsewhere
+ * sttm_spatial must have run on the same ws before (it leaves the node norms there).
+ */
+sttm_status sttm_temporal(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
+                          const int8_t* cover_level, int32_t* link, int32_t* root,
+                          float* temporal_sims, int32_t* device_status, void* stream);
+
+/*
+ * The whole path (Sections 3.2-3.4) for B videos.
+ *   out_feats   [out_capacity_rows, D] out_dtype  packed rows, videos back to back
+ *   out_pos     [out_capacity_rows] int32         position id per row (cell id inside
+ *                                                 its video, or 0..count-1)
+ *   merge_map   [B, T*H*W] int32, may be NULL     per cell: row (inside its video) it
+ *                                                 was merged into
+ *   out_count   [B] int32                         rows per video
+ *   out_offsets [B+1] int64, may be NULL          first row of each video
+ *   device_status int32, may be NULL              OR of (1 << sttm_status) bits; must be
+ *                                                 zeroed by the caller
+ * Rows beyond out_capacity_rows are not written; out_count stays exact.
+ */
+sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
+                          void* out_feats, int32_t* out_pos, int32_t* merge_map,
+                          int32_t* out_count, int64_t* out_offsets, int32_t* device_status,
+                          void* stream);
+
+/*
+ * One bf16 video with default params (lv1 = 4, survived ids, node weights, bf16 output,
+ * capacity T*H*W rows).  Uses a workspace cached per device, grown with cudaMalloc when a
+ * larger problem arrives (so the first call on a device synchronises and allocates).
+ */
+sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_s, float tau_t,
+                       void* out_feats, int32_t* out_pos, int32_t* out_count, void* stream);
+
+/*
+ * Same computation with HOST buffers: copies feats to the device, runs sttm_merge_ex,
+ * copies the used rows back and synchronises.  All pointers are host pointers (pinned
+ * memory makes the copies asynchronous and faster).  h_merge_map and h_out_offsets may
+ * be NULL.  Device buffers are cached per device and grown on demand.
+ */
+sttm_status sttm_merge_host(const void* h_feats, const sttm_params* p,
+                            void* h_out_feats, int32_t* h_out_pos, int32_t* h_merge_map,
+                            int32_t* h_out_count, int64_t* h_out_offsets, int32_t* h_device_status);
+
+/* Frees the cached buffers of sttm_merge / sttm_merge_host on the current device. */
+void sttm_release_cache(void);
+
+/* Number of kernels the last sttm_merge_ex on this thread enqueued (for benchmarks). */
+int sttm_last_launch_count(void);
+
+const char* sttm_status_string(sttm_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,429 @@
+// Host side of the STTM library: argument checks, workspace layout, kernel launches.
+// Exports the C ABI declared in include/sttm.h.
+#include "../../include/sttm.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+
+#include "sttm_kernels.cuh"
+
+namespace {
+
+using namespace sttm;
+
+constexpr int kSmCount = 148;   // B200; the library is built for sm_100a only
+
+thread_local int g_launches = 0;
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct Plan {
+    Geo g;
+    int Tc, nchunk, nslice;
+    long long cells;          // B*N
+    long long partial_slots;
+    // byte offsets into the workspace
+    size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
+        frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status,
+        zero_end, partial, total;
+};
+
+int levels_of(int H, int W, int lv1, int* H1, int* W1, int* Hc, int* Wc) {
+    int L = 1, h = H, w = W;
+    *H1 = H; *W1 = W;
+    while (std::max(h, w) > lv1) {
+        h = (h + 1) / 2;
+        w = (w + 1) / 2;
+        if (L == 1) { *H1 = h; *W1 = w; }
+        L++;
+    }
+    *Hc = h; *Wc = w;
+    return L;
+}
+
+sttm_status make_plan(const sttm_params* p, Plan* pl) {
+    if (p == nullptr) return STTM_ERR_ARG;
+    if (p->B < 1 || p->T < 1 || p->H < 1 || p->W < 1 || p->D < 1 || p->lv1 < 1) return STTM_ERR_ARG;
+    if (p->D % 4 != 0) return STTM_ERR_ARG;
+    if (p->in_dtype != STTM_BF16 && p->in_dtype != STTM_F32) return STTM_ERR_ARG;
+    if (p->out_dtype != STTM_BF16 && p->out_dtype != STTM_F32) return STTM_ERR_ARG;
+    if (p->B > kMaxBatch) return STTM_ERR_UNSUPPORTED;
+    if ((long long)p->B * p->T * p->H * p->W >= (1ll << 31)) return STTM_ERR_UNSUPPORTED;
+    Geo& g = pl->g;
+    g.B = p->B; g.T = p->T; g.H = p->H; g.W = p->W; g.D = p->D;
+    g.L = levels_of(p->H, p->W, p->lv1, &g.H1, &g.W1, &g.Hc, &g.Wc);
+    if (g.L > 3) return STTM_ERR_UNSUPPORTED;
+    g.side = 1 << (g.L - 1);
+    g.ncol = g.Hc * g.Wc;
+    g.HW = p->H * p->W;
+    g.N = p->T * g.HW;
+    g.nsim = g.L == 1 ? 0 : (g.L == 2 ? g.HW : g.HW + g.H1 * g.W1);
+    pl->cells = (long long)g.B * g.N;
+
+    pl->nslice = (g.D + kSliceCh - 1) / kSliceCh;
+    const long long per_chunk = (long long)g.B * g.ncol * pl->nslice;
+    const long long target = 2ll * kSmCount * 16;
+    long long nchunk = (target + per_chunk - 1) / per_chunk;
+    nchunk = std::max(1ll, std::min<long long>(nchunk, std::max(1, g.T / 8)));
+    pl->Tc = (int)((g.T + nchunk - 1) / nchunk);
+    pl->nchunk = (g.T + pl->Tc - 1) / pl->Tc;
+    const int NC = g.side * g.side;
+    pl->partial_slots = 2ll * NC * g.ncol * pl->nchunk * g.B;
+
+    const int NN = g.L == 3 ? 21 : (g.L == 2 ? 5 : 1);
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+    pl->norms = take((size_t)g.B * g.T * g.ncol * NN * sizeof(float));
+    pl->cover = take((size_t)pl->cells);
+    pl->link = take((size_t)pl->cells * 4);
+    pl->root = take((size_t)pl->cells * 4);
+    pl->row_at_root = take((size_t)pl->cells * 4);
+    pl->cell_row = take((size_t)pl->cells * 4);
+    pl->row_anchor = take((size_t)pl->cells * 4);
+    pl->span_off = take((size_t)pl->cells * 4);
+    pl->frame_roots = take((size_t)g.B * g.T * 4);
+    pl->frame_base = take((size_t)g.B * g.T * 4);
+    pl->vid_off = take((size_t)(g.B + 1) * 8);
+    pl->zero_begin = o;
+    pl->frame_counts = take((size_t)g.B * g.T * 4);
+    pl->row_weight = take((size_t)pl->cells * 4);
+    pl->row_last_t = take((size_t)pl->cells * 4);
+    pl->span_total = take(4);
+    pl->status = take(4);
+    pl->zero_end = o;
+    pl->partial = take((size_t)pl->partial_slots * g.D * sizeof(float));
+    pl->total = o;
+    return STTM_OK;
+}
+
+void fill_taus(const sttm_params* p, Taus* t) {
+    for (int b = 0; b < p->B; b++) {
+        t->s[b] = p->tau_s_per_video ? p->tau_s_per_video[b] : p->tau_s;
+        t->t[b] = p->tau_t_per_video ? p->tau_t_per_video[b] : p->tau_t;
+    }
+}
+
+template <typename F>
+sttm_status by_levels_dtype(int L, sttm_dtype dt, F&& f) {
+    if (dt == STTM_BF16) {
+        if (L == 1) return f(std::integral_constant<int, 1>{}, (const __nv_bfloat16*)nullptr);
+        if (L == 2) return f(std::integral_constant<int, 2>{}, (const __nv_bfloat16*)nullptr);
+        return f(std::integral_constant<int, 3>{}, (const __nv_bfloat16*)nullptr);
+    }
+    if (L == 1) return f(std::integral_constant<int, 1>{}, (const float*)nullptr);
+    if (L == 2) return f(std::integral_constant<int, 2>{}, (const float*)nullptr);
+    return f(std::integral_constant<int, 3>{}, (const float*)nullptr);
+}
+
+#define STTM_CUDA_TRY(expr)                          \
+    do {                                             \
+        cudaError_t e_ = (expr);                     \
+        if (e_ != cudaSuccess) return STTM_ERR_CUDA; \
+    } while (0)
+
+inline sttm_status launched() {
+    g_launches++;
+    return cudaPeekAtLastError() == cudaSuccess ? STTM_OK : STTM_ERR_CUDA;
+}
+
+inline unsigned blocks_for(long long items, int per_block) { return (unsigned)((items + per_block - 1) / per_block); }
+
+sttm_status run_spatial(const void* feats, const sttm_params* p, const Plan& pl, char* ws, int8_t* cover,
+                        int32_t* frame_counts, float* sims, cudaStream_t st) {
+    Taus taus;
+    fill_taus(p, &taus);
+    const Geo g = pl.g;
+    float* norms = (float*)(ws + pl.norms);
+    const long long warps = (long long)g.B * g.T * g.ncol;
+    return by_levels_dtype(g.L, p->in_dtype, [&](auto lv, auto* tag) {
+        using T = std::remove_const_t<std::remove_pointer_t<decltype(tag)>>;
+        k_spatial<decltype(lv)::value, T><<<blocks_for(warps, kWarpsPerBlock), kWarpsPerBlock * 32, 0, st>>>(
+            (const T*)feats, g, taus, cover, frame_counts, sims, norms);
+        return launched();
+    });
+}
+
+sttm_status run_temporal(const void* feats, const sttm_params* p, const Plan& pl, char* ws, const int8_t* cover,
+                         int32_t* link, int32_t* root, float* tsim, int32_t* status, cudaStream_t st) {
+    Taus taus;
+    fill_taus(p, &taus);
+    const Geo g = pl.g;
+    const float* norms = (const float*)(ws + pl.norms);
+    const long long warps = (long long)g.B * g.T * g.ncol;
+    int max_rounds = 2;
+    while ((1 << (max_rounds - 2)) < g.T) max_rounds++;
+    return by_levels_dtype(g.L, p->in_dtype, [&](auto lv, auto* tag) {
+        using T = std::remove_const_t<std::remove_pointer_t<decltype(tag)>>;
+        constexpr int LV = decltype(lv)::value;
+        k_temporal<LV, T><<<blocks_for(warps, kWarpsPerBlock), kWarpsPerBlock * 32, 0, st>>>(
+            (const T*)feats, g, taus, cover, norms, link, tsim);
+        sttm_status s = launched();
+        if (s != STTM_OK) return s;
+        k_roots<LV><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, status, max_rounds);
+        return launched();
+    });
+}
+
+template <int LV, typename T, typename OutT>
+sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void* out, long long capacity,
+                              int weight_mode, cudaStream_t st) {
+    const Geo g = pl.g;
+    const size_t smem = (size_t)kAccWarps * Col<LV>::NC * kSliceCh * sizeof(float);
+    static bool configured = false;
+    if (!configured) {
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_accumulate<LV, T, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)smem));
+        configured = true;
+    }
+    const long long warps = (long long)g.B * g.ncol * pl.nchunk * pl.nslice;
+    k_accumulate<LV, T, OutT><<<blocks_for(warps, kAccWarps), kAccWarps * 32, smem, st>>>(
+        (const T*)feats, g, pl.Tc, pl.nchunk, pl.nslice, (const int8_t*)(ws + pl.cover),
+        (const int32_t*)(ws + pl.cell_row), (const int32_t*)(ws + pl.row_weight),
+        (const int32_t*)(ws + pl.span_off), (const int32_t*)(ws + pl.row_anchor), (float*)(ws + pl.partial),
+        (OutT*)out, capacity, weight_mode);
+    sttm_status s = launched();
+    if (s != STTM_OK) return s;
+    k_combine<OutT><<<kSmCount * 2, 256, 0, st>>>(g, pl.Tc, (const long long*)(ws + pl.vid_off),
+                                                 (const int32_t*)(ws + pl.span_off),
+                                                 (const int32_t*)(ws + pl.row_anchor),
+                                                 (const int32_t*)(ws + pl.row_last_t),
+                                                 (const int32_t*)(ws + pl.row_weight),
+                                                 (const float*)(ws + pl.partial), (OutT*)out, capacity);
+    return launched();
+}
+
+bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
+
+// cached buffers for sttm_merge / sttm_merge_host, one set per device
+struct Cache {
+    void* ws = nullptr; size_t ws_bytes = 0;
+    void* feats = nullptr; size_t feats_bytes = 0;
+    void* out = nullptr; size_t out_bytes = 0;
+    void* ints = nullptr; size_t ints_bytes = 0;   // pos, map, count, offsets, status
+};
+Cache g_cache[64];
+
+sttm_status grow(void** ptr, size_t* have, size_t need) {
+    if (*have >= need) return STTM_OK;
+    if (*ptr) { STTM_CUDA_TRY(cudaFree(*ptr)); *ptr = nullptr; *have = 0; }
+    STTM_CUDA_TRY(cudaMalloc(ptr, need));
+    *have = need;
+    return STTM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sttm_status_string(sttm_status s) {
+    switch (s) {
+        case STTM_OK: return "ok";
+        case STTM_ERR_ARG: return "bad argument";
+        case STTM_ERR_UNSUPPORTED: return "unsupported shape";
+        case STTM_ERR_WORKSPACE: return "workspace too small";
+        case STTM_ERR_CAPACITY: return "output capacity exceeded";
+        case STTM_ERR_NOT_CONVERGED: return "root search did not converge";
+        case STTM_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown";
+}
+
+void sttm_default_params(sttm_params* p, int T, int H, int W, int D, float tau_s, float tau_t) {
+    if (!p) return;
+    std::memset(p, 0, sizeof(*p));
+    p->B = 1; p->T = T; p->H = H; p->W = W; p->D = D;
+    p->in_dtype = STTM_BF16; p->out_dtype = STTM_BF16;
+    p->lv1 = 4;
+    p->tau_s = tau_s; p->tau_t = tau_t;
+    p->pos = STTM_POS_SURVIVED; p->wt = STTM_W_NODE;
+    p->out_capacity_rows = (long long)T * H * W;
+}
+
+size_t sttm_workspace_bytes(const sttm_params* p) {
+    Plan pl;
+    if (make_plan(p, &pl) != STTM_OK) return 0;
+    return pl.total;
+}
+
+int sttm_sims_per_frame(int H, int W, int lv1) {
+    if (H < 1 || W < 1 || lv1 < 1) return 0;
+    int n = 0, h = H, w = W;
+    while (std::max(h, w) > lv1) { n += h * w; h = (h + 1) / 2; w = (w + 1) / 2; }
+    return n;
+}
+
+int sttm_last_launch_count(void) { return g_launches; }
+
+sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
+                         int8_t* cover_level, int32_t* frame_counts, float* spatial_sims, void* stream) {
+    Plan pl;
+    sttm_status s = make_plan(p, &pl);
+    if (s != STTM_OK) return s;
+    if (!feats || !ws || !cover_level || !frame_counts) return STTM_ERR_ARG;
+    if (misaligned(feats, 16) || misaligned(ws, 256)) return STTM_ERR_ARG;
+    if (ws_bytes < pl.total) return STTM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    g_launches = 0;
+    STTM_CUDA_TRY(cudaMemsetAsync(frame_counts, 0, (size_t)pl.g.B * pl.g.T * 4, st));
+    return run_spatial(feats, p, pl, (char*)ws, cover_level, frame_counts, spatial_sims, st);
+}
+
+sttm_status sttm_temporal(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
+                          const int8_t* cover_level, int32_t* link, int32_t* root, float* temporal_sims,
+                          int32_t* device_status, void* stream) {
+    Plan pl;
+    sttm_status s = make_plan(p, &pl);
+    if (s != STTM_OK) return s;
+    if (!feats || !ws || !cover_level || !link || !root) return STTM_ERR_ARG;
+    if (misaligned(feats, 16) || misaligned(ws, 256)) return STTM_ERR_ARG;
+    if (ws_bytes < pl.total) return STTM_ERR_WORKSPACE;
+    g_launches = 0;
+    return run_temporal(feats, p, pl, (char*)ws, cover_level, link, root, temporal_sims, device_status,
+                        (cudaStream_t)stream);
+}
+
+sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, size_t ws_bytes, void* out_feats,
+                          int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
+                          int32_t* device_status, void* stream) {
+    Plan pl;
+    sttm_status s = make_plan(p, &pl);
+    if (s != STTM_OK) return s;
+    if (!feats || !ws_ || !out_feats || !out_pos || !out_count) return STTM_ERR_ARG;
+    if (p->out_capacity_rows < 0) return STTM_ERR_ARG;
+    if (misaligned(feats, 16) || misaligned(ws_, 256) || misaligned(out_feats, 16)) return STTM_ERR_ARG;
+    if (ws_bytes < pl.total) return STTM_ERR_WORKSPACE;
+    char* ws = (char*)ws_;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Geo g = pl.g;
+    g_launches = 0;
+
+    STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.zero_begin, 0, pl.zero_end - pl.zero_begin, st));
+    int8_t* cover = (int8_t*)(ws + pl.cover);
+    int32_t* link = (int32_t*)(ws + pl.link);
+    int32_t* root = (int32_t*)(ws + pl.root);
+    s = run_spatial(feats, p, pl, ws, cover, (int32_t*)(ws + pl.frame_counts), nullptr, st);
+    if (s != STTM_OK) return s;
+    s = run_temporal(feats, p, pl, ws, cover, link, root, nullptr, device_status, st);
+    if (s != STTM_OK) return s;
+
+    int32_t* frame_roots = (int32_t*)(ws + pl.frame_roots);
+    int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
+    long long* vid_off = (long long*)(ws + pl.vid_off);
+    int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
+    int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
+    k_frame_roots<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_roots);
+    if ((s = launched()) != STTM_OK) return s;
+    k_scan_frames<<<1, 1024, 0, st>>>(g, frame_roots, frame_base, out_count, vid_off, out_offsets);
+    if ((s = launched()) != STTM_OK) return s;
+    k_rows<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_base, vid_off, row_at_root, row_anchor, out_pos,
+                                      p->out_capacity_rows, (int)p->pos, device_status);
+    if ((s = launched()) != STTM_OK) return s;
+    k_members<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, cover, root, row_at_root, vid_off,
+                                                        (int32_t*)(ws + pl.cell_row), merge_map,
+                                                        (int32_t*)(ws + pl.row_weight),
+                                                        (int32_t*)(ws + pl.row_last_t), (int)p->wt);
+    if ((s = launched()) != STTM_OK) return s;
+    k_span<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, pl.Tc, vid_off, row_anchor,
+                                                     (const int32_t*)(ws + pl.row_last_t),
+                                                     (int32_t*)(ws + pl.span_off), (int32_t*)(ws + pl.span_total));
+    if ((s = launched()) != STTM_OK) return s;
+
+    return by_levels_dtype(g.L, p->in_dtype, [&](auto lv, auto* tag) {
+        using T = std::remove_const_t<std::remove_pointer_t<decltype(tag)>>;
+        constexpr int LV = decltype(lv)::value;
+        if (p->out_dtype == STTM_BF16)
+            return launch_accumulate<LV, T, __nv_bfloat16>(feats, pl, ws, out_feats, p->out_capacity_rows,
+                                                           (int)p->wt, st);
+        return launch_accumulate<LV, T, float>(feats, pl, ws, out_feats, p->out_capacity_rows, (int)p->wt, st);
+    });
+}
+
+sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_s, float tau_t, void* out_feats,
+                       int32_t* out_pos, int32_t* out_count, void* stream) {
+    sttm_params p;
+    sttm_default_params(&p, T, H, W, D, tau_s, tau_t);
+    const size_t need = sttm_workspace_bytes(&p);
+    if (need == 0) {
+        Plan pl;
+        return make_plan(&p, &pl);
+    }
+    int dev = 0;
+    STTM_CUDA_TRY(cudaGetDevice(&dev));
+    Cache& c = g_cache[dev % 64];
+    if (c.ws_bytes < need) {
+        STTM_CUDA_TRY(cudaDeviceSynchronize());
+        sttm_status s = grow(&c.ws, &c.ws_bytes, need);
+        if (s != STTM_OK) return s;
+    }
+    return sttm_merge_ex(feats, &p, c.ws, c.ws_bytes, out_feats, out_pos, nullptr, out_count, nullptr, nullptr,
+                         stream);
+}
+
+sttm_status sttm_merge_host(const void* h_feats, const sttm_params* p, void* h_out_feats, int32_t* h_out_pos,
+                            int32_t* h_merge_map, int32_t* h_out_count, int64_t* h_out_offsets,
+                            int32_t* h_device_status) {
+    Plan pl;
+    sttm_status s = make_plan(p, &pl);
+    if (s != STTM_OK) return s;
+    if (!h_feats || !h_out_feats || !h_out_pos || !h_out_count) return STTM_ERR_ARG;
+    if (p->out_capacity_rows < 0) return STTM_ERR_ARG;
+    int dev = 0;
+    STTM_CUDA_TRY(cudaGetDevice(&dev));
+    Cache& c = g_cache[dev % 64];
+    const Geo g = pl.g;
+    const size_t in_elt = p->in_dtype == STTM_BF16 ? 2 : 4, out_elt = p->out_dtype == STTM_BF16 ? 2 : 4;
+    const size_t feats_bytes = (size_t)pl.cells * g.D * in_elt;
+    const size_t out_bytes = (size_t)p->out_capacity_rows * g.D * out_elt;
+    // ints: out_pos [cap] | merge_map [cells] | out_count [B] | status [1] | offsets [B+1] (int64)
+    const size_t o_pos = 0, o_map = align_up((size_t)p->out_capacity_rows * 4),
+                 o_cnt = o_map + align_up((size_t)pl.cells * 4), o_status = o_cnt + align_up((size_t)g.B * 4),
+                 o_off = o_status + 256, ints_bytes = o_off + align_up((size_t)(g.B + 1) * 8);
+    if (c.ws_bytes < pl.total || c.feats_bytes < feats_bytes || c.out_bytes < out_bytes ||
+        c.ints_bytes < ints_bytes) {
+        STTM_CUDA_TRY(cudaDeviceSynchronize());
+        if ((s = grow(&c.ws, &c.ws_bytes, pl.total)) != STTM_OK) return s;
+        if ((s = grow(&c.feats, &c.feats_bytes, feats_bytes)) != STTM_OK) return s;
+        if ((s = grow(&c.out, &c.out_bytes, std::max<size_t>(out_bytes, 256))) != STTM_OK) return s;
+        if ((s = grow(&c.ints, &c.ints_bytes, ints_bytes)) != STTM_OK) return s;
+    }
+    char* ints = (char*)c.ints;
+    cudaStream_t st = 0;
+    STTM_CUDA_TRY(cudaMemcpyAsync(c.feats, h_feats, feats_bytes, cudaMemcpyHostToDevice, st));
+    STTM_CUDA_TRY(cudaMemsetAsync(ints + o_status, 0, 4, st));
+    s = sttm_merge_ex(c.feats, p, c.ws, c.ws_bytes, c.out, (int32_t*)(ints + o_pos),
+                      h_merge_map ? (int32_t*)(ints + o_map) : nullptr, (int32_t*)(ints + o_cnt),
+                      (int64_t*)(ints + o_off), (int32_t*)(ints + o_status), st);
+    if (s != STTM_OK) return s;
+    long long offsets[kMaxBatch + 1];
+    STTM_CUDA_TRY(cudaMemcpyAsync(offsets, ints + o_off, (size_t)(g.B + 1) * 8, cudaMemcpyDeviceToHost, st));
+    STTM_CUDA_TRY(cudaMemcpyAsync(h_out_count, ints + o_cnt, (size_t)g.B * 4, cudaMemcpyDeviceToHost, st));
+    int32_t status = 0;
+    STTM_CUDA_TRY(cudaMemcpyAsync(&status, ints + o_status, 4, cudaMemcpyDeviceToHost, st));
+    STTM_CUDA_TRY(cudaStreamSynchronize(st));
+    const long long rows = std::min<long long>(offsets[g.B], p->out_capacity_rows);
+    STTM_CUDA_TRY(cudaMemcpyAsync(h_out_feats, c.out, (size_t)rows * g.D * out_elt, cudaMemcpyDeviceToHost, st));
+    STTM_CUDA_TRY(cudaMemcpyAsync(h_out_pos, ints + o_pos, (size_t)rows * 4, cudaMemcpyDeviceToHost, st));
+    if (h_merge_map)
+        STTM_CUDA_TRY(cudaMemcpyAsync(h_merge_map, ints + o_map, (size_t)pl.cells * 4, cudaMemcpyDeviceToHost, st));
+    STTM_CUDA_TRY(cudaStreamSynchronize(st));
+    if (h_out_offsets) std::memcpy(h_out_offsets, offsets, (size_t)(g.B + 1) * 8);
+    if (h_device_status) *h_device_status = status;
+    return STTM_OK;
+}
+
+void sttm_release_cache(void) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return;
+    Cache& c = g_cache[dev % 64];
+    cudaDeviceSynchronize();
+    if (c.ws) cudaFree(c.ws);
+    if (c.feats) cudaFree(c.feats);
+    if (c.out) cudaFree(c.out);
+    if (c.ints) cudaFree(c.ints);
+    c = Cache();
+}
+
+}  // extern "C"

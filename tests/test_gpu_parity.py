@@ -1,0 +1,194 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded inputs.  Structure (cover map, links, roots, merge map, position ids,
+counts) must match bit for bit; merged features within the tolerance in helpers."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2507_07990_b200 import binding, inputs
+from tests import helpers
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_compare(video_np, tau_s, tau_t, lv1=4, out_dtype=torch.float32, wt=binding.W_NODE,
+                    pos=binding.POS_SURVIVED, stages=True):
+    T, H, W, D = video_np.shape
+    N = T * H * W
+    ref = oracle.merge(video_np, tau_s, tau_t, lv1=lv1, weight_mode=wt, pos_mode=pos, want_sims=True, want_pairs=True)
+    dev = helpers.to_torch(video_np)
+    out = binding.sttm_merge_ex(dev, tau_s, tau_t, lv1=lv1, out_dtype=out_dtype, wt=wt, pos=pos)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    count = int(out.out_count[0].item())
+    assert count == ref.count
+    assert out.out_offsets.tolist() == [0, ref.count]
+    np.testing.assert_array_equal(out.merge_map[0].cpu().numpy(), ref.merge_map)
+    np.testing.assert_array_equal(out.out_pos[:count].cpu().numpy(), ref.out_pos)
+    helpers.assert_features_close(out.out_feats[:count].float().cpu().numpy(), ref.out_feats,
+                                  out_dtype == torch.bfloat16)
+    if stages:
+        cover, counts, sims, ws = binding.sttm_spatial(dev, tau_s, lv1=lv1, want_sims=True)
+        link, root, tsim, status = binding.sttm_temporal(dev, cover, tau_s, tau_t, ws, lv1=lv1, want_sims=True)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        np.testing.assert_array_equal(cover[0].cpu().numpy(), ref.cover_level)
+        np.testing.assert_array_equal(link[0].cpu().numpy(), ref.link)
+        np.testing.assert_array_equal(root[0].cpu().numpy(), ref.root)
+        per_frame = []
+        for t in range(T):
+            n = 0
+            for (y, x), l in np.ndenumerate(ref.cover_level[t]):
+                m = (1 << int(l)) - 1
+                n += int((y & m) == 0 and (x & m) == 0)      # anchors of kept nodes
+            per_frame.append(n)
+        assert counts[0].cpu().tolist() == per_frame
+        if ref.spatial_sims.size:
+            np.testing.assert_allclose(sims[0].cpu().numpy(), ref.spatial_sims, rtol=0, atol=2e-5)
+        ts = tsim[0].cpu().numpy()
+        got = {}
+        for v in np.nonzero(~np.isnan(ts))[0]:
+            got[int(v)] = float(ts[v])
+        assert len(got) == len(ref.tsim)
+        HW = H * W
+        for v, u, s in zip(ref.tsim_v, ref.tsim_u, ref.tsim):
+            # a pair is stored at the anchor of its finer node, in frame t's numbering
+            key = int(v) if ref.cover_level.ravel()[v] <= ref.cover_level.ravel()[u] else int(u) + HW
+            assert abs(got[key] - s) < 2e-5
+    return ref
+
+
+SHAPES = [  # T, H, W, D, lv1, dtype
+    (4, 8, 8, 64, 4, "f32"),
+    (4, 8, 8, 64, 2, "f32"),
+    (6, 13, 13, 256, 4, "bf16"),
+    (5, 16, 16, 384, 4, "bf16"),
+    (3, 14, 14, 128, 4, "bf16"),
+    (4, 4, 4, 128, 4, "bf16"),       # single level: temporal only
+    (3, 7, 5, 132, 4, "bf16"),       # ragged channel tail, non-square
+    (9, 3, 3, 64, 2, "f32"),
+    (2, 1, 1, 8, 4, "f32"),
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "T%dH%dW%dD%dlv%d%s" % s)
+@pytest.mark.parametrize("q_s,q_t", [(0.5, 0.5), (0.15, 0.8), (0.9, 0.2)])
+def test_parity_small(shape, q_s, q_t):
+    T, H, W, D, lv1, dtype = shape
+    done = 0
+    for seed in range(3):
+        spec = helpers.small_spec(100 + seed, T, H, W, D, dtype=dtype, sigma=0.3 if D < 200 else 0.05)
+        video = inputs.make_video(spec)
+        taus = helpers.safe_thresholds(video, q_s, q_t, lv1)
+        if taus is None:
+            continue
+        for out_dtype in (torch.float32, torch.bfloat16):
+            run_and_compare(video, taus[0], taus[1], lv1=lv1, out_dtype=out_dtype)
+        done += 1
+    assert done >= 1, "no seed gave thresholds with a margin"
+
+
+def test_parity_weight_and_position_modes():
+    spec = helpers.small_spec(7, 6, 13, 13, 256)
+    video = inputs.make_video(spec)
+    tau_s, tau_t = helpers.safe_thresholds(video, 0.4, 0.5)
+    run_and_compare(video, tau_s, tau_t, wt=binding.W_AREA, stages=False)
+    run_and_compare(video, tau_s, tau_t, pos=binding.POS_REASSIGNED, stages=False)
+
+
+def test_degenerate_thresholds():
+    spec = helpers.small_spec(8, 12, 13, 13, 128)
+    video = inputs.make_video(spec)
+    for tau_s, tau_t in [(2.0, 2.0), (-2.0, 2.0), (2.0, -2.0), (-2.0, -2.0)]:
+        ref = run_and_compare(video, tau_s, tau_t)
+    assert ref.count == 16          # everything merges: the 4x4 coarsest map of frame 0
+
+
+def test_tiny_config_fixed_thresholds():
+    entry = inputs.load_thresholds()["tiny"]
+    spec = inputs.config_videos("tiny", entry["seed_bump"])[0]
+    video = inputs.make_video(spec)
+    fixed = entry["videos"][0]["fixed"]
+    for lv1, expect in ((4, fixed["count"]), (2, fixed["count_lv1_2"])):
+        ref = run_and_compare(video, fixed["tau_s"], fixed["tau_t"], lv1=lv1)
+        assert ref.count == expect
+
+
+def test_long_chains_cross_time_chunks():
+    """A static video: every chain spans all frames, so rows are summed across the
+    averaging kernel's time chunks."""
+    spec = helpers.small_spec(9, 96, 13, 13, 128, p_static=0.97)
+    video = inputs.make_video(spec)
+    taus = helpers.safe_thresholds(video, 0.5, 0.3)
+    assert taus is not None
+    ref = run_and_compare(video, taus[0], taus[1], stages=False)
+    assert ref.out_members.max() >= 40
+
+
+def test_batch_with_per_video_thresholds():
+    specs = [helpers.small_spec(20 + v, 8, 13, 13, 256, p_static=p) for v, p in enumerate((0.9, 0.5, 0.2))]
+    videos = [inputs.make_video(s) for s in specs]
+    taus = [helpers.safe_thresholds(v, 0.5, 0.5) for v in videos]
+    assert all(t is not None for t in taus)
+    dev = helpers.to_torch(np.stack(videos))
+    out = binding.sttm_merge_ex(dev, [t[0] for t in taus], [t[1] for t in taus], out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    offs = out.out_offsets.tolist()
+    for b, (video, (ts, tt)) in enumerate(zip(videos, taus)):
+        ref = oracle.merge(video, ts, tt)
+        assert int(out.out_count[b]) == ref.count and offs[b + 1] - offs[b] == ref.count
+        np.testing.assert_array_equal(out.merge_map[b].cpu().numpy(), ref.merge_map)
+        np.testing.assert_array_equal(out.out_pos[offs[b]:offs[b + 1]].cpu().numpy(), ref.out_pos)
+        helpers.assert_features_close(out.out_feats[offs[b]:offs[b + 1]].cpu().numpy(), ref.out_feats, False)
+
+
+def test_capacity_overflow_is_reported_not_fatal():
+    spec = helpers.small_spec(30, 4, 8, 8, 64, dtype="f32", sigma=0.3)
+    video = inputs.make_video(spec)
+    ref = oracle.merge(video, 2.0, 2.0)
+    dev = helpers.to_torch(video)
+    out = binding.sttm_merge_ex(dev, 2.0, 2.0, out_dtype=torch.float32, capacity=100)
+    torch.cuda.synchronize()
+    assert int(out.out_count[0]) == ref.count == 256
+    assert int(out.device_status.item()) & (1 << 4)
+    helpers.assert_features_close(out.out_feats[:100].cpu().numpy(), ref.out_feats[:100], False)
+
+
+def test_host_buffer_entry_point_and_simple_merge():
+    spec = helpers.small_spec(31, 6, 13, 13, 256)
+    video = inputs.make_video(spec)
+    tau_s, tau_t = helpers.safe_thresholds(video, 0.5, 0.5)
+    ref = oracle.merge(video, tau_s, tau_t)
+    h = torch.from_numpy(video.view(np.int16)).view(torch.bfloat16).pin_memory()
+    out = binding.sttm_merge_host(h, tau_s, tau_t, want_map=True)
+    assert int(out.out_count[0]) == ref.count
+    np.testing.assert_array_equal(out.merge_map[0].numpy(), ref.merge_map)
+    np.testing.assert_array_equal(out.out_pos[:ref.count].numpy(), ref.out_pos)
+    helpers.assert_features_close(out.out_feats[:ref.count].float().numpy(), ref.out_feats, True)
+    feats, pos, cnt = binding.sttm_merge(h.cuda(), tau_s, tau_t)
+    torch.cuda.synchronize()
+    assert int(cnt) == ref.count
+    np.testing.assert_array_equal(pos[:ref.count].cpu().numpy(), ref.out_pos)
+    helpers.assert_features_close(feats[:ref.count].float().cpu().numpy(), ref.out_feats, True)
+
+
+def test_bad_arguments_are_rejected_on_the_host():
+    dev = torch.zeros((1, 2, 4, 4, 6), dtype=torch.bfloat16, device="cuda")     # D not a multiple of 4
+    with pytest.raises(binding.SttmError) as e:
+        binding.sttm_merge_ex(dev, 0.5, 0.5)
+    assert e.value.code == 1
+    dev = torch.zeros((1, 2, 13, 13, 8), dtype=torch.bfloat16, device="cuda")   # 13 -> 7 -> 4 -> 2: four levels
+    with pytest.raises(binding.SttmError) as e:
+        binding.sttm_merge_ex(dev, 0.5, 0.5, lv1=2)
+    assert e.value.code == 2
+    prob = binding.make_params((1, 2, 13, 13, 8), torch.bfloat16, 0.5, 0.5)
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    lib = binding.load_library()
+    import ctypes as C
+    code = lib.sttm_merge_ex(C.c_void_p(dev.data_ptr()), C.byref(prob.params), C.c_void_p(ws.data_ptr()), 1024,
+                             C.c_void_p(dev.data_ptr()), C.c_void_p(dev.data_ptr()), None,
+                             C.c_void_p(dev.data_ptr()), None, None, None)
+    assert code == 3

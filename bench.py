@@ -1,0 +1,298 @@
+#!/usr/bin/env python
+"""Benchmark of the STTM token-merging path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload long]
+
+One step = one pass of the whole path (spatial quadtree search, temporal linking, root
+resolution, ordering, averaging into a packed output) over one synthetic video of the
+named workload, through the C ABI (sttm_merge_ex).  The default workload is the
+1024-frame, 13x13, D=3584 bf16 video (1.24 GB, ten times the L2) with the thresholds
+stored for it.  With N > 1 every rank merges its own copy of the video (independent
+videos, no data-path collective); the time is the maximum over ranks.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2507_07990_b200 import inputs  # noqa: E402
+
+METRIC = "input visual tokens/sec merged on 1 B200; achieved HBM GB/s vs peak"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic per launch of the dominant kernel, from the ncu capture summarised under
+# profiles/ (bytes read + written for the benchmark's workload); None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def workload_setup(name: str):
+    cfg = inputs.CONFIGS[name]
+    table = inputs.load_thresholds()[name]
+    spec = inputs.config_videos(name, table.get("seed_bump", 0))[0]
+    per_budget = table["videos"][0]
+    key = "fixed" if "fixed" in per_budget else "%.2f" % cfg["budgets"][-1]
+    th = per_budget[key]
+    return cfg, spec, th, key
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_baseline(video_np, th, frames):
+    """The oracle as it stands, on the host cores, on the first `frames` frames."""
+    from oracle import oracle
+    sample = video_np[:frames]
+    t0 = time.perf_counter()
+    r = oracle.merge(sample, th["tau_s"], th["tau_t"], want_feats=True)
+    dt = time.perf_counter() - t0
+    tokens = sample.shape[0] * sample.shape[1] * sample.shape[2]
+    # want_feats runs the structure pass twice (once to size the output buffer)
+    return {"value": tokens / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "first %d of %d frames (%d tokens), one thread, fp64, %.2f s, %d rows"
+                      % (sample.shape[0], video_np.shape[0], tokens, dt, r.count)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cfg, spec, th, key = workload_setup(args.workload)
+    frames = min(spec.T, args.reference_frames)
+    import dataclasses
+    video = inputs.make_video(dataclasses.replace(spec, T=frames))
+    from oracle import oracle
+    tokens = frames * spec.H * spec.W
+    for _ in range(args.warmup):
+        oracle.merge(video, th["tau_s"], th["tau_t"], want_feats=True)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.merge(video, th["tau_s"], th["tau_t"], want_feats=True)
+    dt = time.perf_counter() - t0
+    value = tokens * args.steps / dt
+    sample = "first %d of %d frames (%d tokens) per step, one thread, fp64" % (frames, spec.T, tokens)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(args.workload, spec, th, key),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(name, spec, th, key):
+    return {"workload": "%s: 1 video/GPU, T=%d, %dx%d grid, D=%d %s, block generator p_static=%.2f sigma=%.2f"
+                        % (name, spec.T, spec.H, spec.W, spec.D, spec.dtype, spec.p_static, spec.sigma),
+            "budget": key, "tau_s": th["tau_s"], "tau_t": th["tau_t"], "lv1": 4,
+            "kept_fraction": th["fraction"], "out_rows": th["count"],
+            "l2": "input (%.0f MB) larger than L2; no flush" % (spec.tokens * spec.D * 2 / 1e6)
+                  if spec.tokens * spec.D * 2 > 200e6 else "L2 flushed between steps"}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2507_07990_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.load_library()
+
+    cfg, spec, th, key = workload_setup(args.workload)
+    N = spec.tokens
+    in_bytes = N * spec.D * (2 if spec.dtype == "bf16" else 4)
+    small = in_bytes <= 200e6
+    tdtype = torch.bfloat16 if spec.dtype == "bf16" else torch.float32
+
+    # the video, generated once into pinned host memory and copied to the device
+    h_feats = torch.empty((1, spec.T, spec.H, spec.W, spec.D), dtype=tdtype).pin_memory()
+    view = h_feats.view(torch.int16).numpy().view(np.uint16) if spec.dtype == "bf16" else h_feats.numpy()
+    inputs.make_video(spec, out=view[0])
+    d_feats = h_feats.cuda()
+    plan = binding.MergePlan((1, spec.T, spec.H, spec.W, spec.D), tdtype, th["tau_s"], th["tau_t"],
+                             out_dtype=torch.bfloat16, want_map=False)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    out = None
+    for _ in range(max(args.warmup, 3)):
+        out = plan.run(d_feats)
+    torch.cuda.synchronize()
+    count = int(out.out_count[0].item())
+    status = int(out.device_status.item())
+    if status != 0:
+        raise RuntimeError("device status %d" % status)
+    launches_per_step = out.launches
+
+    timers = [binding.StageTimer() for _ in range(args.steps)]
+    lib = binding.load_library()
+    step_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    for k in range(args.steps):
+        if flush is not None:
+            flush.fill_(k & 0xff)
+        lib.sttm_set_stage_events(timers[k]._handles)
+        step_events[k][0].record()
+        plan.run(d_feats)
+        step_events[k][1].record()
+    lib.sttm_set_stage_events(None)
+    barrier()
+    clocks = sampler.stop() if sampler is not None else None
+    step_ms = [a.elapsed_time(b) for a, b in step_events]
+    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
+    total_ms = float(total_ms.item())
+    ms_per_step = total_ms / args.steps
+    value = world * N * args.steps / (total_ms / 1e3)
+
+    # per-stage times over the timed region (events on the launching stream)
+    stage_ms = {}
+    for tm in timers:
+        for n, v in tm.stage_ms().items():
+            stage_ms[n] = stage_ms.get(n, 0.0) + v / args.steps
+    out_bytes = count * spec.D * 2
+    id_bytes = count * 4
+    path_bytes = in_bytes + out_bytes + id_bytes
+    # algorithmic bytes per launch of each feature-touching stage
+    stage_bytes = {"spatial": in_bytes, "temporal+roots": in_bytes, "accumulate": in_bytes + out_bytes}
+    dominant = max(stage_bytes, key=lambda n: stage_ms.get(n, 0.0))
+    peak, peak_kind = measured_peak()
+    achieved = stage_bytes[dominant] / (stage_ms[dominant] / 1e3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": "of " + peak_kind,
+                "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+                "algorithmic_bytes": stage_bytes[dominant], "kernel_ms": stage_ms[dominant],
+                "stage_ms": stage_ms,
+                "path": {"algorithmic_bytes": path_bytes, "achieved": path_bytes / (ms_per_step / 1e3) / 1e9,
+                         "frac": path_bytes / (ms_per_step / 1e3) / 1e9 / peak,
+                         "frac_of_8000": path_bytes / (ms_per_step / 1e3) / 1e9 / 8000.0}}
+
+    # end to end through the host-buffer entry point: H2D of the video, D2H of the result
+    e2e_steps = max(1, min(args.steps, 5 if not small else args.steps))
+    h_out = torch.empty((N, spec.D), dtype=torch.bfloat16).pin_memory()
+    h_pos = torch.empty((N,), dtype=torch.int32).pin_memory()
+    binding.sttm_merge_host(h_feats, th["tau_s"], th["tau_t"], h_out_feats=h_out, h_out_pos=h_pos)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        r = binding.sttm_merge_host(h_feats, th["tau_s"], th["tau_t"], h_out_feats=h_out, h_out_pos=h_pos)
+    barrier()
+    e2e_s = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+    e2e = {"value": world * N * e2e_steps / float(e2e_s.item()), "unit": UNIT, "h2d_bytes_per_step": in_bytes,
+           "d2h_bytes_per_step": out_bytes + id_bytes + 4 + 16, "steps": e2e_steps,
+           "ms_per_step": 1e3 * float(e2e_s.item()) / e2e_steps}
+    assert int(r.out_count[0]) == count
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": workload_config(args.workload, spec, th, key), "out_rows": count,
+                "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+                "clocks": clocks}
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(view[0], th, min(spec.T, args.baseline_frames))
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long", choices=list(inputs.CONFIGS))
+    ap.add_argument("--baseline-frames", type=int, default=512,
+                    help="frames of the workload the CPU-baseline leg runs the oracle on")
+    ap.add_argument("--reference-frames", type=int, default=64,
+                    help="frames per step of the --impl reference arm")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

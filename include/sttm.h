@@ -148,6 +148,17 @@ void sttm_release_cache(void);
 /* Number of kernels the last sttm_merge_ex on this thread enqueued (for benchmarks). */
 int sttm_last_launch_count(void);
 
+/*
+ * Per-stage timing of sttm_merge_ex for benchmarks.  The path runs as
+ * sttm_stage_count() consecutive stages.  After sttm_set_stage_events(events), with
+ * `events` a host array of sttm_stage_count()+1 cudaEvent_t handles created by the
+ * caller, every sttm_merge_ex on this thread records events[i] on its stream before
+ * stage i and events[i+1] after it.  Pass NULL to switch recording off (the default).
+ */
+int sttm_stage_count(void);
+const char* sttm_stage_name(int i);
+void sttm_set_stage_events(void** events);
+
 const char* sttm_status_string(sttm_status s);
 
 #ifdef __cplusplus

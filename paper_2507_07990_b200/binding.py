@@ -24,7 +24,8 @@ STATUS_NAMES = ["ok", "bad argument", "unsupported shape", "workspace too small"
 
 EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame", "sttm_spatial",
            "sttm_temporal", "sttm_merge_ex", "sttm_merge", "sttm_merge_host", "sttm_release_cache",
-           "sttm_last_launch_count", "sttm_status_string"]
+           "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
+           "sttm_set_stage_events"]
 
 
 class SttmParams(C.Structure):
@@ -75,6 +76,12 @@ def load_library(path: Optional[str] = None):
     lib.sttm_release_cache.restype = None
     lib.sttm_last_launch_count.argtypes = []
     lib.sttm_last_launch_count.restype = C.c_int
+    lib.sttm_stage_count.argtypes = []
+    lib.sttm_stage_count.restype = C.c_int
+    lib.sttm_stage_name.argtypes = [C.c_int]
+    lib.sttm_stage_name.restype = C.c_char_p
+    lib.sttm_set_stage_events.argtypes = [C.POINTER(C.c_void_p)]
+    lib.sttm_set_stage_events.restype = None
     lib.sttm_status_string.argtypes = [C.c_int]
     lib.sttm_status_string.restype = C.c_char_p
     if path == _build.LIB_PATH:
@@ -280,3 +287,28 @@ def sttm_merge_host(h_feats: torch.Tensor, tau_s, tau_t, lv1: int = 4, out_dtype
                                           _ptr(h_map), _ptr(h_cnt), _ptr(h_off), _ptr(h_status)),
            "sttm_merge_host")
     return MergeOutput(h_out_feats, h_out_pos, h_cnt, h_off, h_map, h_status, 0)
+
+
+class StageTimer:
+    """Records one CUDA event per stage boundary of sttm_merge_ex (on the stream the
+    kernels run on) and reports the time each stage took."""
+
+    def __init__(self):
+        lib = load_library()
+        self.names = [lib.sttm_stage_name(i).decode() for i in range(lib.sttm_stage_count())]
+        self.events = [torch.cuda.Event(enable_timing=True) for _ in range(len(self.names) + 1)]
+        for e in self.events:
+            e.record()                      # forces creation of the underlying cudaEvent_t
+        torch.cuda.synchronize()
+        self._handles = (C.c_void_p * len(self.events))(*[C.c_void_p(e.cuda_event) for e in self.events])
+
+    def __enter__(self):
+        load_library().sttm_set_stage_events(self._handles)
+        return self
+
+    def __exit__(self, *exc):
+        load_library().sttm_set_stage_events(None)
+
+    def stage_ms(self):
+        """Call after a synchronize: milliseconds of every stage of the last call."""
+        return {n: self.events[i].elapsed_time(self.events[i + 1]) for i, n in enumerate(self.names)}

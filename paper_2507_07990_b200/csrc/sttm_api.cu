@@ -17,6 +17,14 @@ using namespace sttm;
 constexpr int kSmCount = 148;   // B200; the library is built for sm_100a only
 
 thread_local int g_launches = 0;
+thread_local cudaEvent_t* g_stage_events = nullptr;   // when set: event i is recorded after stage i-1
+
+constexpr int kStageCount = 5;
+const char* const kStageNames[kStageCount] = {"spatial", "temporal+roots", "ordering", "accumulate", "combine"};
+
+inline void mark_stage(int boundary, cudaStream_t st) {
+    if (g_stage_events != nullptr) cudaEventRecord(g_stage_events[boundary], st);
+}
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
@@ -186,13 +194,16 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
         (OutT*)out, capacity, weight_mode);
     sttm_status s = launched();
     if (s != STTM_OK) return s;
+    mark_stage(4, st);
     k_combine<OutT><<<kSmCount * 2, 256, 0, st>>>(g, pl.Tc, (const long long*)(ws + pl.vid_off),
                                                  (const int32_t*)(ws + pl.span_off),
                                                  (const int32_t*)(ws + pl.row_anchor),
                                                  (const int32_t*)(ws + pl.row_last_t),
                                                  (const int32_t*)(ws + pl.row_weight),
                                                  (const float*)(ws + pl.partial), (OutT*)out, capacity);
-    return launched();
+    s = launched();
+    mark_stage(5, st);
+    return s;
 }
 
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
@@ -257,6 +268,12 @@ int sttm_sims_per_frame(int H, int W, int lv1) {
 
 int sttm_last_launch_count(void) { return g_launches; }
 
+int sttm_stage_count(void) { return kStageCount; }
+
+const char* sttm_stage_name(int i) { return i >= 0 && i < kStageCount ? kStageNames[i] : ""; }
+
+void sttm_set_stage_events(void** events) { g_stage_events = (cudaEvent_t*)events; }
+
 sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
                          int8_t* cover_level, int32_t* frame_counts, float* spatial_sims, void* stream) {
     Plan pl;
@@ -301,13 +318,16 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
     g_launches = 0;
 
     STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.zero_begin, 0, pl.zero_end - pl.zero_begin, st));
+    mark_stage(0, st);
     int8_t* cover = (int8_t*)(ws + pl.cover);
     int32_t* link = (int32_t*)(ws + pl.link);
     int32_t* root = (int32_t*)(ws + pl.root);
     s = run_spatial(feats, p, pl, ws, cover, (int32_t*)(ws + pl.frame_counts), nullptr, st);
     if (s != STTM_OK) return s;
+    mark_stage(1, st);
     s = run_temporal(feats, p, pl, ws, cover, link, root, nullptr, device_status, st);
     if (s != STTM_OK) return s;
+    mark_stage(2, st);
 
     int32_t* frame_roots = (int32_t*)(ws + pl.frame_roots);
     int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
@@ -330,6 +350,7 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
                                                      (const int32_t*)(ws + pl.row_last_t),
                                                      (int32_t*)(ws + pl.span_off), (int32_t*)(ws + pl.span_total));
     if ((s = launched()) != STTM_OK) return s;
+    mark_stage(3, st);
 
     return by_levels_dtype(g.L, p->in_dtype, [&](auto lv, auto* tag) {
         using T = std::remove_const_t<std::remove_pointer_t<decltype(tag)>>;

@@ -10,16 +10,15 @@ MARGIN = 1e-4
 
 def _pick(values, quantile, margin=MARGIN):
     """A threshold near the given quantile of `values` that keeps `margin` distance from
-    every value: the midpoint of the widest gap among the 40 gaps nearest the quantile."""
+    every value: the midpoint of the gap (wider than 2.2 * margin) nearest to the quantile."""
     s = np.unique(np.asarray(values, dtype=np.float64).ravel())
-    if len(s) == 0:
-        return 0.5
-    k = int(np.clip(round(quantile * (len(s) - 1)), 0, len(s) - 1))
-    lo, hi = max(0, k - 20), min(len(s) - 1, k + 20)
-    d = np.diff(s[lo:hi + 1])
-    if len(d) == 0 or d.max() < 2.2 * margin:
+    if len(s) < 2:
+        return 0.5 if len(s) == 0 else float(s[0]) - 0.01
+    k = int(np.clip(round(quantile * (len(s) - 1)), 0, len(s) - 2))
+    wide = np.nonzero(np.diff(s) >= 2.2 * margin)[0]
+    if len(wide) == 0:
         return None
-    i = int(np.argmax(d)) + lo
+    i = int(wide[np.argmin(np.abs(wide - k))])
     return float((s[i] + s[i + 1]) / 2)
 
 

@@ -165,7 +165,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    binding.load_library()
+    binding.load_library().sttm_set_tuning(*[int(v) for v in args.tuning.split(",")])
 
     cfg, spec, th, key = workload_setup(args.workload)
     N = spec.tokens
@@ -229,8 +229,13 @@ def run_ours(args):
     out_bytes = count * spec.D * 2
     id_bytes = count * 4
     path_bytes = in_bytes + out_bytes + id_bytes
-    # algorithmic bytes per launch of each feature-touching stage
-    stage_bytes = {"spatial": in_bytes, "temporal+roots": in_bytes, "accumulate": in_bytes + out_bytes}
+    # algorithmic bytes per launch of each feature-touching stage: every stage of the three-pass
+    # kernels reads the input once; the fused kernel reads it once and writes every output row once
+    # (to its staging place), the gather moves every output row once more
+    if lib.sttm_last_path() == 1:
+        stage_bytes = {"fused": in_bytes + out_bytes, "gather": 2 * out_bytes}
+    else:
+        stage_bytes = {"spatial": in_bytes, "temporal+roots": in_bytes, "accumulate": in_bytes + out_bytes}
     dominant = max(stage_bytes, key=lambda n: stage_ms.get(n, 0.0))
     peak, peak_kind = measured_peak()
     achieved = stage_bytes[dominant] / (stage_ms[dominant] / 1e3) / 1e9
@@ -288,6 +293,8 @@ def main():
     ap.add_argument("--reference-frames", type=int, default=64,
                     help="frames per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tuning", default="0,0,0",
+                    help="path,cluster_size,frames_per_item for sttm_set_tuning (0 = library's choice)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

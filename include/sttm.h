@@ -150,7 +150,8 @@ int sttm_last_launch_count(void);
 
 /*
  * Per-stage timing of sttm_merge_ex for benchmarks.  The path runs as
- * sttm_stage_count() consecutive stages.  After sttm_set_stage_events(events), with
+ * sttm_stage_count() consecutive stages (their names depend on which kernels the last
+ * call ran, see sttm_last_path).  After sttm_set_stage_events(events), with
  * `events` a host array of sttm_stage_count()+1 cudaEvent_t handles created by the
  * caller, every sttm_merge_ex on this thread records events[i] on its stream before
  * stage i and events[i+1] after it.  Pass NULL to switch recording off (the default).
@@ -158,6 +159,20 @@ int sttm_last_launch_count(void);
 int sttm_stage_count(void);
 const char* sttm_stage_name(int i);
 void sttm_set_stage_events(void** events);
+
+/*
+ * Benchmark and test knobs; 0 leaves a choice to the library.
+ *   path             1: always the three-pass kernels, 2 or 0: the fused single-read kernel
+ *                    wherever it applies (bf16 input, D a multiple of 16, at most 64 tiles of
+ *                    4x4 cells per frame, D / cluster_size <= 1024)
+ *   cluster_size     CTAs that share one tile's channels (1, 2, 4 or 8)
+ *   frames_per_item  frames of one tile that one cluster processes in a row
+ * Not thread safe; affects later calls of every entry point.
+ */
+void sttm_set_tuning(int path, int cluster_size, int frames_per_item);
+
+/* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 fused. */
+int sttm_last_path(void);
 
 const char* sttm_status_string(sttm_status s);
 

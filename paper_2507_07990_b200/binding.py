@@ -25,7 +25,7 @@ STATUS_NAMES = ["ok", "bad argument", "unsupported shape", "workspace too small"
 EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame", "sttm_spatial",
            "sttm_temporal", "sttm_merge_ex", "sttm_merge", "sttm_merge_host", "sttm_release_cache",
            "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
-           "sttm_set_stage_events"]
+           "sttm_set_stage_events", "sttm_set_tuning", "sttm_last_path"]
 
 
 class SttmParams(C.Structure):
@@ -82,6 +82,10 @@ def load_library(path: Optional[str] = None):
     lib.sttm_stage_name.restype = C.c_char_p
     lib.sttm_set_stage_events.argtypes = [C.POINTER(C.c_void_p)]
     lib.sttm_set_stage_events.restype = None
+    lib.sttm_set_tuning.argtypes = [C.c_int, C.c_int, C.c_int]
+    lib.sttm_set_tuning.restype = None
+    lib.sttm_last_path.argtypes = []
+    lib.sttm_last_path.restype = C.c_int
     lib.sttm_status_string.argtypes = [C.c_int]
     lib.sttm_status_string.restype = C.c_char_p
     if path == _build.LIB_PATH:

@@ -5,10 +5,12 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 
 #include "sttm_kernels.cuh"
+#include "sttm_fused.cuh"
 
 namespace {
 
@@ -20,7 +22,10 @@ thread_local int g_launches = 0;
 thread_local cudaEvent_t* g_stage_events = nullptr;   // when set: event i is recorded after stage i-1
 
 constexpr int kStageCount = 5;
-const char* const kStageNames[kStageCount] = {"spatial", "temporal+roots", "ordering", "accumulate", "combine"};
+const char* const kStageNames[2][kStageCount] = {
+    {"spatial", "temporal+roots", "ordering", "accumulate", "combine"},
+    {"fused", "roots", "ordering", "gather", "-"}};
+thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: fused kernel
 
 inline void mark_stage(int boundary, cudaStream_t st) {
     if (g_stage_events != nullptr) cudaEventRecord(g_stage_events[boundary], st);
@@ -28,16 +33,76 @@ inline void mark_stage(int boundary, cudaStream_t st) {
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
+// Launch shape of the fused kernel for one problem; ok == false: the three-pass kernels run.
+struct FusedPlan {
+    bool ok;
+    int C, S, Wn, NM, R, row_bytes, slot_bytes, F, nseg, nitems, ntiles, Wt;
+    size_t smem;
+    unsigned char tile_order[kMaxTiles];
+};
+
 struct Plan {
     Geo g;
     int Tc, nchunk, nslice;
     long long cells;          // B*N
     long long partial_slots;
+    FusedPlan f;
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
-        frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status,
-        zero_end, partial, total;
+        frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
+        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_next, total;
 };
+
+// benchmark / test knobs (sttm_set_tuning): 0 = choose automatically
+int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0;
+
+constexpr size_t kMaxSmem = 232448;   // 227 KB per CTA on sm_100
+
+void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
+    f->ok = false;
+    if (g_tune_path == 1) return;
+    if (p->in_dtype != STTM_BF16 || g.D % 16 != 0) return;
+    f->Wt = (g.W + 3) / 4;
+    f->ntiles = ((g.H + 3) / 4) * f->Wt;
+    if (f->ntiles > kMaxTiles) return;
+    int C = 0;
+    for (int c = 1; c <= kMaxCluster; c *= 2) {
+        if (g_tune_cluster && c != g_tune_cluster) continue;
+        if (g.D % (16 * c) == 0 && g.D / c <= 64 * kFusedMaxWorkerWarps) { C = c; break; }
+    }
+    if (C == 0) return;
+    f->C = C;
+    f->S = g.D / C;
+    f->Wn = (f->S + 63) / 64;
+    f->NM = std::min(4, f->Wn);
+    f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
+    f->slot_bytes = 16 * f->row_bytes;
+    const size_t fixed = (size_t)f->NM * kGramVals * 4 + (size_t)2 * C * kGramVals * 4 + kGramVals * 4 + 512 * 4 +
+                         32 * 4 + kRecRing * sizeof(FrameRec) + 16 * 8 + 64;
+    int R = (int)((kMaxSmem - fixed) / f->slot_bytes);
+    R = std::min(R, 8);
+    if (R < 4) return;
+    f->R = R;
+    f->smem = (size_t)R * f->slot_bytes + fixed;
+    // frames per item: about four items per resident cluster, counted in full tiles
+    const double tiles_equiv = (double)g.HW / 16.0;
+    const double want = (double)g.B * g.T * tiles_equiv / (4.0 * (kSmCount / C));
+    int F = g_tune_seg > 0 ? g_tune_seg : std::max(8, std::min((int)std::ceil(want), 256));
+    F = std::min(F, g.T);
+    f->F = F;
+    f->nseg = (g.T + F - 1) / F;
+    f->nitems = g.B * f->ntiles * f->nseg;
+    // tiles with more cells inside the grid first
+    int cells[kMaxTiles];
+    for (int t = 0; t < f->ntiles; t++) {
+        const int y0 = (t / f->Wt) * 4, x0 = (t % f->Wt) * 4;
+        cells[t] = std::min(4, g.H - y0) * std::min(4, g.W - x0);
+        f->tile_order[t] = (unsigned char)t;
+    }
+    std::stable_sort(f->tile_order, f->tile_order + f->ntiles,
+                     [&](unsigned char a, unsigned char b) { return cells[a] > cells[b]; });
+    f->ok = true;
+}
 
 int levels_of(int H, int W, int lv1, int* H1, int* W1, int* Hc, int* Wc) {
     int L = 1, h = H, w = W;
@@ -101,8 +166,21 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
     pl->row_last_t = take((size_t)pl->cells * 4);
     pl->span_total = take(4);
     pl->status = take(4);
+    pl->queue = take(4);
     pl->zero_end = o;
     pl->partial = take((size_t)pl->partial_slots * g.D * sizeof(float));
+    plan_fused(p, g, &pl->f);
+    pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = pl->piece_next = o;
+    if (pl->f.ok) {
+        const size_t out_elt = p->out_dtype == STTM_BF16 ? 2 : 4;
+        pl->ones_begin = o;
+        pl->row_head = take((size_t)pl->cells * 4);
+        pl->ones_end = o;
+        pl->staging = take((size_t)pl->cells * g.D * out_elt);
+        pl->pieces = take((size_t)pl->f.nitems * kPieceSlots * g.D * sizeof(float));
+        pl->piece_meta = take((size_t)pl->f.nitems * kPieceSlots * sizeof(int2));
+        pl->piece_next = take((size_t)pl->f.nitems * kPieceSlots * 4);
+    }
     pl->total = o;
     return STTM_OK;
 }
@@ -206,6 +284,87 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
     return s;
 }
 
+// Resident clusters of the fused kernel for a launch shape (cached); falls back to SMs / C.
+int fused_resident_clusters(const FusedPlan& f) {
+    static int cached[kMaxCluster + 1][kFusedMaxWorkerWarps + 2];
+    static size_t cached_smem[kMaxCluster + 1][kFusedMaxWorkerWarps + 2];
+    int& slot = cached[f.C][f.Wn];
+    if (slot > 0 && cached_smem[f.C][f.Wn] == f.smem) return slot;
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kSmCount / f.C * f.C);
+    cfg.blockDim = dim3((f.Wn + 1) * 32);
+    cfg.dynamicSmemBytes = f.smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    if (cudaOccupancyMaxActiveClusters(&n, k_fused, &cfg) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        n = kSmCount / f.C;
+    }
+    slot = n;
+    cached_smem[f.C][f.Wn] = f.smem;
+    return n;
+}
+
+sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, char* ws, int32_t* device_status,
+                      cudaStream_t st) {
+    const Geo g = pl.g;
+    const FusedPlan& f = pl.f;
+    static size_t configured_smem = 0;
+    if (configured_smem < f.smem) {
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        configured_smem = kMaxSmem;
+    }
+    FusedParams fp = {};
+    fp.feats = (const __nv_bfloat16*)feats;
+    fp.B = g.B; fp.T = g.T; fp.H = g.H; fp.W = g.W; fp.D = g.D; fp.L = g.L;
+    fp.HW = g.HW; fp.N = g.N;
+    fp.Wt = f.Wt; fp.ntiles = f.ntiles;
+    fp.C = f.C; fp.S = f.S; fp.Wn = f.Wn; fp.NM = f.NM;
+    fp.row_bytes = f.row_bytes; fp.slot_bytes = f.slot_bytes; fp.R = f.R;
+    fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
+    fp.weight_mode = (int)p->wt;
+    fp.out_f32 = p->out_dtype == STTM_F32;
+    fp.cover = (int8_t*)(ws + pl.cover);
+    fp.link = (int32_t*)(ws + pl.link);
+    fp.staging = ws + pl.staging;
+    fp.pieces = (float*)(ws + pl.pieces);
+    fp.piece_meta = (int2*)(ws + pl.piece_meta);
+    fp.queue = (int*)(ws + pl.queue);
+    fp.status = device_status;
+    std::memcpy(fp.tile_order, f.tile_order, sizeof(fp.tile_order));
+    Taus taus;
+    fill_taus(p, &taus);
+
+    const int nclusters = std::min(f.nitems, fused_resident_clusters(f));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(nclusters * f.C);
+    cfg.blockDim = dim3((f.Wn + 1) * 32);
+    cfg.dynamicSmemBytes = f.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused, fp, taus));
+    g_launches++;
+    return STTM_OK;
+}
+
+template <typename OutT>
+sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacity, cudaStream_t st) {
+    const Geo g = pl.g;
+    k_gather<OutT><<<kSmCount * 8, 256, 0, st>>>(g, (const long long*)(ws + pl.vid_off),
+                                                 (const int32_t*)(ws + pl.row_anchor),
+                                                 (const int32_t*)(ws + pl.row_head),
+                                                 (const int32_t*)(ws + pl.piece_next),
+                                                 (const int32_t*)(ws + pl.row_weight), (const OutT*)(ws + pl.staging),
+                                                 (const float*)(ws + pl.pieces), (OutT*)out, capacity);
+    return launched();
+}
+
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
 
 // cached buffers for sttm_merge / sttm_merge_host, one set per device
@@ -270,9 +429,17 @@ int sttm_last_launch_count(void) { return g_launches; }
 
 int sttm_stage_count(void) { return kStageCount; }
 
-const char* sttm_stage_name(int i) { return i >= 0 && i < kStageCount ? kStageNames[i] : ""; }
+const char* sttm_stage_name(int i) { return i >= 0 && i < kStageCount ? kStageNames[g_last_path][i] : ""; }
+
+int sttm_last_path(void) { return g_last_path; }
 
 void sttm_set_stage_events(void** events) { g_stage_events = (cudaEvent_t*)events; }
+
+void sttm_set_tuning(int path, int cluster_size, int frames_per_item) {
+    g_tune_path = path;
+    g_tune_cluster = cluster_size;
+    g_tune_seg = frames_per_item;
+}
 
 sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
                          int8_t* cover_level, int32_t* frame_counts, float* spatial_sims, void* stream) {
@@ -318,10 +485,54 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
     g_launches = 0;
 
     STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.zero_begin, 0, pl.zero_end - pl.zero_begin, st));
-    mark_stage(0, st);
     int8_t* cover = (int8_t*)(ws + pl.cover);
     int32_t* link = (int32_t*)(ws + pl.link);
     int32_t* root = (int32_t*)(ws + pl.root);
+    g_last_path = pl.f.ok ? 1 : 0;
+    if (pl.f.ok) {
+        // single-read path: fused kernel, roots, ordering, gather
+        STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.ones_begin, 0xff, pl.ones_end - pl.ones_begin, st));
+        mark_stage(0, st);
+        s = run_fused(feats, p, pl, ws, device_status, st);
+        if (s != STTM_OK) return s;
+        mark_stage(1, st);
+        int max_rounds = 2;
+        while ((1 << (max_rounds - 2)) < g.T) max_rounds++;
+        if (g.L == 1) k_roots<1><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, device_status, max_rounds);
+        else if (g.L == 2) k_roots<2><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, device_status, max_rounds);
+        else k_roots<3><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, device_status, max_rounds);
+        if ((s = launched()) != STTM_OK) return s;
+        mark_stage(2, st);
+        int32_t* frame_roots = (int32_t*)(ws + pl.frame_roots);
+        int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
+        long long* vid_off = (long long*)(ws + pl.vid_off);
+        int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
+        int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
+        k_frame_roots<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_roots);
+        if ((s = launched()) != STTM_OK) return s;
+        k_scan_frames<<<1, 1024, 0, st>>>(g, frame_roots, frame_base, out_count, vid_off, out_offsets);
+        if ((s = launched()) != STTM_OK) return s;
+        k_rows<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_base, vid_off, row_at_root, row_anchor, out_pos,
+                                          p->out_capacity_rows, (int)p->pos, device_status);
+        if ((s = launched()) != STTM_OK) return s;
+        if (merge_map != nullptr) {
+            k_merge_map<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, root, row_at_root, merge_map);
+            if ((s = launched()) != STTM_OK) return s;
+        }
+        const int npieces = pl.f.nitems * kPieceSlots;
+        k_piece_link<<<blocks_for(npieces, 256), 256, 0, st>>>(g, npieces, (const int2*)(ws + pl.piece_meta), root,
+                                                              row_at_root, vid_off, (int32_t*)(ws + pl.row_head),
+                                                              (int32_t*)(ws + pl.piece_next),
+                                                              (int32_t*)(ws + pl.row_weight));
+        if ((s = launched()) != STTM_OK) return s;
+        mark_stage(3, st);
+        s = p->out_dtype == STTM_BF16 ? launch_gather<__nv_bfloat16>(pl, ws, out_feats, p->out_capacity_rows, st)
+                                      : launch_gather<float>(pl, ws, out_feats, p->out_capacity_rows, st);
+        mark_stage(4, st);
+        mark_stage(5, st);
+        return s;
+    }
+    mark_stage(0, st);
     s = run_spatial(feats, p, pl, ws, cover, (int32_t*)(ws + pl.frame_counts), nullptr, st);
     if (s != STTM_OK) return s;
     mark_stage(1, st);

@@ -13,6 +13,18 @@ from tests import helpers
 
 pytestmark = pytest.mark.gpu
 
+# (path, cluster size, frames per item) for sttm_set_tuning: the library's own choice, the
+# three-pass kernels, and fused launches that force clusters and many item borders
+TUNINGS = {"auto": (0, 0, 0), "threepass": (1, 0, 0), "c1f3": (2, 1, 3), "c2f2": (2, 2, 2), "c4f5": (2, 4, 5),
+           "c8f1": (2, 8, 1)}
+
+
+@pytest.fixture(params=list(TUNINGS), ids=list(TUNINGS))
+def tuning(request):
+    binding.load_library().sttm_set_tuning(*TUNINGS[request.param])
+    yield request.param
+    binding.load_library().sttm_set_tuning(0, 0, 0)
+
 
 def run_and_compare(video_np, tau_s, tau_t, lv1=4, out_dtype=torch.float32, wt=binding.W_NODE,
                     pos=binding.POS_SURVIVED, stages=True):
@@ -76,7 +88,7 @@ SHAPES = [  # T, H, W, D, lv1, dtype
 
 @pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "T%dH%dW%dD%dlv%d%s" % s)
 @pytest.mark.parametrize("q_s,q_t", [(0.5, 0.5), (0.15, 0.8), (0.9, 0.2)])
-def test_parity_small(shape, q_s, q_t):
+def test_parity_small(shape, q_s, q_t, tuning):
     T, H, W, D, lv1, dtype = shape
     done = 0
     for seed in range(3):
@@ -91,7 +103,7 @@ def test_parity_small(shape, q_s, q_t):
     assert done >= 1, "no seed gave thresholds with a margin"
 
 
-def test_parity_weight_and_position_modes():
+def test_parity_weight_and_position_modes(tuning):
     spec = helpers.small_spec(7, 6, 13, 13, 256)
     video = inputs.make_video(spec)
     tau_s, tau_t = helpers.safe_thresholds(video, 0.4, 0.5)
@@ -99,7 +111,7 @@ def test_parity_weight_and_position_modes():
     run_and_compare(video, tau_s, tau_t, pos=binding.POS_REASSIGNED, stages=False)
 
 
-def test_degenerate_thresholds():
+def test_degenerate_thresholds(tuning):
     spec = helpers.small_spec(8, 12, 13, 13, 128)
     video = inputs.make_video(spec)
     for tau_s, tau_t in [(2.0, 2.0), (-2.0, 2.0), (2.0, -2.0), (-2.0, -2.0)]:
@@ -117,7 +129,7 @@ def test_tiny_config_fixed_thresholds():
         assert ref.count == expect
 
 
-def test_long_chains_cross_time_chunks():
+def test_long_chains_cross_time_chunks(tuning):
     """A static video: every chain spans all frames, so rows are summed across the
     averaging kernel's time chunks."""
     spec = helpers.small_spec(9, 96, 13, 13, 128, p_static=0.97)
@@ -128,7 +140,7 @@ def test_long_chains_cross_time_chunks():
     assert ref.out_members.max() >= 40
 
 
-def test_batch_with_per_video_thresholds():
+def test_batch_with_per_video_thresholds(tuning):
     specs = [helpers.small_spec(20 + v, 8, 13, 13, 256, p_static=p) for v, p in enumerate((0.9, 0.5, 0.2))]
     videos = [inputs.make_video(s) for s in specs]
     taus = [helpers.safe_thresholds(v, 0.5, 0.5) for v in videos]

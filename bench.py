@@ -271,6 +271,7 @@ def run_ours(args):
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": workload_config(args.workload, spec, th, key), "out_rows": count,
+                "launch_shape": binding.sttm_fused_launch_shape(plan.problem),
                 "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "clocks": clocks}
         if world == 1 and not args.no_cpu_baseline:

@@ -174,6 +174,15 @@ void sttm_set_tuning(int path, int cluster_size, int frames_per_item);
 /* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 fused. */
 int sttm_last_path(void);
 
+/*
+ * Launch shape the fused kernel would get for these params (host pointers; queries the
+ * current device for the number of clusters that fit).  shape[10] = {cluster size, channels
+ * per CTA, threads per CTA, ring slots, dynamic shared memory bytes, frames per item, items,
+ * clusters that can be resident, clusters launched, tensor-core warps}.  Returns 1, or 0
+ * when the fused kernel does not apply to the params.
+ */
+int sttm_fused_launch_shape(const sttm_params* p, int* shape);
+
 const char* sttm_status_string(sttm_status s);
 
 #ifdef __cplusplus

@@ -77,8 +77,8 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     f->NM = std::min(4, f->Wn);
     f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
     f->slot_bytes = 16 * f->row_bytes;
-    const size_t fixed = (size_t)f->NM * kGramVals * 4 + (size_t)2 * C * kGramVals * 4 + kGramVals * 4 + 512 * 4 +
-                         32 * 4 + kRecRing * sizeof(FrameRec) + 16 * 8 + 64;
+    const size_t fixed = (size_t)f->NM * kGramVals * 4 + (size_t)2 * C * kSumVals * 4 + 32 * 4 + sizeof(SlotTable) +
+                         kRecRing * sizeof(FrameRec) + 16 * 8 + 64;
     int R = (int)((kMaxSmem - fixed) / f->slot_bytes);
     R = std::min(R, 8);
     if (R < 4) return;
@@ -299,7 +299,9 @@ int fused_resident_clusters(const FusedPlan& f) {
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    if (cudaOccupancyMaxActiveClusters(&n, k_fused, &cfg) != cudaSuccess || n < 1) {
+    const cudaError_t e = cfg.blockDim.x <= 480 ? cudaOccupancyMaxActiveClusters(&n, k_fused<480>, &cfg)
+                                                : cudaOccupancyMaxActiveClusters(&n, k_fused<kFusedMaxThreads>, &cfg);
+    if (e != cudaSuccess || n < 1) {
         cudaGetLastError();
         n = kSmCount / f.C;
     }
@@ -312,10 +314,12 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
                       cudaStream_t st) {
     const Geo g = pl.g;
     const FusedPlan& f = pl.f;
-    static size_t configured_smem = 0;
-    if (configured_smem < f.smem) {
-        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-        configured_smem = kMaxSmem;
+    static bool configured = false;
+    if (!configured) {
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<480>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<kFusedMaxThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)kMaxSmem));
+        configured = true;
     }
     FusedParams fp = {};
     fp.feats = (const __nv_bfloat16*)feats;
@@ -329,6 +333,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.out_f32 = p->out_dtype == STTM_F32;
     fp.cover = (int8_t*)(ws + pl.cover);
     fp.link = (int32_t*)(ws + pl.link);
+    fp.chain_key = (int32_t*)(ws + pl.cell_row);       // the three-pass kernels' cell_row array is free here
     fp.staging = ws + pl.staging;
     fp.pieces = (float*)(ws + pl.pieces);
     fp.piece_meta = (int2*)(ws + pl.piece_meta);
@@ -348,7 +353,9 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused, fp, taus));
+    // two builds of the same kernel: up to 15 warps may use 128 registers per thread, up to 17 only 96
+    if (cfg.blockDim.x <= 480) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<480>, fp, taus));
+    else STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<kFusedMaxThreads>, fp, taus));
     g_launches++;
     return STTM_OK;
 }
@@ -433,6 +440,17 @@ const char* sttm_stage_name(int i) { return i >= 0 && i < kStageCount ? kStageNa
 
 int sttm_last_path(void) { return g_last_path; }
 
+int sttm_fused_launch_shape(const sttm_params* p, int* shape) {
+    Plan pl;
+    if (shape == nullptr || make_plan(p, &pl) != STTM_OK || !pl.f.ok) return 0;
+    const FusedPlan& f = pl.f;
+    const int resident = fused_resident_clusters(f);
+    const int v[10] = {f.C, f.S, (f.Wn + 1) * 32, f.R, (int)f.smem, f.F, f.nitems, resident,
+                       std::min(f.nitems, resident), f.NM};
+    std::memcpy(shape, v, sizeof(v));
+    return 1;
+}
+
 void sttm_set_stage_events(void** events) { g_stage_events = (cudaEvent_t*)events; }
 
 void sttm_set_tuning(int path, int cluster_size, int frames_per_item) {
@@ -496,11 +514,8 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
         s = run_fused(feats, p, pl, ws, device_status, st);
         if (s != STTM_OK) return s;
         mark_stage(1, st);
-        int max_rounds = 2;
-        while ((1 << (max_rounds - 2)) < g.T) max_rounds++;
-        if (g.L == 1) k_roots<1><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, device_status, max_rounds);
-        else if (g.L == 2) k_roots<2><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, device_status, max_rounds);
-        else k_roots<3><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, device_status, max_rounds);
+        k_resolve_roots<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, pl.f.nseg + 1, (const int32_t*)(ws + pl.cell_row),
+                                                                  root, device_status);
         if ((s = launched()) != STTM_OK) return s;
         mark_stage(2, st);
         int32_t* frame_roots = (int32_t*)(ws + pl.frame_roots);

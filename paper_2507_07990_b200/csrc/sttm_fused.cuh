@@ -14,7 +14,10 @@
 //      cosine of Sections 3.2 and 3.3 is a short linear combination of entries of G and C
 //      because parents are averages of cells.  The products of bf16 inputs are exact and
 //      the sums are kept in fp32.
-//   2. partial matrices are added across warps (shared memory) and across the cluster
+//   2. worker threads contract the partial matrices to the 128 numbers the decisions need
+//      (per cell: its squared norm, its products with its parent and with the coarsest node,
+//      and its products with the nodes of the previous frame that contain it or that it
+//      contains) and add them across warps (shared memory) and across the cluster
 //      (distributed shared memory), in a fixed order.
 //   3. one decision warp per CTA turns the totals into the cover map, the links and the
 //      bookkeeping of the running chains (every CTA of the cluster repeats this on the
@@ -28,6 +31,7 @@
 #pragma once
 
 #include "sttm_device.cuh"
+#include "sttm_kernels.cuh"
 
 namespace sttm {
 
@@ -35,6 +39,7 @@ constexpr int kMaxTiles = 64;
 constexpr int kMaxCluster = 8;
 constexpr int kRecRing = 4;
 constexpr int kGramVals = 512;          // G (16x16) then C (16x16)
+constexpr int kSumVals = 128;           // 8 numbers per cell, see combine_sums()
 constexpr int kPieceSlots = 32;         // per item: 16 keyed by a cell of the frame before the item, 16 by chain slot
 constexpr int kFusedMaxWorkerWarps = 16;
 constexpr int kFusedMaxThreads = (kFusedMaxWorkerWarps + 1) * 32;
@@ -62,6 +67,7 @@ struct FusedParams {
     int weight_mode, out_f32;
     int8_t* cover;
     int32_t* link;
+    int32_t* chain_key;      // [B*N] per cell: root cell id of its chain as far as the item knows it
     void* staging;           // [B*N][D] rows of the output dtype
     float* pieces;           // [nitems][kPieceSlots][D]
     int2* piece_meta;        // [nitems][kPieceSlots] {key cell id or -1, weight}
@@ -103,8 +109,8 @@ __device__ __forceinline__ uint32_t cluster_rank() {
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     uint32_t out;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(addr), "r"(rank));
@@ -117,7 +123,7 @@ __device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void named_sync(int id, int count) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+    asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -208,64 +214,90 @@ struct ItemGeo {
     int nvalid;
 };
 
-// What the decision warp carries from frame to frame.
+// What the decision warp carries from frame to frame (lane c < 16: cell c of the tile).
 struct DecState {
-    int prev_lv, prev_slot;      // lane c < 16: level / chain slot of the kept node covering cell c (previous frame)
+    int prev_lv, prev_slot;      // level / chain slot of the kept node covering the cell in the previous frame
     float prev_nk;               // its squared norm
-    int sl_key, sl_weight, sl_virtual, sl_cell;   // lane s < 16: chain slot s
     uint32_t active;             // uniform: slots in use
 };
 
+// Chain slots of the decision warp (shared memory, private to it).
+struct SlotTable {
+    int key[16], weight[16], virt[16], cell[16];
+};
+
+// The 8 numbers of cell c that the decisions need, as linear functions of the tile's Gram
+// matrix G = X_t X_t^T and cross matrix Cm = X_t X_{t-1}^T (row: cell of frame t).  With
+// q(c) the cell's 2x2 block, w1 / w2 the averaging weights of level 1 / level 2:
+//   k=0  |x_c|^2                       k=1  x_c . parent(c)            k=2  x_c . top
+//   k=3  x_c(t) . x_c(t-1)             k=4  x_c(t) . parent(c)(t-1)    k=5  x_c(t) . top(t-1)
+//   k=6  parent(c)(t) . x_c(t-1)       k=7  top(t) . x_c(t-1)
+// `m` points at NM partial matrices of kGramVals floats each; they are added in order.
+__device__ __forceinline__ float combine_sums(const float* m, int NM, int c, int k, const float* W1s,
+                                              const float* W2s) {
+    const int qb = tile_anchor(c, 1);
+    float acc = 0.f;
+    for (int w = 0; w < NM; w++) {
+        const float* G = m + w * kGramVals;
+        const float* Cm = G + 256;
+        float v = 0.f;
+        switch (k) {
+            case 0: v = G[c * 16 + c]; break;
+            case 1: v = ((G[c * 16 + qb] + G[c * 16 + qb + 1]) + (G[c * 16 + qb + 4] + G[c * 16 + qb + 5])) * W1s[c]; break;
+            case 2:
+#pragma unroll
+                for (int i = 0; i < 16; i++) v = fmaf(W2s[i], G[c * 16 + i], v);
+                break;
+            case 3: v = Cm[c * 16 + c]; break;
+            case 4: v = ((Cm[c * 16 + qb] + Cm[c * 16 + qb + 1]) + (Cm[c * 16 + qb + 4] + Cm[c * 16 + qb + 5])) * W1s[c]; break;
+            case 5:
+#pragma unroll
+                for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[c * 16 + i], v);
+                break;
+            case 6: v = ((Cm[qb * 16 + c] + Cm[(qb + 1) * 16 + c]) + (Cm[(qb + 4) * 16 + c] + Cm[(qb + 5) * 16 + c])) * W1s[c]; break;
+            default:
+#pragma unroll
+                for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[i * 16 + c], v);
+                break;
+        }
+        acc += v;
+    }
+    return acc;
+}
+
+// sum over the four cells of the lane's 2x2 block (lanes of the same half warp)
+__device__ __forceinline__ float quad_sum(float v, int lane) {
+    const int hb = lane & 16, qb = tile_anchor(lane & 15, 1);
+    return (__shfl_sync(0xffffffffu, v, hb + qb) + __shfl_sync(0xffffffffu, v, hb + qb + 1)) +
+           (__shfl_sync(0xffffffffu, v, hb + qb + 4) + __shfl_sync(0xffffffffu, v, hb + qb + 5));
+}
+
 // ---------------------------------------------------------------------------------
-// Decisions of one frame (Sections 3.2 and 3.3) from the tile's Gram and cross matrices.
-// All 32 lanes run it; lane and lane+16 work on the same cell c = lane & 15.
+// Decisions of one frame (Sections 3.2 and 3.3) from the cluster totals of the 8 numbers
+// per cell (v[0..7], lane c = cell c; lanes 16..31 mirror lanes 0..15).
 // ---------------------------------------------------------------------------------
 __device__ __forceinline__ void decide_frame(const FusedParams& p, const ItemGeo& it, int j, float tau_s, float tau_t,
-                                             const float* xch, float* dG, float* dY, const float* W1s,
-                                             const float* W2s, DecState& st, FrameRec* rec, uint32_t rank, int lane) {
+                                             const float (&v)[8], const float* W1s, const float* W2s, DecState& st,
+                                             SlotTable* tab, FrameRec* rec, uint32_t rank, int lane) {
     const unsigned full = 0xffffffffu;
     const int c = lane & 15;
+    const bool low = lane < 16;
     const int L = p.L;
     const int t = it.tstart + j;
     const bool has_prev = j > 0;
     const bool is_halo = it.halo && j == 0;
     const bool is_last = j == it.n - 1;
-
-    for (int v = lane; v < kGramVals; v += 32) {
-        float s = 0.f;
-        for (int r = 0; r < p.C; r++) s += xch[r * kGramVals + v];
-        dG[v] = s;
-    }
-    __syncwarp();
-    const float* G = dG;
-    const float* Cm = dG + 256;
-
     const bool valid = (it.vmask >> c) & 1u;
     const uint32_t qm = quad_mask(c);
-    const int qb = tile_anchor(c, 1);
     const float w1 = W1s[c], w2 = W2s[c];
 
-    // Section 3.2: cosine of every node with its parent
-    const float* Gr = G + c * 16;
-    const float n0 = Gr[c];
-    float d0 = 0.f, rr = 0.f;
-    if (L >= 2) d0 = ((Gr[qb] + Gr[qb + 1]) + (Gr[qb + 4] + Gr[qb + 5])) * w1;      // x_c . parent
-    if (L == 3) {
-#pragma unroll
-        for (int k = 0; k < 16; k++) rr = fmaf(W2s[k], Gr[k], rr);                      // x_c . coarsest node
-    }
-    const int hb = lane & 16;
-    const float sd0 = (__shfl_sync(full, d0, hb + qb) + __shfl_sync(full, d0, hb + qb + 1)) +
-                      (__shfl_sync(full, d0, hb + qb + 4) + __shfl_sync(full, d0, hb + qb + 5));
-    const float srr = (__shfl_sync(full, rr, hb + qb) + __shfl_sync(full, rr, hb + qb + 1)) +
-                      (__shfl_sync(full, rr, hb + qb + 4) + __shfl_sync(full, rr, hb + qb + 5));
-    const float n1 = w1 * sd0;                  // |parent|^2
-    const float d1 = w1 * srr;                  // parent . coarsest node
-    const float n2 = half_warp_sum(w2 * rr);    // |coarsest node|^2
+    // Section 3.2: cosine of every node with its parent, then the coarse-to-fine search
+    const float n0 = v[0], d0 = v[1], rr = v[2];
+    const float n1 = w1 * quad_sum(d0, lane);          // |parent|^2
+    const float d1 = w1 * quad_sum(rr, lane);          // parent . top
+    const float n2 = half_warp_sum(w2 * rr);           // |top|^2
     const float s0 = cos_from(d0, n0, n1);
     const float s1 = cos_from(d1, n1, n2);
-
-    // coarse-to-fine search
     int lv = 0;
     if (L >= 2) {
         const bool p0 = !valid || s0 > tau_s;
@@ -282,32 +314,18 @@ __device__ __forceinline__ void decide_frame(const FusedParams& p, const ItemGeo
     }
     const float nk = lv == 0 ? n0 : (lv == 1 ? n1 : n2);
 
-    // Section 3.3: compare with the overlapping kept nodes of the previous frame
+    // Section 3.3: the node covering the cell against the overlapping kept node of the
+    // previous frame; a pair is evaluated at the top-left cell of its finer node
     int link_local = -1;
     if (has_prev) {
         const int lu = st.prev_lv;
-        float* Yr = dY + (lane >> 4) * 256 + c * 16;     // Y[a][u] = x_a(t) . node u(t-1), row a = c
-#pragma unroll
-        for (int k = 0; k < 16; k++) Yr[k] = 0.f;
-        for (int b = 0; b < 16; b++) {
-            const int lub = __shfl_sync(full, lu, b);
-            const int au = tile_anchor(b, lub);
-            const float wu = lub == 0 ? 1.f : (lub == 1 ? W1s[b] : W2s[b]);
-            Yr[au] = fmaf(wu, Cm[c * 16 + b], Yr[au]);
-        }
-        __syncwarp();
+        const float t11 = w1 * quad_sum(v[4], lane), t12 = w1 * quad_sum(v[5], lane);
+        const float t21 = w1 * quad_sum(v[7], lane), t22 = half_warp_sum(w2 * v[5]);
+        float dot;
+        if (lv == 0) dot = lu == 0 ? v[3] : (lu == 1 ? v[4] : v[5]);
+        else if (lv == 1) dot = lu == 0 ? v[6] : (lu == 1 ? t11 : t12);
+        else dot = lu == 0 ? v[7] : (lu == 1 ? t21 : t22);
         const bool rep = valid && tile_anchor(c, min(lv, lu)) == c;
-        float dot = 0.f;
-        if (rep) {
-            const int au = tile_anchor(c, lu), av = tile_anchor(c, lv);
-            const float* Y = dY + (lane >> 4) * 256;
-            for (int a = 0; a < 16; a++) {
-                if (tile_anchor(a, lv) == av) {
-                    const float wv = lv == 0 ? 1.f : (lv == 1 ? W1s[a] : W2s[a]);
-                    dot = fmaf(wv, Y[a * 16 + au], dot);
-                }
-            }
-        }
         const float s = cos_from(dot, nk, st.prev_nk);
         const bool pass = rep && s > tau_t;
         const uint32_t passm = __ballot_sync(full, pass) & 0xffffu;
@@ -317,113 +335,98 @@ __device__ __forceinline__ void decide_frame(const FusedParams& p, const ItemGeo
         link_local = cand ? tile_anchor(cstar, lu_star) : -1;
     }
 
-    if (rank == 0 && !is_halo && lane < 16 && valid) {
-        const long long gc = (long long)it.b * p.N + (long long)t * p.HW + (it.y0 + (c >> 2)) * p.W + it.x0 + (c & 3);
+    // chains: nodes with a link join the chain of their target; chains without a member in
+    // this frame have ended; the remaining nodes start new chains in free slots
+    const bool anchor = valid && tile_anchor(c, lv) == c;
+    const bool linked = anchor && link_local >= 0;
+    const bool fresh = anchor && link_local < 0;
+    const int slot_linked = __shfl_sync(full, st.prev_slot, link_local < 0 ? 0 : link_local);
+    const uint32_t memb = __reduce_or_sync(full, linked ? 1u << slot_linked : 0u);
+    const uint32_t dead = st.active & ~memb;
+    const uint32_t freem = ~memb & 0xffffu;
+    const uint32_t freshm = __ballot_sync(full, fresh && low);
+    const int slot_fresh = __fns(freem, 0, __popc(freshm & ((1u << c) - 1)) + 1);
+    const int node_slot = linked ? slot_linked : slot_fresh;
+    const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + tile_anchor(c, lv));
+    const int wint = p.weight_mode ? __popc(it.vmask & region_mask(c, lv)) : 1;
+    const long long gc = (long long)it.b * p.N + (long long)t * p.HW + (it.y0 + (c >> 2)) * p.W + it.x0 + (c & 3);
+
+    // chains that ended: lane s looks at slot s (before the slot is given away again)
+    const bool my_dead = low && ((dead >> lane) & 1u);
+    if (my_dead) {
+        const int at = __popc(dead & ((1u << lane) - 1));
+        if (tab->virt[lane]) {
+            const int pc = it.item * kPieceSlots + tab->cell[lane];
+            rec->pre[at] = FlushCmd{lane, 1, pc, 0.f};
+            if (rank == 0) p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
+        } else {
+            rec->pre[at] = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
+        }
+    }
+    __syncwarp();
+    if (low && fresh) {
+        tab->key[slot_fresh] = (int)gc;
+        tab->weight[slot_fresh] = is_halo ? 0 : wint;
+        tab->virt[slot_fresh] = is_halo ? 1 : 0;
+        tab->cell[slot_fresh] = c;
+    }
+    if (low && linked) atomicAdd(&tab->weight[slot_linked], wint);
+    const uint32_t anchorm = __ballot_sync(full, anchor && low);
+    if (low && anchor && !is_halo) {
+        const float wn = lv == 1 ? w1 * (float)wint : (float)wint;
+        rec->node[__popc(anchorm & ((1u << c) - 1))] = NodeCmd{c, lv, node_slot, wn};
+    }
+    const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
+    __syncwarp();
+
+    if (rank == 0 && !is_halo && low && valid) {
         p.cover[gc] = (int8_t)lv;
         p.link[gc] = link_local < 0 ? -1
                                     : (t - 1) * p.HW + (it.y0 + (link_local >> 2)) * p.W + it.x0 + (link_local & 3);
+        p.chain_key[gc] = tab->key[cur_slot] - it.b * p.N;
     }
-
-    // chains: nodes with a link join the chain of their target; chains without a member in
-    // this frame have ended; the remaining nodes start new chains
-    uint32_t memb = 0;
-    int cur_slot = 0, nn = 0;
-    for (int a = 0; a < 16; a++) {
-        const int lva = __shfl_sync(full, lv, a);
-        const int lka = __shfl_sync(full, link_local, a);
-        if (!((it.vmask >> a) & 1u) || tile_anchor(a, lva) != a || lka < 0) continue;
-        const int s = __shfl_sync(full, st.prev_slot, lka);
-        memb |= 1u << s;
-        if (tile_anchor(c, lva) == a) cur_slot = s;
-        const int wint = p.weight_mode ? __popc(it.vmask & region_mask(a, lva)) : 1;
-        if (lane == s) st.sl_weight += wint;
-        if (lane == 0) {
-            const float wn = lva == 1 ? W1s[a] * (float)wint : (float)wint;
-            rec->node[nn] = NodeCmd{a, lva, s, wn};
-        }
-        nn++;
-    }
-    int npre = 0;
-    for (uint32_t dead = st.active & ~memb; dead; dead &= dead - 1) {
-        const int s = __ffs(dead) - 1;
-        const int key = __shfl_sync(full, st.sl_key, s), wgt = __shfl_sync(full, st.sl_weight, s);
-        const int virt = __shfl_sync(full, st.sl_virtual, s), cell = __shfl_sync(full, st.sl_cell, s);
-        if (lane == 0) {
-            if (virt) {
-                rec->pre[npre] = FlushCmd{s, 1, it.item * kPieceSlots + cell, 0.f};
-                if (rank == 0) p.piece_meta[it.item * kPieceSlots + cell] = make_int2(key, wgt);
-            } else {
-                rec->pre[npre] = FlushCmd{s, 0, key, (float)wgt};
-            }
-        }
-        npre++;
-    }
-    uint32_t freem = ~memb & 0xffffu;
-    for (int a = 0; a < 16; a++) {
-        const int lva = __shfl_sync(full, lv, a);
-        const int lka = __shfl_sync(full, link_local, a);
-        if (!((it.vmask >> a) & 1u) || tile_anchor(a, lva) != a || lka >= 0) continue;
-        const int s = __ffs(freem) - 1;
-        freem &= ~(1u << s);
-        memb |= 1u << s;
-        if (tile_anchor(c, lva) == a) cur_slot = s;
-        const int wint = p.weight_mode ? __popc(it.vmask & region_mask(a, lva)) : 1;
-        if (lane == s) {
-            st.sl_key = (int)((long long)it.b * p.N + (long long)t * p.HW + (it.y0 + (a >> 2)) * p.W + it.x0 + (a & 3));
-            st.sl_weight = is_halo ? 0 : wint;
-            st.sl_virtual = is_halo ? 1 : 0;
-            st.sl_cell = a;
-        }
-        if (!is_halo) {
-            if (lane == 0) {
-                const float wn = lva == 1 ? W1s[a] * (float)wint : (float)wint;
-                rec->node[nn] = NodeCmd{a, lva, s, wn};
-            }
-            nn++;
-        }
-    }
-    st.active = memb;
-    st.prev_lv = lv;
-    st.prev_slot = cur_slot;
-    st.prev_nk = nk;
 
     int npost = 0;
     if (is_last) {
-        for (uint32_t live = memb; live; live &= live - 1) {
-            const int s = __ffs(live) - 1;
-            const int key = __shfl_sync(full, st.sl_key, s), wgt = __shfl_sync(full, st.sl_weight, s);
-            const int virt = __shfl_sync(full, st.sl_virtual, s);
-            if (lane == 0) {
-                if (!virt && it.last_seg) {
-                    rec->post[npost] = FlushCmd{s, 0, key, (float)wgt};
-                } else {
-                    rec->post[npost] = FlushCmd{s, 1, it.item * kPieceSlots + 16 + s, 0.f};
-                    if (rank == 0) p.piece_meta[it.item * kPieceSlots + 16 + s] = make_int2(key, wgt);
-                }
+        npost = __popc(active);
+        if (low && ((active >> lane) & 1u)) {
+            const int at = __popc(active & ((1u << lane) - 1));
+            if (!tab->virt[lane] && it.last_seg) {
+                rec->post[at] = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
+            } else {
+                const int pc = it.item * kPieceSlots + 16 + lane;
+                rec->post[at] = FlushCmd{lane, 1, pc, 0.f};
+                if (rank == 0) p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
             }
-            npost++;
         }
-        st.active = 0;
     }
-    if (lane == 0) { rec->n_pre = npre; rec->n_nodes = nn; rec->n_post = npost; }
+    if (lane == 0) {
+        rec->n_pre = __popc(dead);
+        rec->n_nodes = is_halo ? 0 : __popc(anchorm);
+        rec->n_post = npost;
+    }
+    st.active = is_last ? 0u : active;
+    st.prev_lv = lv;
+    st.prev_slot = cur_slot;
+    st.prev_nk = nk;
     __syncwarp();
 }
 
 // ---------------------------------------------------------------------------------
 // The kernel.  blockDim.x = (Wn + 1) * 32: Wn worker warps, then the decision warp.
 // ---------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kFusedMaxThreads, 1)
+template <int MAX_THREADS>
+__global__ void __launch_bounds__(MAX_THREADS, 1)
 k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus) {
     extern __shared__ __align__(128) unsigned char smem[];
     // carve-up
     unsigned char* ring = smem;
     size_t off = (size_t)p.R * p.slot_bytes;
     float* red = reinterpret_cast<float*>(smem + off);      off += (size_t)p.NM * kGramVals * 4;
-    float* xchg = reinterpret_cast<float*>(smem + off);     off += (size_t)2 * p.C * kGramVals * 4;
-    float* dG = reinterpret_cast<float*>(smem + off);       off += kGramVals * 4;
-    float* dY = reinterpret_cast<float*>(smem + off);       off += 512 * 4;
+    float* xchg = reinterpret_cast<float*>(smem + off);     off += (size_t)2 * p.C * kSumVals * 4;
     float* W1s = reinterpret_cast<float*>(smem + off);      off += 16 * 4;
     float* W2s = reinterpret_cast<float*>(smem + off);      off += 16 * 4;
+    SlotTable* tab = reinterpret_cast<SlotTable*>(smem + off); off += sizeof(SlotTable);
     FrameRec* recs = reinterpret_cast<FrameRec*>(smem + off); off += kRecRing * sizeof(FrameRec);
     unsigned long long* full_bar = reinterpret_cast<unsigned long long*>(smem + off); off += 16 * 8;
     int* ctl = reinterpret_cast<int*>(smem + off);          // [0] current item, [1] records published
@@ -529,15 +532,18 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     }
                     if (warp < p.NM) {
                         // Gram and cross matrices over this warp's share of the channels
+                        // two independent accumulator sets keep twice as many tensor-core operations in flight
                         float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
                         float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+                        float h0[4] = {0.f, 0.f, 0.f, 0.f}, h1[4] = {0.f, 0.f, 0.f, 0.f};
+                        float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
                         const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
                         const uint32_t cur = ring_base + s * p.slot_bytes + lrow * p.row_bytes + lk * 2;
                         const int sp = (q - 1 + p.R) % p.R;
                         const uint32_t prv = ring_base + sp * p.slot_bytes + lrow * p.row_bytes + lk * 2;
                         const int ksteps = p.S >> 4;
                         if (j > 0) {
-                            for (int ks = warp; ks < ksteps; ks += p.NM) {
+                            for (int ks = warp; ks < ksteps; ks += 2 * p.NM) {
                                 uint32_t a[4], b[4];
                                 ldmatrix_x4(cur + ks * 32, a);
                                 ldmatrix_x4(prv + ks * 32, b);
@@ -545,15 +551,30 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                                 mma_bf16(g1, a, a[1], a[3]);
                                 mma_bf16(c0, a, b[0], b[2]);
                                 mma_bf16(c1, a, b[1], b[3]);
+                                if (ks + p.NM < ksteps) {
+                                    ldmatrix_x4(cur + (ks + p.NM) * 32, a);
+                                    ldmatrix_x4(prv + (ks + p.NM) * 32, b);
+                                    mma_bf16(h0, a, a[0], a[2]);
+                                    mma_bf16(h1, a, a[1], a[3]);
+                                    mma_bf16(e0, a, b[0], b[2]);
+                                    mma_bf16(e1, a, b[1], b[3]);
+                                }
                             }
                         } else {
-                            for (int ks = warp; ks < ksteps; ks += p.NM) {
+                            for (int ks = warp; ks < ksteps; ks += 2 * p.NM) {
                                 uint32_t a[4];
                                 ldmatrix_x4(cur + ks * 32, a);
                                 mma_bf16(g0, a, a[0], a[2]);
                                 mma_bf16(g1, a, a[1], a[3]);
+                                if (ks + p.NM < ksteps) {
+                                    ldmatrix_x4(cur + (ks + p.NM) * 32, a);
+                                    mma_bf16(h0, a, a[0], a[2]);
+                                    mma_bf16(h1, a, a[1], a[3]);
+                                }
                             }
                         }
+#pragma unroll
+                        for (int i = 0; i < 4; i++) { g0[i] += h0[i]; g1[i] += h1[i]; c0[i] += e0[i]; c1[i] += e1[i]; }
                         float* r = red + warp * kGramVals;
                         const int gr = lane >> 2, gc = (lane & 3) * 2;
                         *reinterpret_cast<float2*>(r + gr * 16 + gc) = make_float2(g0[0], g0[1]);
@@ -568,13 +589,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 }
                 named_sync(1, nworkers);
                 if (j < it.n) {
-                    // add the warps' partial matrices and hand the CTA's total to every CTA of the cluster
-                    float* mine = xchg + ((qbase + j) & 1) * p.C * kGramVals + rank * kGramVals;
-                    for (int v = tid; v < kGramVals; v += nworkers) {
-                        float s = 0.f;
-                        for (int w = 0; w < p.NM; w++) s += red[w * kGramVals + v];
-                        const uint32_t a = smem_u32(mine + v);
-                        for (int r = 0; r < p.C; r++) st_cluster_f32(map_to_rank(a, r), s);
+                    // contract the warps' partial matrices to the 8 numbers per cell and hand the CTA's
+                    // share to every CTA of the cluster
+                    for (int i = tid; i < kSumVals; i += nworkers) {
+                        const float sum = combine_sums(red, p.NM, i & 15, i >> 4, W1s, W2s);
+                        const uint32_t a = smem_u32(xchg + ((qbase + j) & 1) * p.C * kSumVals + rank * kSumVals + i);
+                        for (int r = 0; r < p.C; r++) st_cluster_f32(map_to_rank(a, r), sum);
                     }
                 }
                 cluster_arrive();
@@ -641,16 +661,27 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             // ------------------------------ decision warp ------------------------------
             DecState st;
             st.prev_lv = 0; st.prev_slot = 0; st.prev_nk = 0.f;
-            st.sl_key = -1; st.sl_weight = 0; st.sl_virtual = 0; st.sl_cell = 0;
             st.active = 0;
             const float tau_s = taus.s[it.b], tau_t = taus.t[it.b];
+            cluster_arrive();
             for (int j = 0; j < it.n + 2; j++) {
-                cluster_arrive();
                 cluster_wait();
+                // take this frame's totals out of the exchange buffer, then let the cluster go on:
+                // the decisions themselves run beside the workers' next frame
+                float v[8];
                 if (j < it.n) {
-                    const float* xch = xchg + ((qbase + j) & 1) * p.C * kGramVals;
+                    const float* xch = xchg + ((qbase + j) & 1) * p.C * kSumVals;
+#pragma unroll
+                    for (int k = 0; k < 8; k++) {
+                        float sum = 0.f;
+                        for (int r = 0; r < p.C; r++) sum += xch[r * kSumVals + k * 16 + (lane & 15)];
+                        v[k] = sum;
+                    }
+                }
+                if (j + 1 < it.n + 2) cluster_arrive();
+                if (j < it.n) {
                     FrameRec* rec = recs + ((qbase + j) % kRecRing);
-                    decide_frame(p, it, j, tau_s, tau_t, xch, dG, dY, W1s, W2s, st, rec, rank, lane);
+                    decide_frame(p, it, j, tau_s, tau_t, v, W1s, W2s, st, tab, rec, rank, lane);
                     if (lane == 0) st_release_cta(ctl + 1, qbase + j + 1);
                 }
             }
@@ -659,6 +690,32 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         __syncthreads();
     }
     if (timed_out && p.status != nullptr) atomicOr(p.status, kStatusWaitTimeout);
+}
+
+// ---------------------------------------------------------------------------------
+// Roots (Section 3.3, "common root node").  Inside an item the fused kernel already follows
+// every chain to its first node; a chain that enters an item from the frame before it is
+// known there by that earlier node, whose own entry names a node further back.  One thread
+// per cell walks these hand-overs (at most one per item border).
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_resolve_roots(Geo g, int max_hops, const int32_t* __restrict__ chain_key, int32_t* __restrict__ root,
+                int32_t* status) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)g.B * g.N) return;
+    const long long vb = i / g.N * g.N;
+    int r = chain_key[i];
+    int hops = 0;
+    while (true) {
+        const int up = chain_key[vb + r];
+        if (up == r) break;
+        r = up;
+        if (++hops > max_hops) {
+            if (status != nullptr) atomicOr(status, kStatusNotConverged);
+            break;
+        }
+    }
+    root[i] = r;
 }
 
 // ---------------------------------------------------------------------------------
@@ -692,23 +749,34 @@ k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict
     const int lane = threadIdx.x & 31;
     const long long nrows = min(vid_off[g.B], capacity);
     const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+    const int n16 = (int)((size_t)g.D * sizeof(OutT) / 16);
     for (long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < nrows; r += nwarps) {
         const int head = row_head[r];
         if (head < 0) {
-            // video of the row: vid_off is short, walk it
-            int b = 0;
+            int b = 0;                                  // video of the row: vid_off is short, walk it
             while (b + 1 < g.B && vid_off[b + 1] <= r) b++;
             const long long src = (long long)b * g.N + row_anchor[r];
             const uint4* s4 = reinterpret_cast<const uint4*>(staging + src * g.D);
             uint4* d4 = reinterpret_cast<uint4*>(out + r * g.D);
-            const int n16 = (int)((size_t)g.D * sizeof(OutT) / 16);
-            for (int i = lane; i < n16; i += 32) d4[i] = s4[i];
+            for (int i0 = 0; i0 < n16; i0 += 8 * 32) {  // eight loads in flight per lane
+                uint4 v[8];
+#pragma unroll
+                for (int k = 0; k < 8; k++) {
+                    const int i = i0 + k * 32 + lane;
+                    if (i < n16) v[k] = __ldcs(s4 + i);
+                }
+#pragma unroll
+                for (int k = 0; k < 8; k++) {
+                    const int i = i0 + k * 32 + lane;
+                    if (i < n16) __stcs(d4 + i, v[k]);
+                }
+            }
         } else {
             const float wsum = (float)row_weight[r];
             for (int d = lane * VEC; d < g.D; d += kSliceCh) {
                 float sum[VEC] = {0.f, 0.f, 0.f, 0.f};
                 int last = -1;
-                while (true) {          // next larger piece index on the list
+                while (true) {          // next larger piece index on the row's (short) list
                     int best = 0x7fffffff;
                     for (int pc = head; pc >= 0; pc = piece_next[pc])
                         if (pc > last && pc < best) best = pc;

@@ -178,7 +178,7 @@ int sttm_last_path(void);
  * Launch shape the fused kernel would get for these params (host pointers; queries the
  * current device for the number of clusters that fit).  shape[10] = {cluster size, channels
  * per CTA, threads per CTA, ring slots, dynamic shared memory bytes, frames per item, items,
- * clusters that can be resident, clusters launched, tensor-core warps}.  Returns 1, or 0
+ * clusters that can be resident, clusters launched, tensor-core (Gram) warps}.  Returns 1, or 0
  * when the fused kernel does not apply to the params.
  */
 int sttm_fused_launch_shape(const sttm_params* p, int* shape);

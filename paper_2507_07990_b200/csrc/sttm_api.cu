@@ -36,7 +36,7 @@ inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 // Launch shape of the fused kernel for one problem; ok == false: the three-pass kernels run.
 struct FusedPlan {
     bool ok;
-    int C, S, Wn, NM, R, row_bytes, slot_bytes, F, nseg, nitems, ntiles, Wt;
+    int C, S, NM, NA, R, row_bytes, slot_bytes, F, nseg, nitems, ntiles, Wt;
     size_t smem;
     unsigned char tile_order[kMaxTiles];
 };
@@ -68,19 +68,21 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     int C = 0;
     for (int c = 1; c <= kMaxCluster; c *= 2) {
         if (g_tune_cluster && c != g_tune_cluster) continue;
-        if (g.D % (16 * c) == 0 && g.D / c <= 64 * kFusedMaxWorkerWarps) { C = c; break; }
+        if (g.D % (16 * c) == 0 && g.D / c <= 128 * kMaxSumWarps) { C = c; break; }
     }
     if (C == 0) return;
     f->C = C;
     f->S = g.D / C;
-    f->Wn = (f->S + 63) / 64;
-    f->NM = std::min(4, f->Wn);
+    const int ksteps = f->S / 16;
+    f->NM = ksteps >= 8 ? 4 : (ksteps >= 4 ? 2 : 1);
+    f->NA = (f->S + 127) / 128;
     f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
     f->slot_bytes = 16 * f->row_bytes;
-    const size_t fixed = (size_t)f->NM * kGramVals * 4 + (size_t)2 * C * kSumVals * 4 + 32 * 4 + sizeof(SlotTable) +
-                         kRecRing * sizeof(FrameRec) + 16 * 8 + 64;
+    const size_t fixed = (size_t)f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
+                         16 * 32 * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) +
+                         (2 * kMaxRing + 6 * kRecRing) * 8;
     int R = (int)((kMaxSmem - fixed) / f->slot_bytes);
-    R = std::min(R, 8);
+    R = std::min(R, kMaxRing);
     if (R < 4) return;
     f->R = R;
     f->smem = (size_t)R * f->slot_bytes + fixed;
@@ -286,27 +288,27 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
 
 // Resident clusters of the fused kernel for a launch shape (cached); falls back to SMs / C.
 int fused_resident_clusters(const FusedPlan& f) {
-    static int cached[kMaxCluster + 1][kFusedMaxWorkerWarps + 2];
-    static size_t cached_smem[kMaxCluster + 1][kFusedMaxWorkerWarps + 2];
-    int& slot = cached[f.C][f.Wn];
-    if (slot > 0 && cached_smem[f.C][f.Wn] == f.smem) return slot;
+    static int cached[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
+    static size_t cached_smem[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
+    const int warps = f.NM + f.NA + 3;
+    int& slot = cached[f.C][warps];
+    if (slot > 0 && cached_smem[f.C][warps] == f.smem) return slot;
     int n = 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kSmCount / f.C * f.C);
-    cfg.blockDim = dim3((f.Wn + 1) * 32);
+    cfg.blockDim = dim3(warps * 32);
     cfg.dynamicSmemBytes = f.smem;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    const cudaError_t e = cfg.blockDim.x <= 480 ? cudaOccupancyMaxActiveClusters(&n, k_fused<480>, &cfg)
-                                                : cudaOccupancyMaxActiveClusters(&n, k_fused<kFusedMaxThreads>, &cfg);
-    if (e != cudaSuccess || n < 1) {
+    cudaFuncSetAttribute(k_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+    if (cudaOccupancyMaxActiveClusters(&n, k_fused, &cfg) != cudaSuccess || n < 1) {
         cudaGetLastError();
         n = kSmCount / f.C;
     }
     slot = n;
-    cached_smem[f.C][f.Wn] = f.smem;
+    cached_smem[f.C][warps] = f.smem;
     return n;
 }
 
@@ -316,9 +318,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     const FusedPlan& f = pl.f;
     static bool configured = false;
     if (!configured) {
-        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<480>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<kFusedMaxThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         configured = true;
     }
     FusedParams fp = {};
@@ -326,7 +326,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.B = g.B; fp.T = g.T; fp.H = g.H; fp.W = g.W; fp.D = g.D; fp.L = g.L;
     fp.HW = g.HW; fp.N = g.N;
     fp.Wt = f.Wt; fp.ntiles = f.ntiles;
-    fp.C = f.C; fp.S = f.S; fp.Wn = f.Wn; fp.NM = f.NM;
+    fp.C = f.C; fp.S = f.S; fp.NM = f.NM; fp.NA = f.NA;
     fp.row_bytes = f.row_bytes; fp.slot_bytes = f.slot_bytes; fp.R = f.R;
     fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
     fp.weight_mode = (int)p->wt;
@@ -337,7 +337,6 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.staging = ws + pl.staging;
     fp.pieces = (float*)(ws + pl.pieces);
     fp.piece_meta = (int2*)(ws + pl.piece_meta);
-    fp.queue = (int*)(ws + pl.queue);
     fp.status = device_status;
     std::memcpy(fp.tile_order, f.tile_order, sizeof(fp.tile_order));
     Taus taus;
@@ -346,16 +345,14 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     const int nclusters = std::min(f.nitems, fused_resident_clusters(f));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nclusters * f.C);
-    cfg.blockDim = dim3((f.Wn + 1) * 32);
+    cfg.blockDim = dim3((f.NM + f.NA + 3) * 32);
     cfg.dynamicSmemBytes = f.smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    // two builds of the same kernel: up to 15 warps may use 128 registers per thread, up to 17 only 96
-    if (cfg.blockDim.x <= 480) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<480>, fp, taus));
-    else STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<kFusedMaxThreads>, fp, taus));
+    STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused, fp, taus));
     g_launches++;
     return STTM_OK;
 }
@@ -445,7 +442,7 @@ int sttm_fused_launch_shape(const sttm_params* p, int* shape) {
     if (shape == nullptr || make_plan(p, &pl) != STTM_OK || !pl.f.ok) return 0;
     const FusedPlan& f = pl.f;
     const int resident = fused_resident_clusters(f);
-    const int v[10] = {f.C, f.S, (f.Wn + 1) * 32, f.R, (int)f.smem, f.F, f.nitems, resident,
+    const int v[10] = {f.C, f.S, (f.NM + f.NA + 3) * 32, f.R, (int)f.smem, f.F, f.nitems, resident,
                        std::min(f.nitems, resident), f.NM};
     std::memcpy(shape, v, sizeof(v));
     return 1;

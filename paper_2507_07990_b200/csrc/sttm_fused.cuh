@@ -5,26 +5,26 @@
 // node when the tree has three levels; four / sixteen independent regions when it has two
 // / one).  Everything that touches features stays inside one tile through time, so a work
 // item is (video, tile, run of consecutive frames).  A thread-block cluster of C CTAs owns
-// an item; each CTA owns D/C channels of the tile and streams them frame by frame through
-// a shared-memory ring filled by bulk asynchronous copies (one per cell).
+// a fixed list of items; each CTA owns D/C channels of the tile and streams them frame by
+// frame through a shared-memory ring filled by bulk asynchronous copies (one per cell).
 //
-// Per frame j of an item:
-//   1. tensor-core warps form the tile's Gram matrix G_j = X_j X_j^T and the cross matrix
-//      C_j = X_j X_{j-1}^T over the CTA's channels (X = the 16 cells of the tile); every
-//      cosine of Sections 3.2 and 3.3 is a short linear combination of entries of G and C
-//      because parents are averages of cells.  The products of bf16 inputs are exact and
-//      the sums are kept in fp32.
-//   2. worker threads contract the partial matrices to the 128 numbers the decisions need
-//      (per cell: its squared norm, its products with its parent and with the coarsest node,
-//      and its products with the nodes of the previous frame that contain it or that it
-//      contains) and add them across warps (shared memory) and across the cluster
-//      (distributed shared memory), in a fixed order.
-//   3. one decision warp per CTA turns the totals into the cover map, the links and the
-//      bookkeeping of the running chains (every CTA of the cluster repeats this on the
-//      same numbers and gets the same answer), and leaves a small command record.
-//   4. two frames later the worker threads execute the record on the frame that is still
-//      in the ring: each thread owns two channels, keeps the running sums of up to 16
-//      chains in registers, adds the nodes of the frame and writes out chains that ended.
+// The warps of a CTA are specialised and hand frames to each other through mbarriers, so
+// that every stage works on a different frame at the same time:
+//   producer warp   issues the bulk copies of the next frames as ring slots come free;
+//   Gram warps      form the tile's Gram matrix G = X_t X_t^T and cross matrix
+//                   C = X_t X_{t-1}^T over the CTA's channels on the tensor cores (X = the 16
+//                   cells of the tile; products of bf16 inputs are exact, sums are fp32),
+//                   add the warps' parts, contract them to the 128 numbers the decisions
+//                   need (every cosine of Sections 3.2 and 3.3 is a short linear combination
+//                   of entries of G and C because parents are averages of cells) and send
+//                   them to every CTA of the cluster (stores that signal a remote mbarrier);
+//   similarity warp adds the cluster's shares in a fixed order and takes the decisions of
+//                   Section 3.2 (cover map) and Section 3.3 (links), the same in every CTA;
+//   chain warp      follows the chains through time: which running sum each kept node
+//                   joins, which chains ended; leaves a command record per frame;
+//   sum warps       execute the records on the frame that is still in the ring: a thread
+//                   owns four channels and keeps the running sums of up to 16 chains in
+//                   registers.
 // Finished chains go to a staging row indexed by the root's cell id (their final row is
 // only known after the global ordering); chains cut by the end of an item go to an fp32
 // piece buffer and are put together by the gather kernel.
@@ -37,23 +37,27 @@ namespace sttm {
 
 constexpr int kMaxTiles = 64;
 constexpr int kMaxCluster = 8;
-constexpr int kRecRing = 4;
+constexpr int kRecRing = 4;             // command records, hand-over slots and exchange buffers in flight
 constexpr int kGramVals = 512;          // G (16x16) then C (16x16)
 constexpr int kSumVals = 128;           // 8 numbers per cell, see combine_sums()
 constexpr int kPieceSlots = 32;         // per item: 16 keyed by a cell of the frame before the item, 16 by chain slot
-constexpr int kFusedMaxWorkerWarps = 16;
-constexpr int kFusedMaxThreads = (kFusedMaxWorkerWarps + 1) * 32;
-constexpr int kSpinLimit = 1 << 20;   // after the first wait that runs out, later waits are skipped
+constexpr int kMaxRing = 12;
+constexpr int kMaxGramWarps = 4;
+constexpr int kMaxSumWarps = 8;         // 128 channels each: at most 1024 channels per CTA
+constexpr int kFusedMaxThreads = (kMaxGramWarps + kMaxSumWarps + 3) * 32;
+constexpr int kSpinLimit = 1 << 20;     // after the first wait that runs out, later waits are skipped
 
 enum : int { kStatusWaitTimeout = 1 << 6 };
 
 struct FlushCmd { int slot, kind, dst; float weight; };     // kind 0: finished row, 1: piece
-struct NodeCmd { int cell, lv, slot; float w; };
+struct NodeCmd { int cell, lv, slot; float w; };            // lv: level | (cells of the node inside the grid) << 4
+// Commands of one frame for the sum warps: first write out and clear the listed chain sums
+// (chains that got no member in this frame; at the first frame of an item: everything the
+// previous item left), then add the frame's kept nodes.
 struct FrameRec {
-    int n_pre, n_nodes, n_post, pad;
-    FlushCmd pre[16];
+    int n_flush, n_nodes, cls, pad;
+    FlushCmd flush[16];
     NodeCmd node[16];
-    FlushCmd post[16];
 };
 
 struct FusedParams {
@@ -61,7 +65,7 @@ struct FusedParams {
     int B, T, H, W, D, L;
     int HW, N;
     int Wt, ntiles;
-    int C, S, Wn, NM;        // cluster size, channels per CTA, worker warps, tensor-core warps
+    int C, S, NM, NA;        // cluster size, channels per CTA, Gram warps, sum warps
     int row_bytes, slot_bytes, R;
     int F, nseg, nitems;
     int weight_mode, out_f32;
@@ -71,7 +75,6 @@ struct FusedParams {
     void* staging;           // [B*N][D] rows of the output dtype
     float* pieces;           // [nitems][kPieceSlots][D]
     int2* piece_meta;        // [nitems][kPieceSlots] {key cell id or -1, weight}
-    int* queue;
     int* status;
     unsigned char tile_order[kMaxTiles];
 };
@@ -84,19 +87,36 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// arrive on an mbarrier of another CTA of the cluster (address from map_to_rank)
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
+}
+// Bounded wait for the `use`-th completion (0-based) of an mbarrier.  Once a wait has run
+// out the thread stops waiting altogether, so the kernel still ends; the host sees
+// kStatusWaitTimeout in the status word.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, int use, bool& timed_out) {
+    const uint32_t parity = (uint32_t)(use & 1);
+    int spins = 0;
+    while (!timed_out && !mbar_try_wait(bar, parity)) {
+        if (++spins > kSpinLimit) timed_out = true;
+    }
 }
 // global -> this CTA's shared memory, completion counted in bytes on an mbarrier
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -104,9 +124,26 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// 4-byte store into the shared memory of a CTA of the cluster that also counts 4 bytes on an
+// mbarrier of that CTA
+__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(cluster_addr),
+                 "r"(__float_as_uint(v)), "r"(cluster_bar)
+                 : "memory");
+}
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_count() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
     return r;
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
@@ -115,12 +152,6 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     uint32_t out;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(addr), "r"(rank));
     return out;
-}
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
-    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void named_sync(int id, int count) {
     asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -137,18 +168,10 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+__device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
-}
-__device__ __forceinline__ int ld_acquire_cta(const int* p) {
-    int v;
-    asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release_cta(int* p, int v) {
-    asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
 
 // tile-local cell c = dy*4 + dx; top-left cell of the level-lv node that holds c
@@ -160,44 +183,62 @@ __device__ __forceinline__ uint32_t quad_mask(int c) { return 0x33u << (8 * (c >
 __device__ __forceinline__ uint32_t region_mask(int c, int lv) {
     return lv == 0 ? (1u << c) : (lv == 1 ? quad_mask(c) : 0xffffu);
 }
+// position of the k-th (0-based) set bit of a 16-bit mask that has more than k bits set
+__device__ __forceinline__ int kth_set_bit16(uint32_t m, int k) {
+    int pos = 0;
+    int n = __popc(m & 0xffu);
+    if (k >= n) { k -= n; pos = 8; }
+    n = __popc((m >> pos) & 0xfu);
+    if (k >= n) { k -= n; pos += 4; }
+    n = __popc((m >> pos) & 0x3u);
+    if (k >= n) { k -= n; pos += 2; }
+    n = (int)((m >> pos) & 1u);
+    if (k >= n) pos += 1;
+    return pos;
+}
 
-// running sums of the chains: 16 slots x 2 channels, in registers; the slot index is
-// uniform over the block, so the switch does not diverge
+// running sums of the chains: 16 slots x 4 channels, in registers; the slot index is
+// uniform over the warp, so the switch does not diverge
 struct ChainAcc {
-    float2 a[16];
+    float4 a[16];
     __device__ __forceinline__ void clear() {
 #pragma unroll
-        for (int i = 0; i < 16; i++) a[i] = make_float2(0.f, 0.f);
+        for (int i = 0; i < 16; i++) a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-#define STTM_ACC_CASE(i) case i: a[i].x += f.x; a[i].y += f.y; break;
-    __device__ __forceinline__ void add(int slot, float2 f) {
+#define STTM_ACC_BODY(i) a[i].x += f.x; a[i].y += f.y; a[i].z += f.z; a[i].w += f.w; break;
+#define STTM_ACC_CASE(i) case i: STTM_ACC_BODY(i)
+    __device__ __forceinline__ void add(int slot, float4 f) {
         switch (slot) {
             STTM_ACC_CASE(0) STTM_ACC_CASE(1) STTM_ACC_CASE(2) STTM_ACC_CASE(3) STTM_ACC_CASE(4) STTM_ACC_CASE(5)
             STTM_ACC_CASE(6) STTM_ACC_CASE(7) STTM_ACC_CASE(8) STTM_ACC_CASE(9) STTM_ACC_CASE(10) STTM_ACC_CASE(11)
-            STTM_ACC_CASE(12) STTM_ACC_CASE(13) STTM_ACC_CASE(14) default: a[15].x += f.x; a[15].y += f.y; break;
+            STTM_ACC_CASE(12) STTM_ACC_CASE(13) STTM_ACC_CASE(14) default: STTM_ACC_BODY(15)
         }
     }
 #undef STTM_ACC_CASE
-#define STTM_TAKE_CASE(i) case i: v = a[i]; a[i] = make_float2(0.f, 0.f); break;
-    __device__ __forceinline__ float2 take(int slot) {
-        float2 v;
+#undef STTM_ACC_BODY
+#define STTM_TAKE_BODY(i) v = a[i]; a[i] = make_float4(0.f, 0.f, 0.f, 0.f); break;
+#define STTM_TAKE_CASE(i) case i: STTM_TAKE_BODY(i)
+    __device__ __forceinline__ float4 take(int slot) {
+        float4 v;
         switch (slot) {
             STTM_TAKE_CASE(0) STTM_TAKE_CASE(1) STTM_TAKE_CASE(2) STTM_TAKE_CASE(3) STTM_TAKE_CASE(4)
             STTM_TAKE_CASE(5) STTM_TAKE_CASE(6) STTM_TAKE_CASE(7) STTM_TAKE_CASE(8) STTM_TAKE_CASE(9)
             STTM_TAKE_CASE(10) STTM_TAKE_CASE(11) STTM_TAKE_CASE(12) STTM_TAKE_CASE(13) STTM_TAKE_CASE(14)
-            default: v = a[15]; a[15] = make_float2(0.f, 0.f); break;
+            default: STTM_TAKE_BODY(15)
         }
         return v;
     }
 #undef STTM_TAKE_CASE
+#undef STTM_TAKE_BODY
 };
 
-__device__ __forceinline__ float2 unpack_bf16x2(uint32_t w) {
-    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+__device__ __forceinline__ float4 unpack_bf16x4(uint2 w) {
+    return make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u), __uint_as_float(w.y << 16),
+                       __uint_as_float(w.y & 0xffff0000u));
 }
-__device__ __forceinline__ uint32_t pack_bf16x2(float2 v) {
-    const __nv_bfloat162 h = __floats2bfloat162_rn(v.x, v.y);
-    return *reinterpret_cast<const uint32_t*>(&h);
+__device__ __forceinline__ uint2 pack_bf16x4(float4 v) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    return make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
 }
 
 // sum over lanes that share (lane & 16): every lane of a half gets its half's total
@@ -206,25 +247,53 @@ __device__ __forceinline__ float half_warp_sum(float v) {
     for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
+// sum over the four cells of the lane's 2x2 block (lane = cell, or cell + 16)
+__device__ __forceinline__ float quad_sum(float v) {
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    return v;
+}
+// cos(a, b) > tau from a.b, |a|^2, |b|^2 without a division; a zero vector has cosine 0
+__device__ __forceinline__ bool cos_above(float dot, float na, float nb, float tau) {
+    if (na == 0.f || nb == 0.f) return 0.f > tau;
+    return dot > tau * (sqrtf(na) * sqrtf(nb));
+}
 
 struct ItemGeo {
-    int item, b, t0, t1, tstart, n, halo, last_seg;
-    int y0, x0;
+    int item, b, tstart, n, halo, last_seg;
+    int y0, x0, cls;
     uint32_t vmask;     // bit c: cell c of the tile lies inside the grid
     int nvalid;
 };
 
-// What the decision warp carries from frame to frame (lane c < 16: cell c of the tile).
-struct DecState {
-    int prev_lv, prev_slot;      // level / chain slot of the kept node covering the cell in the previous frame
-    float prev_nk;               // its squared norm
-    uint32_t active;             // uniform: slots in use
-};
-
-// Chain slots of the decision warp (shared memory, private to it).
-struct SlotTable {
-    int key[16], weight[16], virt[16], cell[16];
-};
+// The round-th item of this cluster: items are numbered from the most expensive tile to the
+// cheapest and dealt to the clusters back and forth.  Returns false past the last round;
+// `skip` says that this cluster has no item in the round.
+__device__ __forceinline__ bool next_item(const FusedParams& p, int round, uint32_t cid, uint32_t ncl, ItemGeo& it,
+                                          bool& skip) {
+    const long long base = (long long)round * ncl;
+    if (base >= p.nitems) return false;
+    const long long idx = base + ((round & 1) ? (long long)(ncl - 1 - cid) : (long long)cid);
+    skip = idx >= p.nitems;
+    if (skip) return true;
+    it.item = (int)idx;
+    const int seg = it.item % p.nseg;
+    const int tb = it.item / p.nseg;
+    it.b = tb % p.B;
+    const int tile = p.tile_order[tb / p.B];
+    const int t0 = seg * p.F, t1 = min(p.T, t0 + p.F);
+    it.halo = t0 > 0;
+    it.tstart = t0 - it.halo;
+    it.n = t1 - it.tstart;
+    it.last_seg = t1 == p.T;
+    it.y0 = (tile / p.Wt) * 4;
+    it.x0 = (tile % p.Wt) * 4;
+    const int rows = min(4, p.H - it.y0), cols = min(4, p.W - it.x0);
+    it.cls = (rows - 1) * 4 + (cols - 1);
+    it.vmask = (0xfu >> (4 - cols)) * (0x1111u >> (4 * (4 - rows)));
+    it.nvalid = rows * cols;
+    return true;
+}
 
 // The 8 numbers of cell c that the decisions need, as linear functions of the tile's Gram
 // matrix G = X_t X_t^T and cross matrix Cm = X_t X_{t-1}^T (row: cell of frame t).  With
@@ -232,463 +301,506 @@ struct SlotTable {
 //   k=0  |x_c|^2                       k=1  x_c . parent(c)            k=2  x_c . top
 //   k=3  x_c(t) . x_c(t-1)             k=4  x_c(t) . parent(c)(t-1)    k=5  x_c(t) . top(t-1)
 //   k=6  parent(c)(t) . x_c(t-1)       k=7  top(t) . x_c(t-1)
-// `m` points at NM partial matrices of kGramVals floats each; they are added in order.
-__device__ __forceinline__ float combine_sums(const float* m, int NM, int c, int k, const float* W1s,
+// Ring rows of cells outside the grid hold stale finite data: such columns are masked or
+// get weight 0 here, and the similarity warp drops the numbers of such cells.
+__device__ __forceinline__ float combine_sums(const float* G, int c, int k, uint32_t vmask, const float* W1s,
                                               const float* W2s) {
+    const float* Cm = G + 256;
     const int qb = tile_anchor(c, 1);
-    float acc = 0.f;
-    for (int w = 0; w < NM; w++) {
-        const float* G = m + w * kGramVals;
-        const float* Cm = G + 256;
-        float v = 0.f;
-        switch (k) {
-            case 0: v = G[c * 16 + c]; break;
-            case 1: v = ((G[c * 16 + qb] + G[c * 16 + qb + 1]) + (G[c * 16 + qb + 4] + G[c * 16 + qb + 5])) * W1s[c]; break;
-            case 2:
+    const float m0 = (vmask >> qb) & 1u ? 1.f : 0.f, m1 = (vmask >> (qb + 1)) & 1u ? 1.f : 0.f;
+    const float m2 = (vmask >> (qb + 4)) & 1u ? 1.f : 0.f, m3 = (vmask >> (qb + 5)) & 1u ? 1.f : 0.f;
+    float v = 0.f;
+    switch (k) {
+        case 0: v = G[c * 16 + c]; break;
+        case 1:
+            v = ((m0 * G[c * 16 + qb] + m1 * G[c * 16 + qb + 1]) + (m2 * G[c * 16 + qb + 4] + m3 * G[c * 16 + qb + 5])) *
+                W1s[c];
+            break;
+        case 2:
 #pragma unroll
-                for (int i = 0; i < 16; i++) v = fmaf(W2s[i], G[c * 16 + i], v);
-                break;
-            case 3: v = Cm[c * 16 + c]; break;
-            case 4: v = ((Cm[c * 16 + qb] + Cm[c * 16 + qb + 1]) + (Cm[c * 16 + qb + 4] + Cm[c * 16 + qb + 5])) * W1s[c]; break;
-            case 5:
+            for (int i = 0; i < 16; i++) v = fmaf(W2s[i], G[c * 16 + i], v);
+            break;
+        case 3: v = Cm[c * 16 + c]; break;
+        case 4:
+            v = ((m0 * Cm[c * 16 + qb] + m1 * Cm[c * 16 + qb + 1]) +
+                 (m2 * Cm[c * 16 + qb + 4] + m3 * Cm[c * 16 + qb + 5])) * W1s[c];
+            break;
+        case 5:
 #pragma unroll
-                for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[c * 16 + i], v);
-                break;
-            case 6: v = ((Cm[qb * 16 + c] + Cm[(qb + 1) * 16 + c]) + (Cm[(qb + 4) * 16 + c] + Cm[(qb + 5) * 16 + c])) * W1s[c]; break;
-            default:
+            for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[c * 16 + i], v);
+            break;
+        case 6:
+            v = ((m0 * Cm[qb * 16 + c] + m1 * Cm[(qb + 1) * 16 + c]) +
+                 (m2 * Cm[(qb + 4) * 16 + c] + m3 * Cm[(qb + 5) * 16 + c])) * W1s[c];
+            break;
+        default:
 #pragma unroll
-                for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[i * 16 + c], v);
-                break;
-        }
-        acc += v;
+            for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[i * 16 + c], v);
+            break;
     }
-    return acc;
+    return v;
 }
 
-// sum over the four cells of the lane's 2x2 block (lanes of the same half warp)
-__device__ __forceinline__ float quad_sum(float v, int lane) {
-    const int hb = lane & 16, qb = tile_anchor(lane & 15, 1);
-    return (__shfl_sync(0xffffffffu, v, hb + qb) + __shfl_sync(0xffffffffu, v, hb + qb + 1)) +
-           (__shfl_sync(0xffffffffu, v, hb + qb + 4) + __shfl_sync(0xffffffffu, v, hb + qb + 5));
-}
+// Chain slots of the chain warp (shared memory, private to it).
+struct SlotTable {
+    int key[16], weight[16], virt[16], cell[16];
+};
 
 // ---------------------------------------------------------------------------------
-// Decisions of one frame (Sections 3.2 and 3.3) from the cluster totals of the 8 numbers
-// per cell (v[0..7], lane c = cell c; lanes 16..31 mirror lanes 0..15).
+// The kernel.  Warps: [0, NM) Gram, [NM, NM+NA) sum, then similarity, chain, producer.
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void decide_frame(const FusedParams& p, const ItemGeo& it, int j, float tau_s, float tau_t,
-                                             const float (&v)[8], const float* W1s, const float* W2s, DecState& st,
-                                             SlotTable* tab, FrameRec* rec, uint32_t rank, int lane) {
-    const unsigned full = 0xffffffffu;
-    const int c = lane & 15;
-    const bool low = lane < 16;
-    const int L = p.L;
-    const int t = it.tstart + j;
-    const bool has_prev = j > 0;
-    const bool is_halo = it.halo && j == 0;
-    const bool is_last = j == it.n - 1;
-    const bool valid = (it.vmask >> c) & 1u;
-    const uint32_t qm = quad_mask(c);
-    const float w1 = W1s[c], w2 = W2s[c];
-
-    // Section 3.2: cosine of every node with its parent, then the coarse-to-fine search
-    const float n0 = v[0], d0 = v[1], rr = v[2];
-    const float n1 = w1 * quad_sum(d0, lane);          // |parent|^2
-    const float d1 = w1 * quad_sum(rr, lane);          // parent . top
-    const float n2 = half_warp_sum(w2 * rr);           // |top|^2
-    const float s0 = cos_from(d0, n0, n1);
-    const float s1 = cos_from(d1, n1, n2);
-    int lv = 0;
-    if (L >= 2) {
-        const bool p0 = !valid || s0 > tau_s;
-        const uint32_t pm0 = __ballot_sync(full, p0) & 0xffffu;
-        const bool quad_pass = (pm0 & qm) == qm;
-        if (L == 3) {
-            const bool quad_exists = (it.vmask & qm) != 0;
-            const bool p1 = !quad_exists || s1 > tau_s;
-            const uint32_t pm1 = __ballot_sync(full, p1) & 0xffffu;
-            lv = pm1 == 0xffffu ? 2 : (quad_pass ? 1 : 0);
-        } else {
-            lv = quad_pass ? 1 : 0;
-        }
-    }
-    const float nk = lv == 0 ? n0 : (lv == 1 ? n1 : n2);
-
-    // Section 3.3: the node covering the cell against the overlapping kept node of the
-    // previous frame; a pair is evaluated at the top-left cell of its finer node
-    int link_local = -1;
-    if (has_prev) {
-        const int lu = st.prev_lv;
-        const float t11 = w1 * quad_sum(v[4], lane), t12 = w1 * quad_sum(v[5], lane);
-        const float t21 = w1 * quad_sum(v[7], lane), t22 = half_warp_sum(w2 * v[5]);
-        float dot;
-        if (lv == 0) dot = lu == 0 ? v[3] : (lu == 1 ? v[4] : v[5]);
-        else if (lv == 1) dot = lu == 0 ? v[6] : (lu == 1 ? t11 : t12);
-        else dot = lu == 0 ? v[7] : (lu == 1 ? t21 : t22);
-        const bool rep = valid && tile_anchor(c, min(lv, lu)) == c;
-        const float s = cos_from(dot, nk, st.prev_nk);
-        const bool pass = rep && s > tau_t;
-        const uint32_t passm = __ballot_sync(full, pass) & 0xffffu;
-        const uint32_t cand = passm & region_mask(c, lv);
-        const int cstar = cand ? __ffs(cand) - 1 : 0;         // first in row-major order: the top-left one
-        const int lu_star = __shfl_sync(full, lu, cstar);
-        link_local = cand ? tile_anchor(cstar, lu_star) : -1;
-    }
-
-    // chains: nodes with a link join the chain of their target; chains without a member in
-    // this frame have ended; the remaining nodes start new chains in free slots
-    const bool anchor = valid && tile_anchor(c, lv) == c;
-    const bool linked = anchor && link_local >= 0;
-    const bool fresh = anchor && link_local < 0;
-    const int slot_linked = __shfl_sync(full, st.prev_slot, link_local < 0 ? 0 : link_local);
-    const uint32_t memb = __reduce_or_sync(full, linked ? 1u << slot_linked : 0u);
-    const uint32_t dead = st.active & ~memb;
-    const uint32_t freem = ~memb & 0xffffu;
-    const uint32_t freshm = __ballot_sync(full, fresh && low);
-    const int slot_fresh = __fns(freem, 0, __popc(freshm & ((1u << c) - 1)) + 1);
-    const int node_slot = linked ? slot_linked : slot_fresh;
-    const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + tile_anchor(c, lv));
-    const int wint = p.weight_mode ? __popc(it.vmask & region_mask(c, lv)) : 1;
-    const long long gc = (long long)it.b * p.N + (long long)t * p.HW + (it.y0 + (c >> 2)) * p.W + it.x0 + (c & 3);
-
-    // chains that ended: lane s looks at slot s (before the slot is given away again)
-    const bool my_dead = low && ((dead >> lane) & 1u);
-    if (my_dead) {
-        const int at = __popc(dead & ((1u << lane) - 1));
-        if (tab->virt[lane]) {
-            const int pc = it.item * kPieceSlots + tab->cell[lane];
-            rec->pre[at] = FlushCmd{lane, 1, pc, 0.f};
-            if (rank == 0) p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
-        } else {
-            rec->pre[at] = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
-        }
-    }
-    __syncwarp();
-    if (low && fresh) {
-        tab->key[slot_fresh] = (int)gc;
-        tab->weight[slot_fresh] = is_halo ? 0 : wint;
-        tab->virt[slot_fresh] = is_halo ? 1 : 0;
-        tab->cell[slot_fresh] = c;
-    }
-    if (low && linked) atomicAdd(&tab->weight[slot_linked], wint);
-    const uint32_t anchorm = __ballot_sync(full, anchor && low);
-    if (low && anchor && !is_halo) {
-        const float wn = lv == 1 ? w1 * (float)wint : (float)wint;
-        rec->node[__popc(anchorm & ((1u << c) - 1))] = NodeCmd{c, lv, node_slot, wn};
-    }
-    const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
-    __syncwarp();
-
-    if (rank == 0 && !is_halo && low && valid) {
-        p.cover[gc] = (int8_t)lv;
-        p.link[gc] = link_local < 0 ? -1
-                                    : (t - 1) * p.HW + (it.y0 + (link_local >> 2)) * p.W + it.x0 + (link_local & 3);
-        p.chain_key[gc] = tab->key[cur_slot] - it.b * p.N;
-    }
-
-    int npost = 0;
-    if (is_last) {
-        npost = __popc(active);
-        if (low && ((active >> lane) & 1u)) {
-            const int at = __popc(active & ((1u << lane) - 1));
-            if (!tab->virt[lane] && it.last_seg) {
-                rec->post[at] = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
-            } else {
-                const int pc = it.item * kPieceSlots + 16 + lane;
-                rec->post[at] = FlushCmd{lane, 1, pc, 0.f};
-                if (rank == 0) p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
-            }
-        }
-    }
-    if (lane == 0) {
-        rec->n_pre = __popc(dead);
-        rec->n_nodes = is_halo ? 0 : __popc(anchorm);
-        rec->n_post = npost;
-    }
-    st.active = is_last ? 0u : active;
-    st.prev_lv = lv;
-    st.prev_slot = cur_slot;
-    st.prev_nk = nk;
-    __syncwarp();
-}
-
-// ---------------------------------------------------------------------------------
-// The kernel.  blockDim.x = (Wn + 1) * 32: Wn worker warps, then the decision warp.
-// ---------------------------------------------------------------------------------
-template <int MAX_THREADS>
-__global__ void __launch_bounds__(MAX_THREADS, 1)
+__global__ void __launch_bounds__(kFusedMaxThreads, 1)
 k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus) {
     extern __shared__ __align__(128) unsigned char smem[];
-    // carve-up
     unsigned char* ring = smem;
     size_t off = (size_t)p.R * p.slot_bytes;
-    float* red = reinterpret_cast<float*>(smem + off);      off += (size_t)p.NM * kGramVals * 4;
-    float* xchg = reinterpret_cast<float*>(smem + off);     off += (size_t)2 * p.C * kSumVals * 4;
-    float* W1s = reinterpret_cast<float*>(smem + off);      off += 16 * 4;
-    float* W2s = reinterpret_cast<float*>(smem + off);      off += 16 * 4;
+    float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)p.NM * kGramVals * 4;
+    float* redsum = reinterpret_cast<float*>(smem + off);    off += kGramVals * 4;
+    float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * p.C * kSumVals * 4;
+    float* wtab = reinterpret_cast<float*>(smem + off);      off += 16 * 32 * 4;      // [shape][W1 x16, W2 x16]
+    int* hand = reinterpret_cast<int*>(smem + off);          off += kRecRing * 16 * 4;
     SlotTable* tab = reinterpret_cast<SlotTable*>(smem + off); off += sizeof(SlotTable);
     FrameRec* recs = reinterpret_cast<FrameRec*>(smem + off); off += kRecRing * sizeof(FrameRec);
-    unsigned long long* full_bar = reinterpret_cast<unsigned long long*>(smem + off); off += 16 * 8;
-    int* ctl = reinterpret_cast<int*>(smem + off);          // [0] current item, [1] records published
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + off);
+    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t full_bar = bar0, empty_bar = bar0 + 8 * kMaxRing;
+    const uint32_t xfull_bar = bar0 + 16 * kMaxRing, xempty_bar = xfull_bar + 8 * kRecRing;
+    const uint32_t hfull_bar = xempty_bar + 8 * kRecRing, hempty_bar = hfull_bar + 8 * kRecRing;
+    const uint32_t rfull_bar = hempty_bar + 8 * kRecRing, rempty_bar = rfull_bar + 8 * kRecRing;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nworkers = p.Wn * 32;
-    const bool is_dec = warp == p.Wn;
-    const uint32_t rank = cluster_rank();
+    const uint32_t rank = cluster_rank(), cid = cluster_id(), ncl = cluster_count();
     const uint32_t ring_base = smem_u32(ring);
+    const int w_sim = p.NM + p.NA, w_chain = w_sim + 1, w_prod = w_sim + 2;
 
+    // set-up: barriers, a ring without NaN patterns, the pooling weights of all 16 tile shapes
     if (tid == 0) {
-        for (int s = 0; s < p.R; s++) mbar_init(smem_u32(full_bar + s), 1);
-        ctl[0] = 0;
-        ctl[1] = 0;
+        for (int s = 0; s < p.R; s++) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, p.NM + p.NA);
+        }
+        for (int s = 0; s < kRecRing; s++) {
+            mbar_init(xfull_bar + 8 * s, 1);
+            mbar_init(xempty_bar + 8 * s, p.C);
+            mbar_init(hfull_bar + 8 * s, 1);
+            mbar_init(hempty_bar + 8 * s, 1);
+            mbar_init(rfull_bar + 8 * s, 1);
+            mbar_init(rempty_bar + 8 * s, p.NA);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    ChainAcc acc;
-    acc.clear();
+    for (int k = tid * 16; k < p.R * p.slot_bytes; k += blockDim.x * 16)
+        *reinterpret_cast<uint4*>(ring + k) = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < 256; i += blockDim.x) {
+        const int cls = i >> 4, c = i & 15;
+        const int rows = (cls >> 2) + 1, cols = (cls & 3) + 1;
+        const uint32_t vm = (0xfu >> (4 - cols)) * (0x1111u >> (4 * (4 - rows)));
+        const int nq = __popc(vm & quad_mask(c));
+        int quads = 0;
+        for (int qd = 0; qd < 4; qd++) quads += (vm & (0x33u << (8 * (qd >> 1) + 2 * (qd & 1)))) ? 1 : 0;
+        const float inv1 = nq ? 1.f / (float)nq : 0.f;
+        wtab[cls * 32 + c] = p.L >= 2 ? inv1 : 0.f;                                        // per 2x2 block
+        wtab[cls * 32 + 16 + c] = p.L == 3 && ((vm >> c) & 1u) ? inv1 * (1.f / (float)quads) : 0.f;
+    }
     __syncthreads();
+    cluster_arrive();
+    cluster_wait();         // every CTA of the cluster has its barriers before anyone signals them
 
-    int qbase = 0;          // frames consumed so far (same in every thread of the cluster)
     bool timed_out = false;
+    ItemGeo it;
+    bool skip;
+    int q = 0;              // frames of this cluster so far (the same in every role)
 
-    while (true) {
-        // next item: rank 0 draws it and tells the cluster
-        if (rank == 0 && tid == 0) {
-            const int item = atomicAdd(p.queue, 1);
-            for (int r = 0; r < p.C; r++) st_cluster_u32(map_to_rank(smem_u32(ctl), r), (uint32_t)item);
-        }
-        cluster_arrive();
-        cluster_wait();
-        ItemGeo it;
-        it.item = *reinterpret_cast<volatile int*>(ctl);
-        if (it.item >= p.nitems) break;
-        {
-            const int seg = it.item % p.nseg;
-            const int bt = it.item / p.nseg;
-            const int tile = p.tile_order[bt % p.ntiles];
-            it.b = bt / p.ntiles;
-            it.t0 = seg * p.F;
-            it.t1 = min(p.T, it.t0 + p.F);
-            it.halo = it.t0 > 0;
-            it.tstart = it.t0 - it.halo;
-            it.n = it.t1 - it.tstart;
-            it.last_seg = it.t1 == p.T;
-            it.y0 = (tile / p.Wt) * 4;
-            it.x0 = (tile % p.Wt) * 4;
-            const int rows = min(4, p.H - it.y0), cols = min(4, p.W - it.x0);
-            it.vmask = 0;
-            for (int c = 0; c < 16; c++)
-                if ((c >> 2) < rows && (c & 3) < cols) it.vmask |= 1u << c;
-            it.nvalid = __popc(it.vmask);
-        }
-        // per-item set-up: zero the rows of cells outside the grid, pooling weights, piece table
-        if (!is_dec) {
-            for (int s = 0; s < p.R; s++)
-                for (int c = 0; c < 16; c++)
-                    if (!((it.vmask >> c) & 1u))
-                        for (int k = tid * 4; k < p.row_bytes; k += nworkers * 4)
-                            *reinterpret_cast<uint32_t*>(ring + (size_t)s * p.slot_bytes + c * p.row_bytes + k) = 0u;
-        } else {
-            if (lane < 16) {
-                const int c = lane;
-                const uint32_t qm = quad_mask(c);
-                const int nq = __popc(it.vmask & qm);
-                int quads = 0;
-                for (int q = 0; q < 4; q++) quads += (it.vmask & (0x33u << (8 * (q >> 1) + 2 * (q & 1)))) ? 1 : 0;
-                const bool valid = (it.vmask >> c) & 1u;
-                const float inv1 = nq ? 1.f / (float)nq : 0.f;
-                W1s[c] = p.L >= 2 ? inv1 : 0.f;      // per quad: also on lanes of cells outside the grid
-                W2s[c] = p.L == 3 && valid ? inv1 * (1.f / (float)quads) : 0.f;
+    if (warp < p.NM) {
+        // ------------------------------------ Gram warps ------------------------------------
+        const int nthr = p.NM * 32;
+        const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
+        const uint32_t loff = lrow * p.row_bytes + lk * 2;
+        const int ksteps = p.S >> 4;
+        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+            if (skip) continue;
+            const float* W1s = wtab + it.cls * 32;
+            const float* W2s = W1s + 16;
+            for (int j = 0; j < it.n; j++, q++) {
+                const int s = q % p.R;
+                mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
+                __syncwarp();
+                float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
+                float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+                float h0[4] = {0.f, 0.f, 0.f, 0.f}, h1[4] = {0.f, 0.f, 0.f, 0.f};
+                float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint32_t cur = ring_base + s * p.slot_bytes + loff;
+                const uint32_t prv = ring_base + ((q + p.R - 1) % p.R) * p.slot_bytes + loff;
+                // two independent accumulator sets keep more tensor-core operations in flight
+                for (int ks = warp; ks < ksteps; ks += 2 * p.NM) {
+                    uint32_t a[4], b[4], a2[4], b2[4];
+                    const bool second = ks + p.NM < ksteps;
+                    ldmatrix_x4(cur + ks * 32, a);
+                    ldmatrix_x4(prv + ks * 32, b);
+                    if (second) {
+                        ldmatrix_x4(cur + (ks + p.NM) * 32, a2);
+                        ldmatrix_x4(prv + (ks + p.NM) * 32, b2);
+                    }
+                    mma_bf16(g0, a, a[0], a[2]);
+                    mma_bf16(g1, a, a[1], a[3]);
+                    mma_bf16(c0, a, b[0], b[2]);
+                    mma_bf16(c1, a, b[1], b[3]);
+                    if (second) {
+                        mma_bf16(h0, a2, a2[0], a2[2]);
+                        mma_bf16(h1, a2, a2[1], a2[3]);
+                        mma_bf16(e0, a2, b2[0], b2[2]);
+                        mma_bf16(e1, a2, b2[1], b2[3]);
+                    }
+                }
+                {
+                    float* r = red + warp * kGramVals;
+                    const int gr = lane >> 2, gc = (lane & 3) * 2;
+                    *reinterpret_cast<float2*>(r + gr * 16 + gc) = make_float2(g0[0] + h0[0], g0[1] + h0[1]);
+                    *reinterpret_cast<float2*>(r + (gr + 8) * 16 + gc) = make_float2(g0[2] + h0[2], g0[3] + h0[3]);
+                    *reinterpret_cast<float2*>(r + gr * 16 + 8 + gc) = make_float2(g1[0] + h1[0], g1[1] + h1[1]);
+                    *reinterpret_cast<float2*>(r + (gr + 8) * 16 + 8 + gc) = make_float2(g1[2] + h1[2], g1[3] + h1[3]);
+                    *reinterpret_cast<float2*>(r + 256 + gr * 16 + gc) = make_float2(c0[0] + e0[0], c0[1] + e0[1]);
+                    *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + gc) = make_float2(c0[2] + e0[2], c0[3] + e0[3]);
+                    *reinterpret_cast<float2*>(r + 256 + gr * 16 + 8 + gc) = make_float2(c1[0] + e1[0], c1[1] + e1[1]);
+                    *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + 8 + gc) =
+                        make_float2(c1[2] + e1[2], c1[3] + e1[3]);
+                }
+                named_sync(1, nthr);
+                // this warp is done with the previous frame's slot (the current one stays for the next frame)
+                if (lane == 0 && q >= 1) mbar_arrive(empty_bar + 8 * ((q - 1) % p.R));
+                // add the warps' parts, each thread a share of the 512 entries
+                for (int i = tid * 4; i < kGramVals; i += nthr * 4) {
+                    float4 sum = *reinterpret_cast<const float4*>(red + i);
+                    for (int w = 1; w < p.NM; w++) {
+                        const float4 v = *reinterpret_cast<const float4*>(red + w * kGramVals + i);
+                        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+                    }
+                    *reinterpret_cast<float4*>(redsum + i) = sum;
+                }
+                named_sync(2, nthr);
+                // contract to 8 numbers per cell and send this CTA's share to every CTA of the cluster
+                const int xb = q % kRecRing;
+                if (q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
+                for (int i = tid; i < kSumVals; i += nthr) {
+                    const float sum = combine_sums(redsum, i & 15, i >> 4, it.vmask, W1s, W2s);
+                    const uint32_t a = smem_u32(xchg + (xb * p.C + rank) * kSumVals + i);
+                    for (int r = 0; r < p.C; r++)
+                        st_async_f32(map_to_rank(a, r), sum, map_to_rank(xfull_bar + 8 * xb, r));
+                }
             }
-            if (rank == 0) p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
         }
-        __syncthreads();
-
-        auto issue = [&](int j) {      // called by the whole warp 0
-            const int q = qbase + j, s = q % p.R;
-            const uint32_t bar = smem_u32(full_bar + s);
-            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
+    } else if (warp < w_sim) {
+        // ------------------------------------ sum warps ------------------------------------
+        ChainAcc acc;
+        acc.clear();
+        const int quad = tid - p.NM * 32;                    // channels 4*quad .. 4*quad+3 of this CTA's slice
+        const bool active = 4 * quad < p.S;
+        const long long ch4 = ((long long)rank * p.S >> 2) + quad, D4 = p.D >> 2;
+        int total = 0;
+        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
+            if (!skip) total += it.n;
+        // one record per frame, and a last one that only writes out what the last item left
+        for (; q <= total; q++) {
+            const int rk = q % kRecRing, s = q % p.R;
+            mbar_wait(rfull_bar + 8 * rk, q / kRecRing, timed_out);
+            if (q < total) mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
             __syncwarp();
-            if (lane < 16 && ((it.vmask >> lane) & 1u)) {
-                const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW + (it.y0 + (lane >> 2)) * p.W +
-                                       it.x0 + (lane & 3);
-                bulk_g2s(ring_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
-                         (uint32_t)(p.S * 2), bar);
+            const FrameRec* rec = recs + rk;
+            const uint32_t fb = ring_base + s * p.slot_bytes + quad * 8;
+            const float* W2s = wtab + rec->cls * 32 + 16;
+            const int n_flush = rec->n_flush, n_nodes = rec->n_nodes;
+#pragma unroll 1
+            for (int i = 0; i < n_flush; i++) {
+                const FlushCmd fc = rec->flush[i];
+                float4 v = acc.take(fc.slot);
+                if (active) {
+                    if (fc.kind == 0) {
+                        v.x = v.x / fc.weight; v.y = v.y / fc.weight; v.z = v.z / fc.weight; v.w = v.w / fc.weight;
+                        if (p.out_f32) reinterpret_cast<float4*>(p.staging)[(long long)fc.dst * D4 + ch4] = v;
+                        else reinterpret_cast<uint2*>(p.staging)[(long long)fc.dst * D4 + ch4] = pack_bf16x4(v);
+                    } else {
+                        reinterpret_cast<float4*>(p.pieces)[(long long)fc.dst * D4 + ch4] = v;
+                    }
+                }
             }
-        };
-        if (warp == 0)
-            for (int j = 0; j < min(p.R, it.n); j++) issue(j);
-
-        if (!is_dec) {
-            // ------------------------------ worker warps ------------------------------
-            const int pair = tid;                       // channels 2*pair, 2*pair+1 of this CTA's slice
-            const bool active = 2 * pair < p.S;
-            for (int j = 0; j < it.n + 2; j++) {
-                if (j < it.n) {
-                    const int q = qbase + j, s = q % p.R;
-                    const uint32_t bar = smem_u32(full_bar + s), parity = (uint32_t)((q / p.R) & 1);
-                    int spins = 0;
-                    while (!timed_out && !mbar_try_wait(bar, parity)) {
-                        if (++spins > kSpinLimit) timed_out = true;
-                    }
-                    if (warp < p.NM) {
-                        // Gram and cross matrices over this warp's share of the channels
-                        // two independent accumulator sets keep twice as many tensor-core operations in flight
-                        float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
-                        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-                        float h0[4] = {0.f, 0.f, 0.f, 0.f}, h1[4] = {0.f, 0.f, 0.f, 0.f};
-                        float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
-                        const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
-                        const uint32_t cur = ring_base + s * p.slot_bytes + lrow * p.row_bytes + lk * 2;
-                        const int sp = (q - 1 + p.R) % p.R;
-                        const uint32_t prv = ring_base + sp * p.slot_bytes + lrow * p.row_bytes + lk * 2;
-                        const int ksteps = p.S >> 4;
-                        if (j > 0) {
-                            for (int ks = warp; ks < ksteps; ks += 2 * p.NM) {
-                                uint32_t a[4], b[4];
-                                ldmatrix_x4(cur + ks * 32, a);
-                                ldmatrix_x4(prv + ks * 32, b);
-                                mma_bf16(g0, a, a[0], a[2]);
-                                mma_bf16(g1, a, a[1], a[3]);
-                                mma_bf16(c0, a, b[0], b[2]);
-                                mma_bf16(c1, a, b[1], b[3]);
-                                if (ks + p.NM < ksteps) {
-                                    ldmatrix_x4(cur + (ks + p.NM) * 32, a);
-                                    ldmatrix_x4(prv + (ks + p.NM) * 32, b);
-                                    mma_bf16(h0, a, a[0], a[2]);
-                                    mma_bf16(h1, a, a[1], a[3]);
-                                    mma_bf16(e0, a, b[0], b[2]);
-                                    mma_bf16(e1, a, b[1], b[3]);
-                                }
-                            }
-                        } else {
-                            for (int ks = warp; ks < ksteps; ks += 2 * p.NM) {
-                                uint32_t a[4];
-                                ldmatrix_x4(cur + ks * 32, a);
-                                mma_bf16(g0, a, a[0], a[2]);
-                                mma_bf16(g1, a, a[1], a[3]);
-                                if (ks + p.NM < ksteps) {
-                                    ldmatrix_x4(cur + (ks + p.NM) * 32, a);
-                                    mma_bf16(h0, a, a[0], a[2]);
-                                    mma_bf16(h1, a, a[1], a[3]);
-                                }
-                            }
+#pragma unroll 1
+            for (int i = 0; i < n_nodes; i++) {
+                const NodeCmd nc = rec->node[i];
+                const int lv = nc.lv & 3;
+                float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (active) {
+                    const uint32_t a0 = fb + nc.cell * p.row_bytes;
+                    if (lv == 0) {
+                        f = unpack_bf16x4(lds_u64(a0));
+                    } else if (lv == 1) {
+                        const int m = nc.lv >> 4;           // which of the block's four cells exist
+                        f = unpack_bf16x4(lds_u64(a0));
+                        if (m & 2) {
+                            const float4 u = unpack_bf16x4(lds_u64(a0 + p.row_bytes));
+                            f.x += u.x; f.y += u.y; f.z += u.z; f.w += u.w;
                         }
-#pragma unroll
-                        for (int i = 0; i < 4; i++) { g0[i] += h0[i]; g1[i] += h1[i]; c0[i] += e0[i]; c1[i] += e1[i]; }
-                        float* r = red + warp * kGramVals;
-                        const int gr = lane >> 2, gc = (lane & 3) * 2;
-                        *reinterpret_cast<float2*>(r + gr * 16 + gc) = make_float2(g0[0], g0[1]);
-                        *reinterpret_cast<float2*>(r + (gr + 8) * 16 + gc) = make_float2(g0[2], g0[3]);
-                        *reinterpret_cast<float2*>(r + gr * 16 + 8 + gc) = make_float2(g1[0], g1[1]);
-                        *reinterpret_cast<float2*>(r + (gr + 8) * 16 + 8 + gc) = make_float2(g1[2], g1[3]);
-                        *reinterpret_cast<float2*>(r + 256 + gr * 16 + gc) = make_float2(c0[0], c0[1]);
-                        *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + gc) = make_float2(c0[2], c0[3]);
-                        *reinterpret_cast<float2*>(r + 256 + gr * 16 + 8 + gc) = make_float2(c1[0], c1[1]);
-                        *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + 8 + gc) = make_float2(c1[2], c1[3]);
-                    }
-                }
-                named_sync(1, nworkers);
-                if (j < it.n) {
-                    // contract the warps' partial matrices to the 8 numbers per cell and hand the CTA's
-                    // share to every CTA of the cluster
-                    for (int i = tid; i < kSumVals; i += nworkers) {
-                        const float sum = combine_sums(red, p.NM, i & 15, i >> 4, W1s, W2s);
-                        const uint32_t a = smem_u32(xchg + ((qbase + j) & 1) * p.C * kSumVals + rank * kSumVals + i);
-                        for (int r = 0; r < p.C; r++) st_cluster_f32(map_to_rank(a, r), sum);
-                    }
-                }
-                cluster_arrive();
-                if (j >= 2) {
-                    // execute the record of frame j-2 on the frame still in the ring
-                    const int jj = j - 2;
-                    const int need = qbase + jj + 1;
-                    int spins = 0;
-                    while (!timed_out && ld_acquire_cta(ctl + 1) < need) {
-                        if (++spins > kSpinLimit) timed_out = true;
-                    }
-                    const FrameRec* rec = recs + ((qbase + jj) % kRecRing);
-                    const int s = (qbase + jj) % p.R;
-                    const uint32_t fb = ring_base + s * p.slot_bytes + pair * 4;
-                    const long long ch2 = ((long long)rank * p.S >> 1) + pair;      // index in units of 2 channels
-                    const long long D2 = p.D >> 1;
-                    auto flush = [&](const FlushCmd& fc) {
-                        float2 v = acc.take(fc.slot);
-                        if (!active) return;
-                        if (fc.kind == 0) {
-                            v.x = v.x / fc.weight;
-                            v.y = v.y / fc.weight;
-                            if (p.out_f32) reinterpret_cast<float2*>(p.staging)[(long long)fc.dst * D2 + ch2] = v;
-                            else reinterpret_cast<uint32_t*>(p.staging)[(long long)fc.dst * D2 + ch2] = pack_bf16x2(v);
-                        } else {
-                            reinterpret_cast<float2*>(p.pieces)[(long long)fc.dst * D2 + ch2] = v;
+                        if (m & 4) {
+                            const float4 u = unpack_bf16x4(lds_u64(a0 + 4 * p.row_bytes));
+                            f.x += u.x; f.y += u.y; f.z += u.z; f.w += u.w;
                         }
-                    };
-                    const int n_pre = rec->n_pre, n_nodes = rec->n_nodes, n_post = rec->n_post;
-                    for (int i = 0; i < n_pre; i++) flush(rec->pre[i]);
-                    for (int i = 0; i < n_nodes; i++) {
-                        const NodeCmd nc = rec->node[i];
-                        float2 f = make_float2(0.f, 0.f);
-                        if (active) {
-                            const uint32_t a0 = fb + nc.cell * p.row_bytes;
-                            if (nc.lv == 0) {
-                                f = unpack_bf16x2(lds_u32(a0));
-                            } else if (nc.lv == 1) {
-                                const float2 u0 = unpack_bf16x2(lds_u32(a0)), u1 = unpack_bf16x2(lds_u32(a0 + p.row_bytes));
-                                const float2 u2 = unpack_bf16x2(lds_u32(a0 + 4 * p.row_bytes));
-                                const float2 u3 = unpack_bf16x2(lds_u32(a0 + 5 * p.row_bytes));
-                                f.x = (u0.x + u1.x) + (u2.x + u3.x);
-                                f.y = (u0.y + u1.y) + (u2.y + u3.y);
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < 16; c++) {
-                                    const float2 u = unpack_bf16x2(lds_u32(fb + c * p.row_bytes));
-                                    f.x = fmaf(W2s[c], u.x, f.x);
-                                    f.y = fmaf(W2s[c], u.y, f.y);
-                                }
-                            }
-                            f.x *= nc.w;
-                            f.y *= nc.w;
+                        if (m & 8) {
+                            const float4 u = unpack_bf16x4(lds_u64(a0 + 5 * p.row_bytes));
+                            f.x += u.x; f.y += u.y; f.z += u.z; f.w += u.w;
                         }
-                        acc.add(nc.slot, f);
+                    } else {
+#pragma unroll 2
+                        for (int c = 0; c < 16; c++) {
+                            const float4 u = unpack_bf16x4(lds_u64(fb + c * p.row_bytes));
+                            const float w = W2s[c];
+                            f.x = fmaf(w, u.x, f.x); f.y = fmaf(w, u.y, f.y);
+                            f.z = fmaf(w, u.z, f.z); f.w = fmaf(w, u.w, f.w);
+                        }
                     }
-                    for (int i = 0; i < n_post; i++) flush(rec->post[i]);
+                    f.x *= nc.w; f.y *= nc.w; f.z *= nc.w; f.w *= nc.w;
                 }
-                cluster_wait();
-                named_sync(1, nworkers);
-                if (warp == 0 && j >= 2 && j - 2 + p.R < it.n) issue(j - 2 + p.R);
+                acc.add(nc.slot, f);
             }
-        } else {
-            // ------------------------------ decision warp ------------------------------
-            DecState st;
-            st.prev_lv = 0; st.prev_slot = 0; st.prev_nk = 0.f;
-            st.active = 0;
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(rempty_bar + 8 * rk);
+                if (q < total) mbar_arrive(empty_bar + 8 * s);
+            }
+        }
+    } else if (warp == w_sim) {
+        // --------------------------------- similarity warp ---------------------------------
+        // lane c (and its mirror c + 16) = cell c of the tile
+        const unsigned full = 0xffffffffu;
+        const int c = lane & 15;
+        const int L = p.L;
+        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+            if (skip) continue;
             const float tau_s = taus.s[it.b], tau_t = taus.t[it.b];
-            cluster_arrive();
-            for (int j = 0; j < it.n + 2; j++) {
-                cluster_wait();
-                // take this frame's totals out of the exchange buffer, then let the cluster go on:
-                // the decisions themselves run beside the workers' next frame
+            const float w1 = wtab[it.cls * 32 + c], w2 = wtab[it.cls * 32 + 16 + c];
+            const bool valid = (it.vmask >> c) & 1u;
+            const uint32_t qm = quad_mask(c);
+            int prev_lv = 0;
+            float prev_nk = 0.f;
+            for (int j = 0; j < it.n; j++, q++) {
+                const int xb = q % kRecRing;
+                if (lane == 0) mbar_expect_tx(xfull_bar + 8 * xb, (uint32_t)(p.C * kSumVals * 4));
+                mbar_wait(xfull_bar + 8 * xb, q / kRecRing, timed_out);
+                __syncwarp();
                 float v[8];
-                if (j < it.n) {
-                    const float* xch = xchg + ((qbase + j) & 1) * p.C * kSumVals;
+                {
+                    const float* xch = xchg + xb * p.C * kSumVals;
 #pragma unroll
                     for (int k = 0; k < 8; k++) {
                         float sum = 0.f;
-                        for (int r = 0; r < p.C; r++) sum += xch[r * kSumVals + k * 16 + (lane & 15)];
-                        v[k] = sum;
+                        for (int r = 0; r < p.C; r++) sum += xch[r * kSumVals + k * 16 + c];
+                        v[k] = valid ? sum : 0.f;       // cells outside the grid: stale ring rows, dropped
                     }
                 }
-                if (j + 1 < it.n + 2) cluster_arrive();
-                if (j < it.n) {
-                    FrameRec* rec = recs + ((qbase + j) % kRecRing);
-                    decide_frame(p, it, j, tau_s, tau_t, v, W1s, W2s, st, tab, rec, rank, lane);
-                    if (lane == 0) st_release_cta(ctl + 1, qbase + j + 1);
+                __syncwarp();
+                if (lane < p.C) mbar_arrive_remote(map_to_rank(xempty_bar + 8 * xb, lane));
+
+                // Section 3.2: cosine of every node with its parent, then the coarse-to-fine search
+                const float n0 = v[0], d0 = v[1], rr = v[2];
+                const float n1 = w1 * quad_sum(d0);              // |parent|^2
+                const float d1 = w1 * quad_sum(rr);              // parent . top
+                const float n2 = half_warp_sum(w2 * rr);         // |top|^2
+                int lv = 0;
+                if (L >= 2) {
+                    const bool p0 = !valid || cos_above(d0, n0, n1, tau_s);
+                    const uint32_t pm0 = __ballot_sync(full, p0) & 0xffffu;
+                    const bool quad_pass = (pm0 & qm) == qm;
+                    if (L == 3) {
+                        const bool quad_exists = (it.vmask & qm) != 0;
+                        const bool p1 = !quad_exists || cos_above(d1, n1, n2, tau_s);
+                        const uint32_t pm1 = __ballot_sync(full, p1) & 0xffffu;
+                        lv = pm1 == 0xffffu ? 2 : (quad_pass ? 1 : 0);
+                    } else {
+                        lv = quad_pass ? 1 : 0;
+                    }
+                }
+                const float nk = lv == 0 ? n0 : (lv == 1 ? n1 : n2);
+
+                // Section 3.3: the node covering the cell against the overlapping kept node of the
+                // previous frame; a pair is evaluated at the top-left cell of its finer node
+                int link_local = -1;
+                if (j > 0) {
+                    const int lu = prev_lv;
+                    const float t11 = w1 * quad_sum(v[4]), t12 = w1 * quad_sum(v[5]);
+                    const float t21 = w1 * quad_sum(v[7]), t22 = half_warp_sum(w2 * v[5]);
+                    float dot;
+                    if (lv == 0) dot = lu == 0 ? v[3] : (lu == 1 ? v[4] : v[5]);
+                    else if (lv == 1) dot = lu == 0 ? v[6] : (lu == 1 ? t11 : t12);
+                    else dot = lu == 0 ? v[7] : (lu == 1 ? t21 : t22);
+                    const bool rep = valid && tile_anchor(c, min(lv, lu)) == c;
+                    const bool pass = rep && cos_above(dot, nk, prev_nk, tau_t);
+                    const uint32_t passm = __ballot_sync(full, pass) & 0xffffu;
+                    const uint32_t cand = passm & region_mask(c, lv);
+                    const int cstar = cand ? __ffs(cand) - 1 : 0;     // first in row-major order: the top-left one
+                    const int lu_star = __shfl_sync(full, lu, cstar);
+                    link_local = cand ? tile_anchor(cstar, lu_star) : -1;
+                }
+                prev_lv = lv;
+                prev_nk = nk;
+
+                // hand the cover level and the link of every cell to the chain warp
+                if (q >= kRecRing) mbar_wait(hempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
+                __syncwarp();
+                if (lane < 16) hand[xb * 16 + c] = lv | ((link_local + 1) << 8);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(hfull_bar + 8 * xb);
+            }
+        }
+    } else if (warp == w_chain) {
+        // ------------------------------------ chain warp ------------------------------------
+        const unsigned full = 0xffffffffu;
+        const int c = lane & 15;
+        const bool low = lane < 16;
+        // what the previous item left running when it ended: written out by the next record
+        FlushCmd carry = FlushCmd{0, 0, 0, 0.f};     // lane s < 16: slot s
+        uint32_t carry_mask = 0;
+        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+            if (skip) continue;
+            const bool valid = (it.vmask >> c) & 1u;
+            const float w1 = wtab[it.cls * 32 + c];
+            if (rank == 0) p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
+            int prev_slot = 0;
+            uint32_t active_slots = 0;
+            for (int j = 0; j < it.n; j++, q++) {
+                const int hb = q % kRecRing;
+                mbar_wait(hfull_bar + 8 * hb, q / kRecRing, timed_out);
+                __syncwarp();
+                const int packed = hand[hb * 16 + c];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(hempty_bar + 8 * hb);
+                const int lv = packed & 3, link_local = (packed >> 8) - 1;
+                if (q >= kRecRing) mbar_wait(rempty_bar + 8 * hb, q / kRecRing - 1, timed_out);
+                __syncwarp();
+                FrameRec* rec = recs + hb;
+                const int t = it.tstart + j;
+                const bool is_halo = it.halo && j == 0;
+                const bool is_last = j == it.n - 1;
+
+                // nodes with a link join the chain of their target; chains without a member in this
+                // frame have ended; the remaining nodes start new chains in free slots
+                const bool anchor = valid && tile_anchor(c, lv) == c;
+                const bool linked = anchor && link_local >= 0;
+                const bool fresh = anchor && link_local < 0;
+                const int slot_linked = __shfl_sync(full, prev_slot, link_local < 0 ? 0 : link_local);
+                const uint32_t memb = __reduce_or_sync(full, linked ? 1u << slot_linked : 0u);
+                const uint32_t dead = active_slots & ~memb;
+                const uint32_t freem = ~memb & 0xffffu;
+                const uint32_t freshm = __ballot_sync(full, fresh && low);
+                const int slot_fresh = kth_set_bit16(freem, __popc(freshm & ((1u << c) - 1)));
+                const int node_slot = linked ? slot_linked : slot_fresh;
+                const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + tile_anchor(c, lv));
+                const uint32_t cells = it.vmask & region_mask(c, lv);
+                const int wint = p.weight_mode ? __popc(cells) : 1;
+                const long long gc =
+                    (long long)it.b * p.N + (long long)t * p.HW + (it.y0 + (c >> 2)) * p.W + it.x0 + (c & 3);
+
+                // chains that ended: lane s looks at slot s (before the slot is given away again); at
+                // the first frame of an item nothing of the item runs yet and the list is the carry
+                if (low && ((dead >> lane) & 1u)) {
+                    const int at = __popc(dead & ((1u << lane) - 1));
+                    if (tab->virt[lane]) {
+                        const int pc = it.item * kPieceSlots + tab->cell[lane];
+                        rec->flush[at] = FlushCmd{lane, 1, pc, 0.f};
+                        if (rank == 0) p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
+                    } else {
+                        rec->flush[at] = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
+                    }
+                }
+                if (low && ((carry_mask >> lane) & 1u))
+                    rec->flush[__popc(dead) + __popc(carry_mask & ((1u << lane) - 1))] = carry;
+                const int n_flush = __popc(dead) + __popc(carry_mask);
+                carry_mask = 0;
+                __syncwarp();
+                if (low && fresh) {
+                    tab->key[slot_fresh] = (int)gc;
+                    tab->weight[slot_fresh] = is_halo ? 0 : wint;
+                    tab->virt[slot_fresh] = is_halo ? 1 : 0;
+                    tab->cell[slot_fresh] = c;
+                }
+                if (low && linked) atomicAdd(&tab->weight[slot_linked], wint);
+                const uint32_t anchorm = __ballot_sync(full, anchor && low);
+                if (low && anchor && !is_halo) {
+                    const float wn = lv == 1 ? w1 * (float)wint : (float)wint;
+                    const int cm = (int)((cells >> c) & 1u) | (int)((cells >> (c + 1)) & 1u) << 1 |
+                                   (int)((cells >> (c + 4)) & 1u) << 2 | (int)((cells >> (c + 5)) & 1u) << 3;
+                    rec->node[__popc(anchorm & ((1u << c) - 1))] = NodeCmd{c, lv | (cm << 4), node_slot, wn};
+                }
+                const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
+                __syncwarp();
+
+                if (rank == 0 && !is_halo && low && valid) {
+                    p.cover[gc] = (int8_t)lv;
+                    p.link[gc] = link_local < 0 ? -1
+                                                : (t - 1) * p.HW + (it.y0 + (link_local >> 2)) * p.W + it.x0 +
+                                                      (link_local & 3);
+                    p.chain_key[gc] = tab->key[cur_slot] - it.b * p.N;
+                }
+                if (is_last) {
+                    // the item ends: everything still running is written out by the next record
+                    carry_mask = active;
+                    if (low && ((active >> lane) & 1u)) {
+                        if (!tab->virt[lane] && it.last_seg) {
+                            carry = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
+                        } else {
+                            const int pc = it.item * kPieceSlots + 16 + lane;
+                            carry = FlushCmd{lane, 1, pc, 0.f};
+                            if (rank == 0) p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
+                        }
+                    }
+                }
+                if (lane == 0) {
+                    rec->n_flush = n_flush;
+                    rec->n_nodes = is_halo ? 0 : __popc(anchorm);
+                    rec->cls = it.cls;
+                }
+                active_slots = is_last ? 0u : active;
+                prev_slot = cur_slot;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
+            }
+        }
+        {
+            // last record: only the carry of the last item
+            const int hb = q % kRecRing;
+            if (q >= kRecRing) mbar_wait(rempty_bar + 8 * hb, q / kRecRing - 1, timed_out);
+            __syncwarp();
+            FrameRec* rec = recs + hb;
+            if (low && ((carry_mask >> lane) & 1u)) rec->flush[__popc(carry_mask & ((1u << lane) - 1))] = carry;
+            if (lane == 0) {
+                rec->n_flush = __popc(carry_mask);
+                rec->n_nodes = 0;
+                rec->cls = 0;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
+        }
+    } else if (warp == w_prod) {
+        // ----------------------------------- producer warp -----------------------------------
+        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+            if (skip) continue;
+            for (int j = 0; j < it.n; j++, q++) {
+                const int s = q % p.R;
+                const uint32_t bar = full_bar + 8 * s;
+                if (q >= p.R) mbar_wait(empty_bar + 8 * s, q / p.R - 1, timed_out);
+                __syncwarp();
+                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
+                __syncwarp();
+                if (lane < 16 && ((it.vmask >> lane) & 1u)) {
+                    const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
+                                           (it.y0 + (lane >> 2)) * p.W + it.x0 + (lane & 3);
+                    bulk_g2s(ring_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
+                             (uint32_t)(p.S * 2), bar);
                 }
             }
         }
-        qbase += it.n;
-        __syncthreads();
     }
+    // nobody leaves while a CTA of the cluster may still store into it or signal its barriers
+    __syncwarp();
+    cluster_arrive();
+    cluster_wait();
     if (timed_out && p.status != nullptr) atomicOr(p.status, kStatusWaitTimeout);
 }
 
@@ -772,18 +884,46 @@ k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict
                 }
             }
         } else {
+            // the row's pieces in increasing index order; lists are short (a few per item border),
+            // so the first eight are found once and kept in registers
+            constexpr int kMaxList = 8;
+            int ids[kMaxList];
+            int n = 0, last = -1;
+            bool longer = false;
+            while (true) {
+                int best = 0x7fffffff;
+                for (int pc = head; pc >= 0; pc = piece_next[pc])
+                    if (pc > last && pc < best) best = pc;
+                if (best == 0x7fffffff) break;
+                if (n == kMaxList) { longer = true; break; }
+#pragma unroll
+                for (int k = 0; k < kMaxList; k++)
+                    if (k == n) ids[k] = best;
+                n++;
+                last = best;
+            }
             const float wsum = (float)row_weight[r];
             for (int d = lane * VEC; d < g.D; d += kSliceCh) {
                 float sum[VEC] = {0.f, 0.f, 0.f, 0.f};
-                int last = -1;
-                while (true) {          // next larger piece index on the row's (short) list
-                    int best = 0x7fffffff;
-                    for (int pc = head; pc >= 0; pc = piece_next[pc])
-                        if (pc > last && pc < best) best = pc;
-                    if (best == 0x7fffffff) break;
-                    const float4 v = *reinterpret_cast<const float4*>(pieces + (long long)best * g.D + d);
-                    sum[0] += v.x; sum[1] += v.y; sum[2] += v.z; sum[3] += v.w;
-                    last = best;
+                if (!longer) {
+#pragma unroll
+                    for (int k = 0; k < kMaxList; k++) {
+                        if (k < n) {
+                            const float4 v = *reinterpret_cast<const float4*>(pieces + (long long)ids[k] * g.D + d);
+                            sum[0] += v.x; sum[1] += v.y; sum[2] += v.z; sum[3] += v.w;
+                        }
+                    }
+                } else {
+                    int lst = -1;
+                    while (true) {
+                        int best = 0x7fffffff;
+                        for (int pc = head; pc >= 0; pc = piece_next[pc])
+                            if (pc > lst && pc < best) best = pc;
+                        if (best == 0x7fffffff) break;
+                        const float4 v = *reinterpret_cast<const float4*>(pieces + (long long)best * g.D + d);
+                        sum[0] += v.x; sum[1] += v.y; sum[2] += v.z; sum[3] += v.w;
+                        lst = best;
+                    }
                 }
 #pragma unroll
                 for (int v = 0; v < VEC; v++) sum[v] = sum[v] / wsum;

@@ -45,19 +45,21 @@ constexpr int kMaxRing = 12;
 constexpr int kMaxGramWarps = 4;
 constexpr int kMaxSumWarps = 8;         // 128 channels each: at most 1024 channels per CTA
 constexpr int kFusedMaxThreads = (kMaxGramWarps + kMaxSumWarps + 3) * 32;
-constexpr int kSpinLimit = 1 << 20;     // after the first wait that runs out, later waits are skipped
+constexpr int kSpinLimit = 1 << 12;     // tries per wait; after the first wait that runs out, later waits are skipped
+constexpr uint32_t kWaitHintNs = 1000000u;   // a try may sleep this long before it reports "not yet"
 
 enum : int { kStatusWaitTimeout = 1 << 6 };
 
 struct FlushCmd { int slot, kind, dst; float weight; };     // kind 0: finished row, 1: piece
-struct NodeCmd { int cell, lv, slot; float w; };            // lv: level | (cells of the node inside the grid) << 4
+struct CellCmd { int slot_cell; float w; };                 // slot << 8 | cell; weight of the cell in its node
 // Commands of one frame for the sum warps: first write out and clear the listed chain sums
 // (chains that got no member in this frame; at the first frame of an item: everything the
-// previous item left), then add the frame's kept nodes.
+// previous item left), then add every cell of the frame, times its weight in its kept node,
+// to the running sum of the node's chain.
 struct FrameRec {
-    int n_flush, n_nodes, cls, pad;
+    int n_flush, n_cells, pad0, pad1;
     FlushCmd flush[16];
-    NodeCmd node[16];
+    CellCmd cell[16];
 };
 
 struct FusedParams {
@@ -101,10 +103,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     return ok != 0;
 }
@@ -168,6 +170,21 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float4 lds_f32x4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint4 lds_u32x4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
     uint2 v;
     asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
@@ -198,16 +215,23 @@ __device__ __forceinline__ int kth_set_bit16(uint32_t m, int k) {
 }
 
 // running sums of the chains: 16 slots x 4 channels, in registers; the slot index is
-// uniform over the warp, so the switch does not diverge
+// uniform over the warp, so the switch does not diverge (the empty asm statements keep the
+// compiler from turning the cases into selects over all 64 registers)
 struct ChainAcc {
     float4 a[16];
     __device__ __forceinline__ void clear() {
 #pragma unroll
         for (int i = 0; i < 16; i++) a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-#define STTM_ACC_BODY(i) a[i].x += f.x; a[i].y += f.y; a[i].z += f.z; a[i].w += f.w; break;
+#define STTM_ACC_BODY(i)              \
+    asm volatile("");                 \
+    a[i].x = fmaf(w, f.x, a[i].x);    \
+    a[i].y = fmaf(w, f.y, a[i].y);    \
+    a[i].z = fmaf(w, f.z, a[i].z);    \
+    a[i].w = fmaf(w, f.w, a[i].w);    \
+    break;
 #define STTM_ACC_CASE(i) case i: STTM_ACC_BODY(i)
-    __device__ __forceinline__ void add(int slot, float4 f) {
+    __device__ __forceinline__ void fma(int slot, float w, float4 f) {
         switch (slot) {
             STTM_ACC_CASE(0) STTM_ACC_CASE(1) STTM_ACC_CASE(2) STTM_ACC_CASE(3) STTM_ACC_CASE(4) STTM_ACC_CASE(5)
             STTM_ACC_CASE(6) STTM_ACC_CASE(7) STTM_ACC_CASE(8) STTM_ACC_CASE(9) STTM_ACC_CASE(10) STTM_ACC_CASE(11)
@@ -216,7 +240,7 @@ struct ChainAcc {
     }
 #undef STTM_ACC_CASE
 #undef STTM_ACC_BODY
-#define STTM_TAKE_BODY(i) v = a[i]; a[i] = make_float4(0.f, 0.f, 0.f, 0.f); break;
+#define STTM_TAKE_BODY(i) asm volatile(""); v = a[i]; a[i] = make_float4(0.f, 0.f, 0.f, 0.f); break;
 #define STTM_TAKE_CASE(i) case i: STTM_TAKE_BODY(i)
     __device__ __forceinline__ float4 take(int slot) {
         float4 v;
@@ -303,40 +327,37 @@ __device__ __forceinline__ bool next_item(const FusedParams& p, int round, uint3
 //   k=6  parent(c)(t) . x_c(t-1)       k=7  top(t) . x_c(t-1)
 // Ring rows of cells outside the grid hold stale finite data: such columns are masked or
 // get weight 0 here, and the similarity warp drops the numbers of such cells.
-__device__ __forceinline__ float combine_sums(const float* G, int c, int k, uint32_t vmask, const float* W1s,
-                                              const float* W2s) {
-    const float* Cm = G + 256;
+__device__ __forceinline__ float combine_sums(uint32_t G, int c, int k, uint32_t vmask, uint32_t W1s, uint32_t W2s) {
+    const uint32_t Cm = G + 256 * 4;
     const int qb = tile_anchor(c, 1);
     const float m0 = (vmask >> qb) & 1u ? 1.f : 0.f, m1 = (vmask >> (qb + 1)) & 1u ? 1.f : 0.f;
     const float m2 = (vmask >> (qb + 4)) & 1u ? 1.f : 0.f, m3 = (vmask >> (qb + 5)) & 1u ? 1.f : 0.f;
     float v = 0.f;
-    switch (k) {
-        case 0: v = G[c * 16 + c]; break;
-        case 1:
-            v = ((m0 * G[c * 16 + qb] + m1 * G[c * 16 + qb + 1]) + (m2 * G[c * 16 + qb + 4] + m3 * G[c * 16 + qb + 5])) *
-                W1s[c];
-            break;
-        case 2:
+    if (k == 0) {
+        v = lds_f32(G + (c * 16 + c) * 4);
+    } else if (k == 3) {
+        v = lds_f32(Cm + (c * 16 + c) * 4);
+    } else if (k == 1 || k == 4 || k == 6) {
+        // the four cells of the 2x2 block: along the row of c (k = 1, 4) or down its column (k = 6)
+        const uint32_t M = k == 1 ? G : Cm;
+        const int step = k == 6 ? 16 : 1;
+        const uint32_t a = M + (k == 6 ? (qb * 16 + c) : (c * 16 + qb)) * 4;
+        const float x0 = lds_f32(a), x1 = lds_f32(a + step * 4), x2 = lds_f32(a + 4 * step * 4),
+                    x3 = lds_f32(a + 5 * step * 4);
+        v = ((m0 * x0 + m1 * x1) + (m2 * x2 + m3 * x3)) * lds_f32(W1s + c * 4);
+    } else {
+        // weighted sum over all 16 cells: along the row of c (k = 2, 5) or down its column (k = 7)
+        const uint32_t M = k == 2 ? G : Cm;
+        if (k == 7) {
 #pragma unroll
-            for (int i = 0; i < 16; i++) v = fmaf(W2s[i], G[c * 16 + i], v);
-            break;
-        case 3: v = Cm[c * 16 + c]; break;
-        case 4:
-            v = ((m0 * Cm[c * 16 + qb] + m1 * Cm[c * 16 + qb + 1]) +
-                 (m2 * Cm[c * 16 + qb + 4] + m3 * Cm[c * 16 + qb + 5])) * W1s[c];
-            break;
-        case 5:
+            for (int i = 0; i < 16; i++) v = fmaf(lds_f32(W2s + i * 4), lds_f32(M + (i * 16 + c) * 4), v);
+        } else {
 #pragma unroll
-            for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[c * 16 + i], v);
-            break;
-        case 6:
-            v = ((m0 * Cm[qb * 16 + c] + m1 * Cm[(qb + 1) * 16 + c]) +
-                 (m2 * Cm[(qb + 4) * 16 + c] + m3 * Cm[(qb + 5) * 16 + c])) * W1s[c];
-            break;
-        default:
-#pragma unroll
-            for (int i = 0; i < 16; i++) v = fmaf(W2s[i], Cm[i * 16 + c], v);
-            break;
+            for (int i = 0; i < 16; i += 4) {
+                const float4 w = lds_f32x4(W2s + i * 4), x = lds_f32x4(M + (c * 16 + i) * 4);
+                v = fmaf(w.x, x.x, v); v = fmaf(w.y, x.y, v); v = fmaf(w.z, x.z, v); v = fmaf(w.w, x.w, v);
+            }
+        }
     }
     return v;
 }
@@ -417,10 +438,10 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
         const uint32_t loff = lrow * p.row_bytes + lk * 2;
         const int ksteps = p.S >> 4;
+        const uint32_t red_a = smem_u32(red), redsum_a = smem_u32(redsum);
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
-            const float* W1s = wtab + it.cls * 32;
-            const float* W2s = W1s + 16;
+            const uint32_t W1s = smem_u32(wtab + it.cls * 32), W2s = W1s + 64;
             for (int j = 0; j < it.n; j++, q++) {
                 const int s = q % p.R;
                 mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
@@ -470,9 +491,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (lane == 0 && q >= 1) mbar_arrive(empty_bar + 8 * ((q - 1) % p.R));
                 // add the warps' parts, each thread a share of the 512 entries
                 for (int i = tid * 4; i < kGramVals; i += nthr * 4) {
-                    float4 sum = *reinterpret_cast<const float4*>(red + i);
+                    float4 sum = lds_f32x4(red_a + i * 4);
                     for (int w = 1; w < p.NM; w++) {
-                        const float4 v = *reinterpret_cast<const float4*>(red + w * kGramVals + i);
+                        const float4 v = lds_f32x4(red_a + (w * kGramVals + i) * 4);
                         sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
                     }
                     *reinterpret_cast<float4*>(redsum + i) = sum;
@@ -482,7 +503,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const int xb = q % kRecRing;
                 if (q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
                 for (int i = tid; i < kSumVals; i += nthr) {
-                    const float sum = combine_sums(redsum, i & 15, i >> 4, it.vmask, W1s, W2s);
+                    const float sum = combine_sums(redsum_a, i & 15, i >> 4, it.vmask, W1s, W2s);
                     const uint32_t a = smem_u32(xchg + (xb * p.C + rank) * kSumVals + i);
                     for (int r = 0; r < p.C; r++)
                         st_async_f32(map_to_rank(a, r), sum, map_to_rank(xfull_bar + 8 * xb, r));
@@ -493,9 +514,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // ------------------------------------ sum warps ------------------------------------
         ChainAcc acc;
         acc.clear();
-        const int quad = tid - p.NM * 32;                    // channels 4*quad .. 4*quad+3 of this CTA's slice
-        const bool active = 4 * quad < p.S;
+        const int quad_raw = tid - p.NM * 32;                // channels 4*quad .. 4*quad+3 of this CTA's slice
+        const bool active = 4 * quad_raw < p.S;
+        const int quad = active ? quad_raw : 0;              // idle lanes of the last warp shadow thread 0, write nothing
         const long long ch4 = ((long long)rank * p.S >> 2) + quad, D4 = p.D >> 2;
+        const uint32_t recs_a = smem_u32(recs);
         int total = 0;
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
             if (!skip) total += it.n;
@@ -505,60 +528,31 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             mbar_wait(rfull_bar + 8 * rk, q / kRecRing, timed_out);
             if (q < total) mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
             __syncwarp();
-            const FrameRec* rec = recs + rk;
+            const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
             const uint32_t fb = ring_base + s * p.slot_bytes + quad * 8;
-            const float* W2s = wtab + rec->cls * 32 + 16;
-            const int n_flush = rec->n_flush, n_nodes = rec->n_nodes;
+            const uint4 head = lds_u32x4(rec);
+            const int n_flush = (int)head.x, n_cells = (int)head.y;
 #pragma unroll 1
             for (int i = 0; i < n_flush; i++) {
-                const FlushCmd fc = rec->flush[i];
-                float4 v = acc.take(fc.slot);
+                const uint4 fc = lds_u32x4(rec + 16 + i * 16);       // slot, kind, dst, weight
+                float4 v = acc.take((int)fc.x);
                 if (active) {
-                    if (fc.kind == 0) {
-                        v.x = v.x / fc.weight; v.y = v.y / fc.weight; v.z = v.z / fc.weight; v.w = v.w / fc.weight;
-                        if (p.out_f32) reinterpret_cast<float4*>(p.staging)[(long long)fc.dst * D4 + ch4] = v;
-                        else reinterpret_cast<uint2*>(p.staging)[(long long)fc.dst * D4 + ch4] = pack_bf16x4(v);
+                    if (fc.y == 0) {
+                        const float wgt = __uint_as_float(fc.w);
+                        v.x = v.x / wgt; v.y = v.y / wgt; v.z = v.z / wgt; v.w = v.w / wgt;
+                        if (p.out_f32) reinterpret_cast<float4*>(p.staging)[(long long)(int)fc.z * D4 + ch4] = v;
+                        else reinterpret_cast<uint2*>(p.staging)[(long long)(int)fc.z * D4 + ch4] = pack_bf16x4(v);
                     } else {
-                        reinterpret_cast<float4*>(p.pieces)[(long long)fc.dst * D4 + ch4] = v;
+                        reinterpret_cast<float4*>(p.pieces)[(long long)(int)fc.z * D4 + ch4] = v;
                     }
                 }
             }
 #pragma unroll 1
-            for (int i = 0; i < n_nodes; i++) {
-                const NodeCmd nc = rec->node[i];
-                const int lv = nc.lv & 3;
-                float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (active) {
-                    const uint32_t a0 = fb + nc.cell * p.row_bytes;
-                    if (lv == 0) {
-                        f = unpack_bf16x4(lds_u64(a0));
-                    } else if (lv == 1) {
-                        const int m = nc.lv >> 4;           // which of the block's four cells exist
-                        f = unpack_bf16x4(lds_u64(a0));
-                        if (m & 2) {
-                            const float4 u = unpack_bf16x4(lds_u64(a0 + p.row_bytes));
-                            f.x += u.x; f.y += u.y; f.z += u.z; f.w += u.w;
-                        }
-                        if (m & 4) {
-                            const float4 u = unpack_bf16x4(lds_u64(a0 + 4 * p.row_bytes));
-                            f.x += u.x; f.y += u.y; f.z += u.z; f.w += u.w;
-                        }
-                        if (m & 8) {
-                            const float4 u = unpack_bf16x4(lds_u64(a0 + 5 * p.row_bytes));
-                            f.x += u.x; f.y += u.y; f.z += u.z; f.w += u.w;
-                        }
-                    } else {
-#pragma unroll 2
-                        for (int c = 0; c < 16; c++) {
-                            const float4 u = unpack_bf16x4(lds_u64(fb + c * p.row_bytes));
-                            const float w = W2s[c];
-                            f.x = fmaf(w, u.x, f.x); f.y = fmaf(w, u.y, f.y);
-                            f.z = fmaf(w, u.z, f.z); f.w = fmaf(w, u.w, f.w);
-                        }
-                    }
-                    f.x *= nc.w; f.y *= nc.w; f.z *= nc.w; f.w *= nc.w;
-                }
-                acc.add(nc.slot, f);
+            for (int i = 0; i < n_cells; i++) {
+                const uint2 cc = lds_u64(rec + 16 + 256 + i * 8);    // slot << 8 | cell, weight
+                const int cell = (int)(cc.x & 0xffu);
+                const float4 x = unpack_bf16x4(lds_u64(fb + cell * p.row_bytes));
+                acc.fma((int)(cc.x >> 8), __uint_as_float(cc.y), x);
             }
             __syncwarp();
             if (lane == 0) {
@@ -572,6 +566,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const unsigned full = 0xffffffffu;
         const int c = lane & 15;
         const int L = p.L;
+        const uint32_t xchg_a = smem_u32(xchg);
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const float tau_s = taus.s[it.b], tau_t = taus.t[it.b];
@@ -587,11 +582,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 __syncwarp();
                 float v[8];
                 {
-                    const float* xch = xchg + xb * p.C * kSumVals;
+                    const uint32_t xch = xchg_a + (xb * p.C * kSumVals + c) * 4;
 #pragma unroll
                     for (int k = 0; k < 8; k++) {
                         float sum = 0.f;
-                        for (int r = 0; r < p.C; r++) sum += xch[r * kSumVals + k * 16 + c];
+                        for (int r = 0; r < p.C; r++) sum += lds_f32(xch + (r * kSumVals + k * 16) * 4);
                         v[k] = valid ? sum : 0.f;       // cells outside the grid: stale ring rows, dropped
                     }
                 }
@@ -660,7 +655,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const bool valid = (it.vmask >> c) & 1u;
-            const float w1 = wtab[it.cls * 32 + c];
+            const float w1 = wtab[it.cls * 32 + c], w2 = wtab[it.cls * 32 + 16 + c];
             if (rank == 0) p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
             int prev_slot = 0;
             uint32_t active_slots = 0;
@@ -721,12 +716,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     tab->cell[slot_fresh] = c;
                 }
                 if (low && linked) atomicAdd(&tab->weight[slot_linked], wint);
-                const uint32_t anchorm = __ballot_sync(full, anchor && low);
-                if (low && anchor && !is_halo) {
-                    const float wn = lv == 1 ? w1 * (float)wint : (float)wint;
-                    const int cm = (int)((cells >> c) & 1u) | (int)((cells >> (c + 1)) & 1u) << 1 |
-                                   (int)((cells >> (c + 4)) & 1u) << 2 | (int)((cells >> (c + 5)) & 1u) << 3;
-                    rec->node[__popc(anchorm & ((1u << c) - 1))] = NodeCmd{c, lv | (cm << 4), node_slot, wn};
+                const int wnode = __shfl_sync(full, wint, (lane & 16) + tile_anchor(c, lv));
+                if (low && valid && !is_halo) {
+                    // weight of this cell in the running sum of its node's chain
+                    const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
+                    rec->cell[__popc(it.vmask & ((1u << c) - 1))] = CellCmd{(cur_slot << 8) | c, wc};
                 }
                 const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
                 __syncwarp();
@@ -753,8 +747,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 }
                 if (lane == 0) {
                     rec->n_flush = n_flush;
-                    rec->n_nodes = is_halo ? 0 : __popc(anchorm);
-                    rec->cls = it.cls;
+                    rec->n_cells = is_halo ? 0 : it.nvalid;
                 }
                 active_slots = is_last ? 0u : active;
                 prev_slot = cur_slot;
@@ -771,8 +764,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             if (low && ((carry_mask >> lane) & 1u)) rec->flush[__popc(carry_mask & ((1u << lane) - 1))] = carry;
             if (lane == 0) {
                 rec->n_flush = __popc(carry_mask);
-                rec->n_nodes = 0;
-                rec->cls = 0;
+                rec->n_cells = 0;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);

@@ -78,9 +78,9 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     f->NA = (f->S + 127) / 128;
     f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
     f->slot_bytes = 16 * f->row_bytes;
-    const size_t fixed = (size_t)f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
+    const size_t fixed = (size_t)2 * f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
                          16 * 32 * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) +
-                         (2 * kMaxRing + 6 * kRecRing) * 8;
+                         (2 * kMaxRing + 6 * kRecRing + 4) * 8;
     int R = (int)((kMaxSmem - fixed) / f->slot_bytes);
     R = std::min(R, kMaxRing);
     if (R < 4) return;
@@ -290,7 +290,7 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
 int fused_resident_clusters(const FusedPlan& f) {
     static int cached[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
     static size_t cached_smem[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
-    const int warps = f.NM + f.NA + 3;
+    const int warps = f.NM + kCombineWarps + f.NA + 3;
     int& slot = cached[f.C][warps];
     if (slot > 0 && cached_smem[f.C][warps] == f.smem) return slot;
     int n = 0;
@@ -345,7 +345,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     const int nclusters = std::min(f.nitems, fused_resident_clusters(f));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nclusters * f.C);
-    cfg.blockDim = dim3((f.NM + f.NA + 3) * 32);
+    cfg.blockDim = dim3((f.NM + kCombineWarps + f.NA + 3) * 32);
     cfg.dynamicSmemBytes = f.smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -442,7 +442,7 @@ int sttm_fused_launch_shape(const sttm_params* p, int* shape) {
     if (shape == nullptr || make_plan(p, &pl) != STTM_OK || !pl.f.ok) return 0;
     const FusedPlan& f = pl.f;
     const int resident = fused_resident_clusters(f);
-    const int v[10] = {f.C, f.S, (f.NM + f.NA + 3) * 32, f.R, (int)f.smem, f.F, f.nitems, resident,
+    const int v[10] = {f.C, f.S, (f.NM + kCombineWarps + f.NA + 3) * 32, f.R, (int)f.smem, f.F, f.nitems, resident,
                        std::min(f.nitems, resident), f.NM};
     std::memcpy(shape, v, sizeof(v));
     return 1;

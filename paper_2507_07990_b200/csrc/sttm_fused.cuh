@@ -13,8 +13,8 @@
 //   producer warp   issues the bulk copies of the next frames as ring slots come free;
 //   Gram warps      form the tile's Gram matrix G = X_t X_t^T and cross matrix
 //                   C = X_t X_{t-1}^T over the CTA's channels on the tensor cores (X = the 16
-//                   cells of the tile; products of bf16 inputs are exact, sums are fp32),
-//                   add the warps' parts, contract them to the 128 numbers the decisions
+//                   cells of the tile; products of bf16 inputs are exact, sums are fp32);
+//   combine warps   add the Gram warps' parts, contract them to the 128 numbers the decisions
 //                   need (every cosine of Sections 3.2 and 3.3 is a short linear combination
 //                   of entries of G and C because parents are averages of cells) and send
 //                   them to every CTA of the cluster (stores that signal a remote mbarrier);
@@ -22,9 +22,11 @@
 //                   Section 3.2 (cover map) and Section 3.3 (links), the same in every CTA;
 //   chain warp      follows the chains through time: which running sum each kept node
 //                   joins, which chains ended; leaves a command record per frame;
-//   sum warps       execute the records on the frame that is still in the ring: a thread
-//                   owns four channels and keeps the running sums of up to 16 chains in
-//                   registers.
+//   sum warps       execute the records on the frame that is still in the ring.  The record
+//                   holds a 16x16 matrix W (chain slot x cell: the weight of the cell in the
+//                   running sum of that chain), so the update of all running sums is one
+//                   small matrix product  sums[16 x channels] += W X  on the tensor cores,
+//                   with the sums living in the accumulator registers of the warps.
 // Finished chains go to a staging row indexed by the root's cell id (their final row is
 // only known after the global ordering); chains cut by the end of an item go to an fp32
 // piece buffer and are put together by the gather kernel.
@@ -43,23 +45,24 @@ constexpr int kSumVals = 128;           // 8 numbers per cell, see combine_sums(
 constexpr int kPieceSlots = 32;         // per item: 16 keyed by a cell of the frame before the item, 16 by chain slot
 constexpr int kMaxRing = 12;
 constexpr int kMaxGramWarps = 4;
+constexpr int kCombineWarps = 4;
 constexpr int kMaxSumWarps = 8;         // 128 channels each: at most 1024 channels per CTA
-constexpr int kFusedMaxThreads = (kMaxGramWarps + kMaxSumWarps + 3) * 32;
+constexpr int kFusedMaxThreads = (kMaxGramWarps + kCombineWarps + kMaxSumWarps + 3) * 32;
 constexpr int kSpinLimit = 1 << 12;     // tries per wait; after the first wait that runs out, later waits are skipped
 constexpr uint32_t kWaitHintNs = 1000000u;   // a try may sleep this long before it reports "not yet"
 
 enum : int { kStatusWaitTimeout = 1 << 6 };
 
 struct FlushCmd { int slot, kind, dst; float weight; };     // kind 0: finished row, 1: piece
-struct CellCmd { int slot_cell; float w; };                 // slot << 8 | cell; weight of the cell in its node
 // Commands of one frame for the sum warps: first write out and clear the listed chain sums
 // (chains that got no member in this frame; at the first frame of an item: everything the
-// previous item left), then add every cell of the frame, times its weight in its kept node,
-// to the running sum of the node's chain.
+// previous item left), then add W X to the running sums, W[slot][cell] (bf16; the weights
+// are small integers times powers of two, hence exact) = weight of the cell in its kept node
+// if that node belongs to the chain in `slot`, else 0.
 struct FrameRec {
-    int n_flush, n_cells, pad0, pad1;
+    int n_flush, pad0, pad1, pad2;
     FlushCmd flush[16];
-    CellCmd cell[16];
+    uint16_t wmat[256];
 };
 
 struct FusedParams {
@@ -163,6 +166,11 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
 // D (16x8, fp32) += A (16x16 bf16, row) * B (16x8 bf16, col)
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -214,55 +222,9 @@ __device__ __forceinline__ int kth_set_bit16(uint32_t m, int k) {
     return pos;
 }
 
-// running sums of the chains: 16 slots x 4 channels, in registers; the slot index is
-// uniform over the warp, so the switch does not diverge (the empty asm statements keep the
-// compiler from turning the cases into selects over all 64 registers)
-struct ChainAcc {
-    float4 a[16];
-    __device__ __forceinline__ void clear() {
-#pragma unroll
-        for (int i = 0; i < 16; i++) a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#define STTM_ACC_BODY(i)              \
-    asm volatile("");                 \
-    a[i].x = fmaf(w, f.x, a[i].x);    \
-    a[i].y = fmaf(w, f.y, a[i].y);    \
-    a[i].z = fmaf(w, f.z, a[i].z);    \
-    a[i].w = fmaf(w, f.w, a[i].w);    \
-    break;
-#define STTM_ACC_CASE(i) case i: STTM_ACC_BODY(i)
-    __device__ __forceinline__ void fma(int slot, float w, float4 f) {
-        switch (slot) {
-            STTM_ACC_CASE(0) STTM_ACC_CASE(1) STTM_ACC_CASE(2) STTM_ACC_CASE(3) STTM_ACC_CASE(4) STTM_ACC_CASE(5)
-            STTM_ACC_CASE(6) STTM_ACC_CASE(7) STTM_ACC_CASE(8) STTM_ACC_CASE(9) STTM_ACC_CASE(10) STTM_ACC_CASE(11)
-            STTM_ACC_CASE(12) STTM_ACC_CASE(13) STTM_ACC_CASE(14) default: STTM_ACC_BODY(15)
-        }
-    }
-#undef STTM_ACC_CASE
-#undef STTM_ACC_BODY
-#define STTM_TAKE_BODY(i) asm volatile(""); v = a[i]; a[i] = make_float4(0.f, 0.f, 0.f, 0.f); break;
-#define STTM_TAKE_CASE(i) case i: STTM_TAKE_BODY(i)
-    __device__ __forceinline__ float4 take(int slot) {
-        float4 v;
-        switch (slot) {
-            STTM_TAKE_CASE(0) STTM_TAKE_CASE(1) STTM_TAKE_CASE(2) STTM_TAKE_CASE(3) STTM_TAKE_CASE(4)
-            STTM_TAKE_CASE(5) STTM_TAKE_CASE(6) STTM_TAKE_CASE(7) STTM_TAKE_CASE(8) STTM_TAKE_CASE(9)
-            STTM_TAKE_CASE(10) STTM_TAKE_CASE(11) STTM_TAKE_CASE(12) STTM_TAKE_CASE(13) STTM_TAKE_CASE(14)
-            default: STTM_TAKE_BODY(15)
-        }
-        return v;
-    }
-#undef STTM_TAKE_CASE
-#undef STTM_TAKE_BODY
-};
-
-__device__ __forceinline__ float4 unpack_bf16x4(uint2 w) {
-    return make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u), __uint_as_float(w.y << 16),
-                       __uint_as_float(w.y & 0xffff0000u));
-}
-__device__ __forceinline__ uint2 pack_bf16x4(float4 v) {
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-    return make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+__device__ __forceinline__ uint32_t pack_bf16x2(float x, float y) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+    return *reinterpret_cast<const uint32_t*>(&h);
 }
 
 // sum over lanes that share (lane & 16): every lane of a half gets its half's total
@@ -375,7 +337,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* ring = smem;
     size_t off = (size_t)p.R * p.slot_bytes;
-    float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)p.NM * kGramVals * 4;
+    float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)2 * p.NM * kGramVals * 4;   // two frames
     float* redsum = reinterpret_cast<float*>(smem + off);    off += kGramVals * 4;
     float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * p.C * kSumVals * 4;
     float* wtab = reinterpret_cast<float*>(smem + off);      off += 16 * 32 * 4;      // [shape][W1 x16, W2 x16]
@@ -388,11 +350,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     const uint32_t xfull_bar = bar0 + 16 * kMaxRing, xempty_bar = xfull_bar + 8 * kRecRing;
     const uint32_t hfull_bar = xempty_bar + 8 * kRecRing, hempty_bar = hfull_bar + 8 * kRecRing;
     const uint32_t rfull_bar = hempty_bar + 8 * kRecRing, rempty_bar = rfull_bar + 8 * kRecRing;
+    const uint32_t gfull_bar = rempty_bar + 8 * kRecRing, gempty_bar = gfull_bar + 16;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank(), cid = cluster_id(), ncl = cluster_count();
     const uint32_t ring_base = smem_u32(ring);
-    const int w_sim = p.NM + p.NA, w_chain = w_sim + 1, w_prod = w_sim + 2;
+    const int w_comb = p.NM, w_sum = p.NM + kCombineWarps, w_sim = w_sum + p.NA, w_chain = w_sim + 1, w_prod = w_sim + 2;
 
     // set-up: barriers, a ring without NaN patterns, the pooling weights of all 16 tile shapes
     if (tid == 0) {
@@ -407,6 +370,10 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             mbar_init(hempty_bar + 8 * s, 1);
             mbar_init(rfull_bar + 8 * s, 1);
             mbar_init(rempty_bar + 8 * s, p.NA);
+        }
+        for (int s = 0; s < 2; s++) {
+            mbar_init(gfull_bar + 8 * s, p.NM);
+            mbar_init(gempty_bar + 8 * s, kCombineWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -434,14 +401,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
 
     if (warp < p.NM) {
         // ------------------------------------ Gram warps ------------------------------------
-        const int nthr = p.NM * 32;
         const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
         const uint32_t loff = lrow * p.row_bytes + lk * 2;
         const int ksteps = p.S >> 4;
-        const uint32_t red_a = smem_u32(red), redsum_a = smem_u32(redsum);
+        const int k0 = ksteps * warp / p.NM, k1 = ksteps * (warp + 1) / p.NM;     // this warp's channel steps
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
-            const uint32_t W1s = smem_u32(wtab + it.cls * 32), W2s = W1s + 64;
             for (int j = 0; j < it.n; j++, q++) {
                 const int s = q % p.R;
                 mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
@@ -452,29 +417,37 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
                 const uint32_t cur = ring_base + s * p.slot_bytes + loff;
                 const uint32_t prv = ring_base + ((q + p.R - 1) % p.R) * p.slot_bytes + loff;
-                // two independent accumulator sets keep more tensor-core operations in flight
-                for (int ks = warp; ks < ksteps; ks += 2 * p.NM) {
-                    uint32_t a[4], b[4], a2[4], b2[4];
-                    const bool second = ks + p.NM < ksteps;
-                    ldmatrix_x4(cur + ks * 32, a);
-                    ldmatrix_x4(prv + ks * 32, b);
-                    if (second) {
-                        ldmatrix_x4(cur + (ks + p.NM) * 32, a2);
-                        ldmatrix_x4(prv + (ks + p.NM) * 32, b2);
+                // two accumulator sets, fragments of the next step loaded before the products of this one
+                uint32_t a[4], b[4], a2[4], b2[4];
+                if (k0 < k1) {
+                    ldmatrix_x4(cur + k0 * 32, a);
+                    ldmatrix_x4(prv + k0 * 32, b);
+                }
+                for (int ks = k0; ks < k1; ks += 2) {
+                    if (ks + 1 < k1) {
+                        ldmatrix_x4(cur + (ks + 1) * 32, a2);
+                        ldmatrix_x4(prv + (ks + 1) * 32, b2);
                     }
                     mma_bf16(g0, a, a[0], a[2]);
                     mma_bf16(g1, a, a[1], a[3]);
                     mma_bf16(c0, a, b[0], b[2]);
                     mma_bf16(c1, a, b[1], b[3]);
-                    if (second) {
+                    if (ks + 2 < k1) {
+                        ldmatrix_x4(cur + (ks + 2) * 32, a);
+                        ldmatrix_x4(prv + (ks + 2) * 32, b);
+                    }
+                    if (ks + 1 < k1) {
                         mma_bf16(h0, a2, a2[0], a2[2]);
                         mma_bf16(h1, a2, a2[1], a2[3]);
                         mma_bf16(e0, a2, b2[0], b2[2]);
                         mma_bf16(e1, a2, b2[1], b2[3]);
                     }
                 }
+                const int gb = q & 1;
+                if (q >= 2) mbar_wait(gempty_bar + 8 * gb, q / 2 - 1, timed_out);
+                __syncwarp();
                 {
-                    float* r = red + warp * kGramVals;
+                    float* r = red + (gb * p.NM + warp) * kGramVals;
                     const int gr = lane >> 2, gc = (lane & 3) * 2;
                     *reinterpret_cast<float2*>(r + gr * 16 + gc) = make_float2(g0[0] + h0[0], g0[1] + h0[1]);
                     *reinterpret_cast<float2*>(r + (gr + 8) * 16 + gc) = make_float2(g0[2] + h0[2], g0[3] + h0[3]);
@@ -486,39 +459,67 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + 8 + gc) =
                         make_float2(c1[2] + e1[2], c1[3] + e1[3]);
                 }
-                named_sync(1, nthr);
-                // this warp is done with the previous frame's slot (the current one stays for the next frame)
-                if (lane == 0 && q >= 1) mbar_arrive(empty_bar + 8 * ((q - 1) % p.R));
-                // add the warps' parts, each thread a share of the 512 entries
-                for (int i = tid * 4; i < kGramVals; i += nthr * 4) {
-                    float4 sum = lds_f32x4(red_a + i * 4);
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(gfull_bar + 8 * gb);
+                    // done with the previous frame's slot (the current one stays for the next frame)
+                    if (q >= 1) mbar_arrive(empty_bar + 8 * ((q - 1) % p.R));
+                }
+            }
+        }
+    } else if (warp < w_sum) {
+        // ----------------------------------- combine warps -----------------------------------
+        const int ctid = tid - w_comb * 32, nthr = kCombineWarps * 32;
+        const uint32_t red_a = smem_u32(red), redsum_a = smem_u32(redsum);
+        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+            if (skip) continue;
+            const uint32_t W1s = smem_u32(wtab + it.cls * 32), W2s = W1s + 64;
+            for (int j = 0; j < it.n; j++, q++) {
+                const int gb = q & 1;
+                mbar_wait(gfull_bar + 8 * gb, q / 2, timed_out);
+                __syncwarp();
+                // add the Gram warps' parts, each thread a share of the 512 entries
+                for (int i = ctid * 4; i < kGramVals; i += nthr * 4) {
+                    float4 sum = lds_f32x4(red_a + (gb * p.NM * kGramVals + i) * 4);
                     for (int w = 1; w < p.NM; w++) {
-                        const float4 v = lds_f32x4(red_a + (w * kGramVals + i) * 4);
+                        const float4 v = lds_f32x4(red_a + ((gb * p.NM + w) * kGramVals + i) * 4);
                         sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
                     }
                     *reinterpret_cast<float4*>(redsum + i) = sum;
                 }
-                named_sync(2, nthr);
+                named_sync(1, nthr);
+                if (lane == 0) mbar_arrive(gempty_bar + 8 * gb);
                 // contract to 8 numbers per cell and send this CTA's share to every CTA of the cluster
                 const int xb = q % kRecRing;
                 if (q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
-                for (int i = tid; i < kSumVals; i += nthr) {
+                for (int i = ctid; i < kSumVals; i += nthr) {
                     const float sum = combine_sums(redsum_a, i & 15, i >> 4, it.vmask, W1s, W2s);
                     const uint32_t a = smem_u32(xchg + (xb * p.C + rank) * kSumVals + i);
                     for (int r = 0; r < p.C; r++)
                         st_async_f32(map_to_rank(a, r), sum, map_to_rank(xfull_bar + 8 * xb, r));
                 }
+                named_sync(2, nthr);       // the sums are read before the next frame overwrites them
             }
         }
     } else if (warp < w_sim) {
         // ------------------------------------ sum warps ------------------------------------
-        ChainAcc acc;
-        acc.clear();
-        const int quad_raw = tid - p.NM * 32;                // channels 4*quad .. 4*quad+3 of this CTA's slice
-        const bool active = 4 * quad_raw < p.S;
-        const int quad = active ? quad_raw : 0;              // idle lanes of the last warp shadow thread 0, write nothing
-        const long long ch4 = ((long long)rank * p.S >> 2) + quad, D4 = p.D >> 2;
+        // Warp a owns channels [128 a, 128 a + 128) of the CTA's slice: 16 tiles of 8 channels.
+        // sums[nt][0..3] is the accumulator fragment of tile nt: chain slots g and g + 8
+        // (g = lane / 4), channels 2 t and 2 t + 1 of the tile (t = lane % 4).
+        float sums[16][4];
+#pragma unroll
+        for (int nt = 0; nt < 16; nt++)
+#pragma unroll
+            for (int k = 0; k < 4; k++) sums[nt][k] = 0.f;
+        const int ch0 = (warp - w_sum) * 128;
+        const int g = lane >> 2, t4 = lane & 3;
         const uint32_t recs_a = smem_u32(recs);
+        // B fragments (cells x 16 channels) by transposing loads: lane l addresses row (cell) l%8 + 8*((l>>3)&1)
+        // of the 8-channel column block l>>4
+        const uint32_t xoff = ((lane & 7) + ((lane >> 3) & 1) * 8) * p.row_bytes + (ch0 + (lane >> 4) * 8) * 2;
+        // A fragment (16 slots x 16 cells) straight from the record
+        const uint32_t woff = 16 + 256 + ((lane & 7) + ((lane >> 3) & 1) * 8) * 32 + (lane >> 4) * 16;
+        const long long chan = (long long)rank * p.S + ch0 + 2 * t4;
         int total = 0;
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
             if (!skip) total += it.n;
@@ -529,30 +530,41 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             if (q < total) mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
             __syncwarp();
             const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
-            const uint32_t fb = ring_base + s * p.slot_bytes + quad * 8;
-            const uint4 head = lds_u32x4(rec);
-            const int n_flush = (int)head.x, n_cells = (int)head.y;
+            const int n_flush = (int)lds_u32x4(rec).x;
 #pragma unroll 1
             for (int i = 0; i < n_flush; i++) {
                 const uint4 fc = lds_u32x4(rec + 16 + i * 16);       // slot, kind, dst, weight
-                float4 v = acc.take((int)fc.x);
-                if (active) {
-                    if (fc.y == 0) {
-                        const float wgt = __uint_as_float(fc.w);
-                        v.x = v.x / wgt; v.y = v.y / wgt; v.z = v.z / wgt; v.w = v.w / wgt;
-                        if (p.out_f32) reinterpret_cast<float4*>(p.staging)[(long long)(int)fc.z * D4 + ch4] = v;
-                        else reinterpret_cast<uint2*>(p.staging)[(long long)(int)fc.z * D4 + ch4] = pack_bf16x4(v);
-                    } else {
-                        reinterpret_cast<float4*>(p.pieces)[(long long)(int)fc.z * D4 + ch4] = v;
+                const int slot = (int)fc.x;
+                if (g == (slot & 7)) {
+                    const bool hi = slot >= 8;
+                    const float wgt = fc.y == 0 ? __uint_as_float(fc.w) : 1.f;
+                    const long long row = (long long)(int)fc.z * p.D + chan;
+#pragma unroll
+                    for (int nt = 0; nt < 16; nt++) {
+                        const float x = (hi ? sums[nt][2] : sums[nt][0]) / wgt, y = (hi ? sums[nt][3] : sums[nt][1]) / wgt;
+                        if (hi) { sums[nt][2] = 0.f; sums[nt][3] = 0.f; } else { sums[nt][0] = 0.f; sums[nt][1] = 0.f; }
+                        if (ch0 + nt * 8 < p.S) {
+                            if (fc.y != 0) *reinterpret_cast<float2*>(p.pieces + row + nt * 8) = make_float2(x, y);
+                            else if (p.out_f32) *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.staging) + row + nt * 8) = make_float2(x, y);
+                            else *reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(p.staging) + row + nt * 8) = pack_bf16x2(x, y);
+                        }
                     }
                 }
             }
-#pragma unroll 1
-            for (int i = 0; i < n_cells; i++) {
-                const uint2 cc = lds_u64(rec + 16 + 256 + i * 8);    // slot << 8 | cell, weight
-                const int cell = (int)(cc.x & 0xffu);
-                const float4 x = unpack_bf16x4(lds_u64(fb + cell * p.row_bytes));
-                acc.fma((int)(cc.x >> 8), __uint_as_float(cc.y), x);
+            __syncwarp();
+            if (q < total) {
+                uint32_t wa[4];
+                ldmatrix_x4(rec + woff, wa);
+                const uint32_t xb = ring_base + s * p.slot_bytes + xoff;
+#pragma unroll
+                for (int pr = 0; pr < 8; pr++) {
+                    if (ch0 + pr * 16 < p.S) {
+                        uint32_t xb4[4];
+                        ldmatrix_x4_trans(xb + pr * 32, xb4);
+                        mma_bf16(sums[2 * pr], wa, xb4[0], xb4[1]);
+                        mma_bf16(sums[2 * pr + 1], wa, xb4[2], xb4[3]);
+                    }
+                }
             }
             __syncwarp();
             if (lane == 0) {
@@ -716,11 +728,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     tab->cell[slot_fresh] = c;
                 }
                 if (low && linked) atomicAdd(&tab->weight[slot_linked], wint);
+                // the frame's weight matrix: row = chain slot, column = cell
+                reinterpret_cast<uint4*>(rec->wmat)[lane] = make_uint4(0u, 0u, 0u, 0u);
                 const int wnode = __shfl_sync(full, wint, (lane & 16) + tile_anchor(c, lv));
+                __syncwarp();
                 if (low && valid && !is_halo) {
-                    // weight of this cell in the running sum of its node's chain
                     const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
-                    rec->cell[__popc(it.vmask & ((1u << c) - 1))] = CellCmd{(cur_slot << 8) | c, wc};
+                    rec->wmat[cur_slot * 16 + c] = __bfloat16_as_ushort(__float2bfloat16_rn(wc));
                 }
                 const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
                 __syncwarp();
@@ -747,7 +761,6 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 }
                 if (lane == 0) {
                     rec->n_flush = n_flush;
-                    rec->n_cells = is_halo ? 0 : it.nvalid;
                 }
                 active_slots = is_last ? 0u : active;
                 prev_slot = cur_slot;
@@ -764,7 +777,6 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             if (low && ((carry_mask >> lane) & 1u)) rec->flush[__popc(carry_mask & ((1u << lane) - 1))] = carry;
             if (lane == 0) {
                 rec->n_flush = __popc(carry_mask);
-                rec->n_cells = 0;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);

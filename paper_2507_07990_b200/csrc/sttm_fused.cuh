@@ -48,8 +48,8 @@ constexpr int kMaxGramWarps = 4;
 constexpr int kCombineWarps = 4;
 constexpr int kMaxSumWarps = 8;         // 128 channels each: at most 1024 channels per CTA
 constexpr int kFusedMaxThreads = (kMaxGramWarps + kCombineWarps + kMaxSumWarps + 3) * 32;
-constexpr int kSpinLimit = 1 << 12;     // tries per wait; after the first wait that runs out, later waits are skipped
-constexpr uint32_t kWaitHintNs = 1000000u;   // a try may sleep this long before it reports "not yet"
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after two seconds
+constexpr uint32_t kWaitHintNs = 100000u;    // one try may sleep this long before it reports "not yet"
 
 enum : int { kStatusWaitTimeout = 1 << 6 };
 
@@ -113,15 +113,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait for the `use`-th completion (0-based) of an mbarrier.  Once a wait has run
-// out the thread stops waiting altogether, so the kernel still ends; the host sees
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for the `use`-th completion (0-based) of an mbarrier: false when it has not
+// come within kWaitLimitNs (or an earlier wait of this thread ran out).  The caller then
+// leaves its loops without touching the data it waited for; the warps that depend on it
+// run out in turn, every CTA still reaches the end of the kernel, and the host sees
 // kStatusWaitTimeout in the status word.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, int use, bool& timed_out) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, int use, bool& timed_out) {
+    if (timed_out) return false;
     const uint32_t parity = (uint32_t)(use & 1);
-    int spins = 0;
-    while (!timed_out && !mbar_try_wait(bar, parity)) {
-        if (++spins > kSpinLimit) timed_out = true;
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    int tries = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++tries & 63) == 0 && global_timer_ns() - t0 > kWaitLimitNs) {
+            timed_out = true;
+            return false;
+        }
     }
+    return true;
 }
 // global -> this CTA's shared memory, completion counted in bytes on an mbarrier
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -160,6 +174,19 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
 }
 __device__ __forceinline__ void named_sync(int id, int count) {
     asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+// named barrier that also returns the OR of a flag over its `count` threads
+__device__ __forceinline__ bool named_sync_or(int id, int count, bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "barrier.red.or.pred q, %2, %3, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)flag), "r"(id), "r"(count)
+        : "memory");
+    return r != 0;
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -405,11 +432,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const uint32_t loff = lrow * p.row_bytes + lk * 2;
         const int ksteps = p.S >> 4;
         const int k0 = ksteps * warp / p.NM, k1 = ksteps * (warp + 1) / p.NM;     // this warp's channel steps
-        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+        for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             for (int j = 0; j < it.n; j++, q++) {
                 const int s = q % p.R;
-                mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
+                if (!mbar_wait(full_bar + 8 * s, q / p.R, timed_out)) break;
                 __syncwarp();
                 float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
                 float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -444,7 +471,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     }
                 }
                 const int gb = q & 1;
-                if (q >= 2) mbar_wait(gempty_bar + 8 * gb, q / 2 - 1, timed_out);
+                if (q >= 2 && !mbar_wait(gempty_bar + 8 * gb, q / 2 - 1, timed_out)) break;
                 __syncwarp();
                 {
                     float* r = red + (gb * p.NM + warp) * kGramVals;
@@ -471,13 +498,14 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // ----------------------------------- combine warps -----------------------------------
         const int ctid = tid - w_comb * 32, nthr = kCombineWarps * 32;
         const uint32_t red_a = smem_u32(red), redsum_a = smem_u32(redsum);
-        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+        for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const uint32_t W1s = smem_u32(wtab + it.cls * 32), W2s = W1s + 64;
             for (int j = 0; j < it.n; j++, q++) {
                 const int gb = q & 1;
-                mbar_wait(gfull_bar + 8 * gb, q / 2, timed_out);
-                __syncwarp();
+                // the first combine warp waits; the named barriers hand the outcome to the others
+                if (warp == w_comb) mbar_wait(gfull_bar + 8 * gb, q / 2, timed_out);
+                if (named_sync_or(3, nthr, timed_out)) { timed_out = true; break; }
                 // add the Gram warps' parts, each thread a share of the 512 entries
                 for (int i = ctid * 4; i < kGramVals; i += nthr * 4) {
                     float4 sum = lds_f32x4(red_a + (gb * p.NM * kGramVals + i) * 4);
@@ -491,14 +519,14 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (lane == 0) mbar_arrive(gempty_bar + 8 * gb);
                 // contract to 8 numbers per cell and send this CTA's share to every CTA of the cluster
                 const int xb = q % kRecRing;
-                if (q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
+                if (warp == w_comb && q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
+                if (named_sync_or(2, nthr, timed_out)) { timed_out = true; break; }
                 for (int i = ctid; i < kSumVals; i += nthr) {
                     const float sum = combine_sums(redsum_a, i & 15, i >> 4, it.vmask, W1s, W2s);
-                    const uint32_t a = smem_u32(xchg + (xb * p.C + rank) * kSumVals + i);
+                    const uint32_t a = smem_u32(xchg + (xb * p.C + rank) * kSumVals + (i & 15) * 8 + (i >> 4));   // [cell][k]
                     for (int r = 0; r < p.C; r++)
                         st_async_f32(map_to_rank(a, r), sum, map_to_rank(xfull_bar + 8 * xb, r));
                 }
-                named_sync(2, nthr);       // the sums are read before the next frame overwrites them
             }
         }
     } else if (warp < w_sim) {
@@ -526,8 +554,8 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // one record per frame, and a last one that only writes out what the last item left
         for (; q <= total; q++) {
             const int rk = q % kRecRing, s = q % p.R;
-            mbar_wait(rfull_bar + 8 * rk, q / kRecRing, timed_out);
-            if (q < total) mbar_wait(full_bar + 8 * s, q / p.R, timed_out);
+            if (!mbar_wait(rfull_bar + 8 * rk, q / kRecRing, timed_out)) break;
+            if (q < total && !mbar_wait(full_bar + 8 * s, q / p.R, timed_out)) break;
             __syncwarp();
             const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
             const int n_flush = (int)lds_u32x4(rec).x;
@@ -537,11 +565,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const int slot = (int)fc.x;
                 if (g == (slot & 7)) {
                     const bool hi = slot >= 8;
-                    const float wgt = fc.y == 0 ? __uint_as_float(fc.w) : 1.f;
+                    const float inv = fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
                     const long long row = (long long)(int)fc.z * p.D + chan;
 #pragma unroll
                     for (int nt = 0; nt < 16; nt++) {
-                        const float x = (hi ? sums[nt][2] : sums[nt][0]) / wgt, y = (hi ? sums[nt][3] : sums[nt][1]) / wgt;
+                        const float x = (hi ? sums[nt][2] : sums[nt][0]) * inv, y = (hi ? sums[nt][3] : sums[nt][1]) * inv;
                         if (hi) { sums[nt][2] = 0.f; sums[nt][3] = 0.f; } else { sums[nt][0] = 0.f; sums[nt][1] = 0.f; }
                         if (ch0 + nt * 8 < p.S) {
                             if (fc.y != 0) *reinterpret_cast<float2*>(p.pieces + row + nt * 8) = make_float2(x, y);
@@ -579,7 +607,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const int c = lane & 15;
         const int L = p.L;
         const uint32_t xchg_a = smem_u32(xchg);
-        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+        for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const float tau_s = taus.s[it.b], tau_t = taus.t[it.b];
             const float w1 = wtab[it.cls * 32 + c], w2 = wtab[it.cls * 32 + 16 + c];
@@ -590,17 +618,20 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             for (int j = 0; j < it.n; j++, q++) {
                 const int xb = q % kRecRing;
                 if (lane == 0) mbar_expect_tx(xfull_bar + 8 * xb, (uint32_t)(p.C * kSumVals * 4));
-                mbar_wait(xfull_bar + 8 * xb, q / kRecRing, timed_out);
+                if (!mbar_wait(xfull_bar + 8 * xb, q / kRecRing, timed_out)) break;
                 __syncwarp();
                 float v[8];
                 {
-                    const uint32_t xch = xchg_a + (xb * p.C * kSumVals + c) * 4;
-#pragma unroll
-                    for (int k = 0; k < 8; k++) {
-                        float sum = 0.f;
-                        for (int r = 0; r < p.C; r++) sum += lds_f32(xch + (r * kSumVals + k * 16) * 4);
-                        v[k] = valid ? sum : 0.f;       // cells outside the grid: stale ring rows, dropped
+                    const uint32_t xch = xchg_a + (xb * p.C * kSumVals + c * 8) * 4;
+                    float4 lo = lds_f32x4(xch), hi = lds_f32x4(xch + 16);
+                    for (int r = 1; r < p.C; r++) {          // the CTAs' shares, in rank order
+                        const float4 l2 = lds_f32x4(xch + r * kSumVals * 4), h2 = lds_f32x4(xch + r * kSumVals * 4 + 16);
+                        lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
+                        hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
                     }
+                    // cells outside the grid: stale ring rows, dropped
+                    v[0] = valid ? lo.x : 0.f; v[1] = valid ? lo.y : 0.f; v[2] = valid ? lo.z : 0.f; v[3] = valid ? lo.w : 0.f;
+                    v[4] = valid ? hi.x : 0.f; v[5] = valid ? hi.y : 0.f; v[6] = valid ? hi.z : 0.f; v[7] = valid ? hi.w : 0.f;
                 }
                 __syncwarp();
                 if (lane < p.C) mbar_arrive_remote(map_to_rank(xempty_bar + 8 * xb, lane));
@@ -649,7 +680,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 prev_nk = nk;
 
                 // hand the cover level and the link of every cell to the chain warp
-                if (q >= kRecRing) mbar_wait(hempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
+                if (q >= kRecRing && !mbar_wait(hempty_bar + 8 * xb, q / kRecRing - 1, timed_out)) break;
                 __syncwarp();
                 if (lane < 16) hand[xb * 16 + c] = lv | ((link_local + 1) << 8);
                 __syncwarp();
@@ -664,7 +695,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // what the previous item left running when it ended: written out by the next record
         FlushCmd carry = FlushCmd{0, 0, 0, 0.f};     // lane s < 16: slot s
         uint32_t carry_mask = 0;
-        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+        for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const bool valid = (it.vmask >> c) & 1u;
             const float w1 = wtab[it.cls * 32 + c], w2 = wtab[it.cls * 32 + 16 + c];
@@ -673,13 +704,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             uint32_t active_slots = 0;
             for (int j = 0; j < it.n; j++, q++) {
                 const int hb = q % kRecRing;
-                mbar_wait(hfull_bar + 8 * hb, q / kRecRing, timed_out);
+                if (!mbar_wait(hfull_bar + 8 * hb, q / kRecRing, timed_out)) break;
                 __syncwarp();
                 const int packed = hand[hb * 16 + c];
                 __syncwarp();
                 if (lane == 0) mbar_arrive(hempty_bar + 8 * hb);
                 const int lv = packed & 3, link_local = (packed >> 8) - 1;
-                if (q >= kRecRing) mbar_wait(rempty_bar + 8 * hb, q / kRecRing - 1, timed_out);
+                if (q >= kRecRing && !mbar_wait(rempty_bar + 8 * hb, q / kRecRing - 1, timed_out)) break;
                 __syncwarp();
                 FrameRec* rec = recs + hb;
                 const int t = it.tstart + j;
@@ -768,10 +799,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
             }
         }
-        {
+        if (q < kRecRing || mbar_wait(rempty_bar + 8 * (q % kRecRing), q / kRecRing - 1, timed_out)) {
             // last record: only the carry of the last item
             const int hb = q % kRecRing;
-            if (q >= kRecRing) mbar_wait(rempty_bar + 8 * hb, q / kRecRing - 1, timed_out);
             __syncwarp();
             FrameRec* rec = recs + hb;
             if (low && ((carry_mask >> lane) & 1u)) rec->flush[__popc(carry_mask & ((1u << lane) - 1))] = carry;
@@ -783,12 +813,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         }
     } else if (warp == w_prod) {
         // ----------------------------------- producer warp -----------------------------------
-        for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++) {
+        for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             for (int j = 0; j < it.n; j++, q++) {
                 const int s = q % p.R;
                 const uint32_t bar = full_bar + 8 * s;
-                if (q >= p.R) mbar_wait(empty_bar + 8 * s, q / p.R - 1, timed_out);
+                if (q >= p.R && !mbar_wait(empty_bar + 8 * s, q / p.R - 1, timed_out)) break;
                 __syncwarp();
                 if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
                 __syncwarp();
@@ -799,6 +829,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                              (uint32_t)(p.S * 2), bar);
                 }
             }
+        }
+        // the CTA must not end with copies in flight: the last R frames issued have landed?
+        // (immediate in a normal run; after a wait ran out, each of these waits is bounded again)
+        for (int qq = max(0, q - p.R); qq < q; qq++) {
+            bool late = false;
+            mbar_wait(full_bar + 8 * (qq % p.R), qq / p.R, late);
+            timed_out |= late;
         }
     }
     // nobody leaves while a CTA of the cluster may still store into it or signal its barriers

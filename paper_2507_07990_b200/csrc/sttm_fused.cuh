@@ -267,9 +267,14 @@ __device__ __forceinline__ float quad_sum(float v) {
     return v;
 }
 // cos(a, b) > tau from a.b, |a|^2, |b|^2 without a division; a zero vector has cosine 0
+__device__ __forceinline__ float sqrt_fast(float x) {
+    float r;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));      // a few ulp: far inside the decision margins
+    return r;
+}
 __device__ __forceinline__ bool cos_above(float dot, float na, float nb, float tau) {
     if (na == 0.f || nb == 0.f) return 0.f > tau;
-    return dot > tau * (sqrtf(na) * sqrtf(nb));
+    return dot > tau * (sqrt_fast(na) * sqrt_fast(nb));
 }
 
 struct ItemGeo {
@@ -444,31 +449,33 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
                 const uint32_t cur = ring_base + s * p.slot_bytes + loff;
                 const uint32_t prv = ring_base + ((q + p.R - 1) % p.R) * p.slot_bytes + loff;
-                // two accumulator sets, fragments of the next step loaded before the products of this one
+                // two accumulator sets; the fragments of a step are loaded before the products of the
+                // step before it are issued (the index is clamped at the end: a repeated load, no branch)
                 uint32_t a[4], b[4], a2[4], b2[4];
-                if (k0 < k1) {
-                    ldmatrix_x4(cur + k0 * 32, a);
-                    ldmatrix_x4(prv + k0 * 32, b);
-                }
-                for (int ks = k0; ks < k1; ks += 2) {
-                    if (ks + 1 < k1) {
-                        ldmatrix_x4(cur + (ks + 1) * 32, a2);
-                        ldmatrix_x4(prv + (ks + 1) * 32, b2);
-                    }
+                const int kl = k1 - 1;
+                ldmatrix_x4(cur + k0 * 32, a);
+                ldmatrix_x4(prv + k0 * 32, b);
+                int ks = k0;
+                for (; ks + 1 < k1; ks += 2) {
+                    ldmatrix_x4(cur + (ks + 1) * 32, a2);
+                    ldmatrix_x4(prv + (ks + 1) * 32, b2);
                     mma_bf16(g0, a, a[0], a[2]);
                     mma_bf16(g1, a, a[1], a[3]);
                     mma_bf16(c0, a, b[0], b[2]);
                     mma_bf16(c1, a, b[1], b[3]);
-                    if (ks + 2 < k1) {
-                        ldmatrix_x4(cur + (ks + 2) * 32, a);
-                        ldmatrix_x4(prv + (ks + 2) * 32, b);
-                    }
-                    if (ks + 1 < k1) {
-                        mma_bf16(h0, a2, a2[0], a2[2]);
-                        mma_bf16(h1, a2, a2[1], a2[3]);
-                        mma_bf16(e0, a2, b2[0], b2[2]);
-                        mma_bf16(e1, a2, b2[1], b2[3]);
-                    }
+                    const int kn = min(ks + 2, kl);
+                    ldmatrix_x4(cur + kn * 32, a);
+                    ldmatrix_x4(prv + kn * 32, b);
+                    mma_bf16(h0, a2, a2[0], a2[2]);
+                    mma_bf16(h1, a2, a2[1], a2[3]);
+                    mma_bf16(e0, a2, b2[0], b2[2]);
+                    mma_bf16(e1, a2, b2[1], b2[3]);
+                }
+                if (ks < k1) {
+                    mma_bf16(g0, a, a[0], a[2]);
+                    mma_bf16(g1, a, a[1], a[3]);
+                    mma_bf16(c0, a, b[0], b[2]);
+                    mma_bf16(c1, a, b[1], b[3]);
                 }
                 const int gb = q & 1;
                 if (q >= 2 && !mbar_wait(gempty_bar + 8 * gb, q / 2 - 1, timed_out)) break;
@@ -498,6 +505,16 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // ----------------------------------- combine warps -----------------------------------
         const int ctid = tid - w_comb * 32, nthr = kCombineWarps * 32;
         const uint32_t red_a = smem_u32(red), redsum_a = smem_u32(redsum);
+        // this thread's entry of the exchange buffers and the matching barrier in every CTA of the cluster
+        // (entry i = 8 numbers x 16 cells, stored [cell][number]; a CTA with fewer than 128 combine
+        // threads would loop, so the addresses are per entry index ctid only when nthr == 128)
+        uint32_t peer_x[kMaxCluster], peer_bar[kMaxCluster];
+#pragma unroll
+        for (int r = 0; r < kMaxCluster; r++) {
+            const uint32_t rr = r < p.C ? r : 0;
+            peer_x[r] = map_to_rank(smem_u32(xchg + rank * kSumVals + (ctid & 15) * 8 + (ctid >> 4)), rr);
+            peer_bar[r] = map_to_rank(xfull_bar, rr);
+        }
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const uint32_t W1s = smem_u32(wtab + it.cls * 32), W2s = W1s + 64;
@@ -521,11 +538,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const int xb = q % kRecRing;
                 if (warp == w_comb && q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
                 if (named_sync_or(2, nthr, timed_out)) { timed_out = true; break; }
-                for (int i = ctid; i < kSumVals; i += nthr) {
-                    const float sum = combine_sums(redsum_a, i & 15, i >> 4, it.vmask, W1s, W2s);
-                    const uint32_t a = smem_u32(xchg + (xb * p.C + rank) * kSumVals + (i & 15) * 8 + (i >> 4));   // [cell][k]
-                    for (int r = 0; r < p.C; r++)
-                        st_async_f32(map_to_rank(a, r), sum, map_to_rank(xfull_bar + 8 * xb, r));
+                {
+                    const float sum = combine_sums(redsum_a, ctid & 15, ctid >> 4, it.vmask, W1s, W2s);
+                    const uint32_t xo = xb * p.C * kSumVals * 4, bo = 8 * xb;
+#pragma unroll
+                    for (int r = 0; r < kMaxCluster; r++)
+                        if (r < p.C) st_async_f32(peer_x[r] + xo, sum, peer_bar[r] + bo);
                 }
             }
         }
@@ -548,6 +566,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // A fragment (16 slots x 16 cells) straight from the record
         const uint32_t woff = 16 + 256 + ((lane & 7) + ((lane >> 3) & 1) * 8) * 32 + (lane >> 4) * 16;
         const long long chan = (long long)rank * p.S + ch0 + 2 * t4;
+        const int ntmax = min(16, (p.S - ch0) >> 3);         // 8-channel tiles of this warp inside the slice
         int total = 0;
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
             if (!skip) total += it.n;
@@ -563,21 +582,34 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             for (int i = 0; i < n_flush; i++) {
                 const uint4 fc = lds_u32x4(rec + 16 + i * 16);       // slot, kind, dst, weight
                 const int slot = (int)fc.x;
+                const bool hi = slot >= 8;
+                const float inv = fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
+                const long long row = (long long)(int)fc.z * p.D + chan;
+                // only the four lanes that hold the slot's rows work; one loop per kind of destination
+                // and per half of the fragment keeps every register index and store offset static
+#define STTM_FLUSH_LOOP(I0, I1, STORE)                                        \
+    _Pragma("unroll") for (int nt = 0; nt < 16; nt++) {                       \
+        const float x = sums[nt][I0] * inv, y = sums[nt][I1] * inv;           \
+        sums[nt][I0] = 0.f;                                                   \
+        sums[nt][I1] = 0.f;                                                   \
+        if (nt < ntmax) { STORE; }                                            \
+    }
+#define STTM_FLUSH_KINDS(I0, I1)                                                                              \
+    if (fc.y != 0) {                                                                                          \
+        float* dst = p.pieces + row;                                                                          \
+        STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x, y))                 \
+    } else if (p.out_f32) {                                                                                   \
+        float* dst = reinterpret_cast<float*>(p.staging) + row;                                               \
+        STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x, y))                 \
+    } else {                                                                                                  \
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.staging) + row;                               \
+        STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<uint32_t*>(dst + nt * 8) = pack_bf16x2(x, y))               \
+    }
                 if (g == (slot & 7)) {
-                    const bool hi = slot >= 8;
-                    const float inv = fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
-                    const long long row = (long long)(int)fc.z * p.D + chan;
-#pragma unroll
-                    for (int nt = 0; nt < 16; nt++) {
-                        const float x = (hi ? sums[nt][2] : sums[nt][0]) * inv, y = (hi ? sums[nt][3] : sums[nt][1]) * inv;
-                        if (hi) { sums[nt][2] = 0.f; sums[nt][3] = 0.f; } else { sums[nt][0] = 0.f; sums[nt][1] = 0.f; }
-                        if (ch0 + nt * 8 < p.S) {
-                            if (fc.y != 0) *reinterpret_cast<float2*>(p.pieces + row + nt * 8) = make_float2(x, y);
-                            else if (p.out_f32) *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.staging) + row + nt * 8) = make_float2(x, y);
-                            else *reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(p.staging) + row + nt * 8) = pack_bf16x2(x, y);
-                        }
-                    }
+                    if (hi) { STTM_FLUSH_KINDS(2, 3) } else { STTM_FLUSH_KINDS(0, 1) }
                 }
+#undef STTM_FLUSH_KINDS
+#undef STTM_FLUSH_LOOP
             }
             __syncwarp();
             if (q < total) {
@@ -602,23 +634,31 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         }
     } else if (warp == w_sim) {
         // --------------------------------- similarity warp ---------------------------------
-        // lane c (and its mirror c + 16) = cell c of the tile
+        // Two frames per pass: lanes 0..15 take frame q, lanes 16..31 frame q + 1; lane c and
+        // lane c + 16 are cell c of the tile.
         const unsigned full = 0xffffffffu;
-        const int c = lane & 15;
+        const int c = lane & 15, half = lane >> 4;
         const int L = p.L;
         const uint32_t xchg_a = smem_u32(xchg);
+        const uint32_t qm = quad_mask(c);
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const float tau_s = taus.s[it.b], tau_t = taus.t[it.b];
             const float w1 = wtab[it.cls * 32 + c], w2 = wtab[it.cls * 32 + 16 + c];
             const bool valid = (it.vmask >> c) & 1u;
-            const uint32_t qm = quad_mask(c);
-            int prev_lv = 0;
-            float prev_nk = 0.f;
-            for (int j = 0; j < it.n; j++, q++) {
-                const int xb = q % kRecRing;
-                if (lane == 0) mbar_expect_tx(xfull_bar + 8 * xb, (uint32_t)(p.C * kSumVals * 4));
-                if (!mbar_wait(xfull_bar + 8 * xb, q / kRecRing, timed_out)) break;
+            const bool quad_exists = (it.vmask & qm) != 0;
+            int carry_lv = 0;               // cover level / squared norm of the node covering cell c in the
+            float carry_nk = 0.f;           // last frame of the previous pass
+            for (int j = 0; j < it.n; j += 2) {
+                const bool two = j + 1 < it.n;
+                const int myq = q + half, xb = myq % kRecRing;
+                const bool mine = half == 0 || two;                 // this half has a frame
+                if (lane == 0) {
+                    mbar_expect_tx(xfull_bar + 8 * (q % kRecRing), (uint32_t)(p.C * kSumVals * 4));
+                    if (two) mbar_expect_tx(xfull_bar + 8 * ((q + 1) % kRecRing), (uint32_t)(p.C * kSumVals * 4));
+                }
+                if (!mbar_wait(xfull_bar + 8 * (q % kRecRing), q / kRecRing, timed_out)) break;
+                if (two && !mbar_wait(xfull_bar + 8 * ((q + 1) % kRecRing), (q + 1) / kRecRing, timed_out)) break;
                 __syncwarp();
                 float v[8];
                 {
@@ -629,12 +669,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                         lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
                         hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
                     }
-                    // cells outside the grid: stale ring rows, dropped
-                    v[0] = valid ? lo.x : 0.f; v[1] = valid ? lo.y : 0.f; v[2] = valid ? lo.z : 0.f; v[3] = valid ? lo.w : 0.f;
-                    v[4] = valid ? hi.x : 0.f; v[5] = valid ? hi.y : 0.f; v[6] = valid ? hi.z : 0.f; v[7] = valid ? hi.w : 0.f;
+                    // cells outside the grid (stale ring rows) and a half without a frame: dropped
+                    const bool keep = valid && mine;
+                    v[0] = keep ? lo.x : 0.f; v[1] = keep ? lo.y : 0.f; v[2] = keep ? lo.z : 0.f; v[3] = keep ? lo.w : 0.f;
+                    v[4] = keep ? hi.x : 0.f; v[5] = keep ? hi.y : 0.f; v[6] = keep ? hi.z : 0.f; v[7] = keep ? hi.w : 0.f;
                 }
                 __syncwarp();
-                if (lane < p.C) mbar_arrive_remote(map_to_rank(xempty_bar + 8 * xb, lane));
+                if (c < p.C && mine) mbar_arrive_remote(map_to_rank(xempty_bar + 8 * xb, c));
 
                 // Section 3.2: cosine of every node with its parent, then the coarse-to-fine search
                 const float n0 = v[0], d0 = v[1], rr = v[2];
@@ -644,12 +685,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 int lv = 0;
                 if (L >= 2) {
                     const bool p0 = !valid || cos_above(d0, n0, n1, tau_s);
-                    const uint32_t pm0 = __ballot_sync(full, p0) & 0xffffu;
+                    const uint32_t pm0 = (__ballot_sync(full, p0) >> (16 * half)) & 0xffffu;
                     const bool quad_pass = (pm0 & qm) == qm;
                     if (L == 3) {
-                        const bool quad_exists = (it.vmask & qm) != 0;
                         const bool p1 = !quad_exists || cos_above(d1, n1, n2, tau_s);
-                        const uint32_t pm1 = __ballot_sync(full, p1) & 0xffffu;
+                        const uint32_t pm1 = (__ballot_sync(full, p1) >> (16 * half)) & 0xffffu;
                         lv = pm1 == 0xffffu ? 2 : (quad_pass ? 1 : 0);
                     } else {
                         lv = quad_pass ? 1 : 0;
@@ -658,33 +698,45 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const float nk = lv == 0 ? n0 : (lv == 1 ? n1 : n2);
 
                 // Section 3.3: the node covering the cell against the overlapping kept node of the
-                // previous frame; a pair is evaluated at the top-left cell of its finer node
+                // previous frame (for the upper half: the lower half's frame); a pair is evaluated
+                // at the top-left cell of its finer node
+                const int lv_lo = __shfl_sync(full, lv, c), lv_hi = __shfl_sync(full, lv, 16 + c);
+                const float nk_lo = __shfl_sync(full, nk, c), nk_hi = __shfl_sync(full, nk, 16 + c);
+                const int lu = half ? lv_lo : carry_lv;
+                const float pnk = half ? nk_lo : carry_nk;
                 int link_local = -1;
-                if (j > 0) {
-                    const int lu = prev_lv;
+                {
                     const float t11 = w1 * quad_sum(v[4]), t12 = w1 * quad_sum(v[5]);
                     const float t21 = w1 * quad_sum(v[7]), t22 = half_warp_sum(w2 * v[5]);
                     float dot;
                     if (lv == 0) dot = lu == 0 ? v[3] : (lu == 1 ? v[4] : v[5]);
                     else if (lv == 1) dot = lu == 0 ? v[6] : (lu == 1 ? t11 : t12);
                     else dot = lu == 0 ? v[7] : (lu == 1 ? t21 : t22);
-                    const bool rep = valid && tile_anchor(c, min(lv, lu)) == c;
-                    const bool pass = rep && cos_above(dot, nk, prev_nk, tau_t);
-                    const uint32_t passm = __ballot_sync(full, pass) & 0xffffu;
+                    const bool has_prev = j + half > 0;
+                    const bool rep = valid && has_prev && tile_anchor(c, min(lv, lu)) == c;
+                    const bool pass = rep && cos_above(dot, nk, pnk, tau_t);
+                    const uint32_t passm = (__ballot_sync(full, pass) >> (16 * half)) & 0xffffu;
                     const uint32_t cand = passm & region_mask(c, lv);
                     const int cstar = cand ? __ffs(cand) - 1 : 0;     // first in row-major order: the top-left one
-                    const int lu_star = __shfl_sync(full, lu, cstar);
+                    const int lu_star = __shfl_sync(full, lu, 16 * half + cstar);
                     link_local = cand ? tile_anchor(cstar, lu_star) : -1;
                 }
-                prev_lv = lv;
-                prev_nk = nk;
+                carry_lv = two ? lv_hi : lv_lo;
+                carry_nk = two ? nk_hi : nk_lo;
 
                 // hand the cover level and the link of every cell to the chain warp
-                if (q >= kRecRing && !mbar_wait(hempty_bar + 8 * xb, q / kRecRing - 1, timed_out)) break;
+                if (q >= kRecRing && !mbar_wait(hempty_bar + 8 * (q % kRecRing), q / kRecRing - 1, timed_out)) break;
+                if (two && q + 1 >= kRecRing &&
+                    !mbar_wait(hempty_bar + 8 * ((q + 1) % kRecRing), (q + 1) / kRecRing - 1, timed_out))
+                    break;
                 __syncwarp();
-                if (lane < 16) hand[xb * 16 + c] = lv | ((link_local + 1) << 8);
+                if (mine) hand[xb * 16 + c] = lv | ((link_local + 1) << 8);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(hfull_bar + 8 * xb);
+                if (lane == 0) {
+                    mbar_arrive(hfull_bar + 8 * (q % kRecRing));
+                    if (two) mbar_arrive(hfull_bar + 8 * ((q + 1) % kRecRing));
+                }
+                q += two ? 2 : 1;
             }
         }
     } else if (warp == w_chain) {

@@ -360,7 +360,9 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
 template <typename OutT>
 sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacity, cudaStream_t st) {
     const Geo g = pl.g;
-    k_gather<OutT><<<kSmCount * 8, 256, 0, st>>>(g, (const long long*)(ws + pl.vid_off),
+    // one warp per row; the row count is only known on the device, so the grid covers the most rows there can be
+    const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
+    k_gather<OutT><<<blocks_for(max_rows, 8), 256, 0, st>>>(g, (const long long*)(ws + pl.vid_off),
                                                  (const int32_t*)(ws + pl.row_anchor),
                                                  (const int32_t*)(ws + pl.row_head),
                                                  (const int32_t*)(ws + pl.piece_next),

@@ -437,18 +437,19 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const uint32_t loff = lrow * p.row_bytes + lk * 2;
         const int ksteps = p.S >> 4;
         const int k0 = ksteps * warp / p.NM, k1 = ksteps * (warp + 1) / p.NM;     // this warp's channel steps
+        int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before (q = use * R + s)
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             for (int j = 0; j < it.n; j++, q++) {
-                const int s = q % p.R;
-                if (!mbar_wait(full_bar + 8 * s, q / p.R, timed_out)) break;
+                if (!mbar_wait(full_bar + 8 * s, use, timed_out)) break;
                 __syncwarp();
                 float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
                 float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
                 float h0[4] = {0.f, 0.f, 0.f, 0.f}, h1[4] = {0.f, 0.f, 0.f, 0.f};
                 float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
                 const uint32_t cur = ring_base + s * p.slot_bytes + loff;
-                const uint32_t prv = ring_base + ((q + p.R - 1) % p.R) * p.slot_bytes + loff;
+                const int sp = s == 0 ? p.R - 1 : s - 1;
+                const uint32_t prv = ring_base + sp * p.slot_bytes + loff;
                 // two accumulator sets; the fragments of a step are loaded before the products of the
                 // step before it are issued (the index is clamped at the end: a repeated load, no branch)
                 uint32_t a[4], b[4], a2[4], b2[4];
@@ -497,8 +498,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (lane == 0) {
                     mbar_arrive(gfull_bar + 8 * gb);
                     // done with the previous frame's slot (the current one stays for the next frame)
-                    if (q >= 1) mbar_arrive(empty_bar + 8 * ((q - 1) % p.R));
+                    if (q >= 1) mbar_arrive(empty_bar + 8 * sp);
                 }
+                if (++s == p.R) { s = 0; use++; }
             }
         }
     } else if (warp < w_sum) {
@@ -571,10 +573,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
             if (!skip) total += it.n;
         // one record per frame, and a last one that only writes out what the last item left
+        int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before
         for (; q <= total; q++) {
-            const int rk = q % kRecRing, s = q % p.R;
+            const int rk = q % kRecRing;
             if (!mbar_wait(rfull_bar + 8 * rk, q / kRecRing, timed_out)) break;
-            if (q < total && !mbar_wait(full_bar + 8 * s, q / p.R, timed_out)) break;
+            if (q < total && !mbar_wait(full_bar + 8 * s, use, timed_out)) break;
             __syncwarp();
             const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
             const int n_flush = (int)lds_u32x4(rec).x;
@@ -631,6 +634,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 mbar_arrive(rempty_bar + 8 * rk);
                 if (q < total) mbar_arrive(empty_bar + 8 * s);
             }
+            if (++s == p.R) { s = 0; use++; }
         }
     } else if (warp == w_sim) {
         // --------------------------------- similarity warp ---------------------------------
@@ -865,12 +869,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         }
     } else if (warp == w_prod) {
         // ----------------------------------- producer warp -----------------------------------
+        int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             for (int j = 0; j < it.n; j++, q++) {
-                const int s = q % p.R;
                 const uint32_t bar = full_bar + 8 * s;
-                if (q >= p.R && !mbar_wait(empty_bar + 8 * s, q / p.R - 1, timed_out)) break;
+                if (use >= 1 && !mbar_wait(empty_bar + 8 * s, use - 1, timed_out)) break;
                 __syncwarp();
                 if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
                 __syncwarp();
@@ -880,6 +884,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     bulk_g2s(ring_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
                              (uint32_t)(p.S * 2), bar);
                 }
+                if (++s == p.R) { s = 0; use++; }
             }
         }
         // the CTA must not end with copies in flight: the last R frames issued have landed?
@@ -996,14 +1001,26 @@ k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict
                 last = best;
             }
             const float wsum = (float)row_weight[r];
-            for (int d = lane * VEC; d < g.D; d += kSliceCh) {
-                float sum[VEC] = {0.f, 0.f, 0.f, 0.f};
+            // four 128-channel groups per trip, so that 4 x n loads are in flight
+            for (int d0 = lane * VEC; d0 < g.D; d0 += 4 * kSliceCh) {
+                float sum[4][VEC];
+#pragma unroll
+                for (int u = 0; u < 4; u++)
+#pragma unroll
+                    for (int v = 0; v < VEC; v++) sum[u][v] = 0.f;
                 if (!longer) {
 #pragma unroll
                     for (int k = 0; k < kMaxList; k++) {
                         if (k < n) {
-                            const float4 v = *reinterpret_cast<const float4*>(pieces + (long long)ids[k] * g.D + d);
-                            sum[0] += v.x; sum[1] += v.y; sum[2] += v.z; sum[3] += v.w;
+                            const float* src = pieces + (long long)ids[k] * g.D;
+#pragma unroll
+                            for (int u = 0; u < 4; u++) {
+                                const int d = d0 + u * kSliceCh;
+                                if (d < g.D) {
+                                    const float4 v = __ldcs(reinterpret_cast<const float4*>(src + d));
+                                    sum[u][0] += v.x; sum[u][1] += v.y; sum[u][2] += v.z; sum[u][3] += v.w;
+                                }
+                            }
                         }
                     }
                 } else {
@@ -1013,14 +1030,27 @@ k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict
                         for (int pc = head; pc >= 0; pc = piece_next[pc])
                             if (pc > lst && pc < best) best = pc;
                         if (best == 0x7fffffff) break;
-                        const float4 v = *reinterpret_cast<const float4*>(pieces + (long long)best * g.D + d);
-                        sum[0] += v.x; sum[1] += v.y; sum[2] += v.z; sum[3] += v.w;
+                        const float* src = pieces + (long long)best * g.D;
+#pragma unroll
+                        for (int u = 0; u < 4; u++) {
+                            const int d = d0 + u * kSliceCh;
+                            if (d < g.D) {
+                                const float4 v = *reinterpret_cast<const float4*>(src + d);
+                                sum[u][0] += v.x; sum[u][1] += v.y; sum[u][2] += v.z; sum[u][3] += v.w;
+                            }
+                        }
                         lst = best;
                     }
                 }
 #pragma unroll
-                for (int v = 0; v < VEC; v++) sum[v] = sum[v] / wsum;
-                store4(out + r * g.D + d, sum);
+                for (int u = 0; u < 4; u++) {
+                    const int d = d0 + u * kSliceCh;
+                    if (d < g.D) {
+#pragma unroll
+                        for (int v = 0; v < VEC; v++) sum[u][v] = sum[u][v] / wsum;
+                        store4(out + r * g.D + d, sum[u]);
+                    }
+                }
             }
         }
     }

@@ -34,9 +34,11 @@ METRIC = "input visual tokens/sec merged on 1 B200; achieved HBM GB/s vs peak"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic per launch of the dominant kernel, from the ncu capture summarised under
-# profiles/ (bytes read + written for the benchmark's workload); None until captured.
-NCU_TRAFFIC_BYTES = {}
+# DRAM traffic of a kernel as a multiple of its algorithmic bytes, from the ncu capture
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on the qwen workload;
+# a streaming kernel's traffic grows in proportion to the bytes it must move, so the ratio is
+# applied to the benchmark workload's algorithmic bytes).  Absent = no capture of the current kernel.
+NCU_TRAFFIC_RATIO = {}
 
 
 def workload_setup(name: str):
@@ -241,7 +243,8 @@ def run_ours(args):
     achieved = stage_bytes[dominant] / (stage_ms[dominant] / 1e3) / 1e9
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": "of " + peak_kind,
-                "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+                "traffic": (NCU_TRAFFIC_RATIO[dominant] * stage_bytes[dominant]
+                            if dominant in NCU_TRAFFIC_RATIO else None),
                 "algorithmic_bytes": stage_bytes[dominant], "kernel_ms": stage_ms[dominant],
                 "stage_ms": stage_ms,
                 "path": {"algorithmic_bytes": path_bytes, "achieved": path_bytes / (ms_per_step / 1e3) / 1e9,

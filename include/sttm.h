@@ -93,6 +93,30 @@ sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size
                          void* stream);
 
 /*
+ * Spatial stage alone, for callers that cannot give the library any device memory beyond
+ * inputs and outputs.  (The paper has no counterpart: this is a deployment convenience.)
+ * Who that is: code running where device allocation is off the table - a serving process whose
+ * whole HBM has already been handed to a tensor pool, a latency-critical loop in which a
+ * cudaMalloc (which may synchronise the device) must not happen, a plug-in that receives raw
+ * pointers and owns no allocator.  Same computation and same outputs as sttm_spatial; the one
+ * scratch buffer the stage needs (a squared norm per quadtree node) sits in a fixed array of
+ * STTM_STATIC_SCRATCH_BYTES inside the library image, which every GPU that loads the library
+ * keeps until the process ends.
+ *   - Problems that need more scratch (B*T*columns*nodes-per-column*4 bytes, e.g. 1024 frames
+ *     of a 13x13 grid need 1.4 MB) are refused with STTM_ERR_WORKSPACE and nothing runs.
+ *   - No allocation, no free, on any path.  The first call on a device asks the runtime for the
+ *     array's device address (with that device current); make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the array and it keeps what the last call left there.  Nothing
+ *     stale is read (the norms are rewritten, the counts are zeroed first), but two calls whose
+ *     kernels overlap on the GPU - different streams, different threads - race on it: serialise
+ *     them.  sttm_temporal needs the norms in a caller workspace, so it does not pair with this.
+ */
+#define STTM_STATIC_SCRATCH_BYTES (4u << 20)
+sttm_status sttm_spatial_static(const void* feats, const sttm_params* p, int8_t* cover_level,
+                                int32_t* frame_counts, float* spatial_sims, void* stream);
+
+/*
  * Temporal stage alone (Section 3.3), given the spatial stage's cover map.
  *   link [B, T*H*W] int32  out, per cell: anchor id of the node (frame t-1) that the
  *                          cell's covering node is linked to, or -1

@@ -26,7 +26,7 @@ EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame",
            "sttm_temporal", "sttm_merge_ex", "sttm_merge", "sttm_merge_host", "sttm_release_cache",
            "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
            "sttm_set_stage_events", "sttm_set_tuning", "sttm_last_path",
-           "sttm_fused_launch_shape"]
+           "sttm_fused_launch_shape", "sttm_spatial_static"]
 
 
 class SttmParams(C.Structure):
@@ -65,6 +65,8 @@ def load_library(path: Optional[str] = None):
     lib.sttm_sims_per_frame.restype = C.c_int
     lib.sttm_spatial.argtypes = [vp, pp, vp, C.c_size_t, vp, vp, vp, vp]
     lib.sttm_spatial.restype = C.c_int
+    lib.sttm_spatial_static.argtypes = [vp, pp, vp, vp, vp, vp]
+    lib.sttm_spatial_static.restype = C.c_int
     lib.sttm_temporal.argtypes = [vp, pp, vp, C.c_size_t, vp, vp, vp, vp, vp, vp]
     lib.sttm_temporal.restype = C.c_int
     lib.sttm_merge_ex.argtypes = [vp, pp, vp, C.c_size_t, vp, vp, vp, vp, vp, vp, vp]
@@ -200,6 +202,18 @@ def sttm_spatial(feats: torch.Tensor, tau_s, lv1: int = 4, want_sims: bool = Fal
     _check(load_library().sttm_spatial(_ptr(feats), C.byref(prob.params), _ptr(ws), ws.numel(), _ptr(cover),
                                        _ptr(counts), _ptr(sims), _stream()), "sttm_spatial")
     return cover, counts, sims, ws
+
+
+def sttm_spatial_static(feats: torch.Tensor, tau_s, cover: torch.Tensor, counts: torch.Tensor,
+                        sims: Optional[torch.Tensor] = None, lv1: int = 4) -> None:
+    """Spatial stage through the entry point that allocates nothing: the caller passes every
+    output buffer (``cover`` int8 [B,T,H,W], ``counts`` int32 [B,T], optionally ``sims`` float32
+    [B,T,sims_per_frame]); the stage's scratch is the fixed array inside the library.  Raises
+    SttmError("workspace too small") when the problem needs more scratch than that array has."""
+    feats = _as5d(feats)
+    prob = make_params(feats.shape, feats.dtype, tau_s, 2.0, lv1)
+    _check(load_library().sttm_spatial_static(_ptr(feats), C.byref(prob.params), _ptr(cover), _ptr(counts),
+                                              _ptr(sims), _stream()), "sttm_spatial_static")
 
 
 def sttm_temporal(feats: torch.Tensor, cover: torch.Tensor, tau_s, tau_t, ws: torch.Tensor, lv1: int = 4,

@@ -373,6 +373,28 @@ sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacit
 
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
 
+// Scratch of sttm_spatial_static: lives in the library image, so every GPU that loads the
+// library holds these bytes until the process exits.  In host code the name below is only a
+// handle for the runtime, never an address a kernel may use; the device address comes from
+// cudaGetSymbolAddress, asked once per device while that device is current.
+constexpr size_t kStaticScratchBytes = STTM_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+void* g_static_scratch_addr[64] = {};
+
+sttm_status static_scratch_address(void** out) {
+    int dev = 0;
+    STTM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return STTM_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        STTM_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (ptr == nullptr) return STTM_ERR_CUDA;
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return STTM_OK;
+}
+
 // cached buffers for sttm_merge / sttm_merge_host, one set per device
 struct Cache {
     void* ws = nullptr; size_t ws_bytes = 0;
@@ -470,6 +492,27 @@ sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size
     g_launches = 0;
     STTM_CUDA_TRY(cudaMemsetAsync(frame_counts, 0, (size_t)pl.g.B * pl.g.T * 4, st));
     return run_spatial(feats, p, pl, (char*)ws, cover_level, frame_counts, spatial_sims, st);
+}
+
+sttm_status sttm_spatial_static(const void* feats, const sttm_params* p, int8_t* cover_level, int32_t* frame_counts,
+                                float* spatial_sims, void* stream) {
+    Plan pl;
+    sttm_status s = make_plan(p, &pl);
+    if (s != STTM_OK) return s;
+    if (!feats || !cover_level || !frame_counts) return STTM_ERR_ARG;
+    if (misaligned(feats, 16)) return STTM_ERR_ARG;
+    // the only scratch of the spatial stage: one squared norm per quadtree node
+    const int nodes_per_column = pl.g.L == 3 ? 21 : (pl.g.L == 2 ? 5 : 1);
+    const size_t need = (size_t)pl.g.B * pl.g.T * pl.g.ncol * nodes_per_column * sizeof(float);
+    if (need > kStaticScratchBytes) return STTM_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    if ((s = static_scratch_address(&scratch)) != STTM_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    g_launches = 0;
+    // the counts are added to, so they start at zero; the norms are overwritten, nothing of an
+    // earlier call is read
+    STTM_CUDA_TRY(cudaMemsetAsync(frame_counts, 0, (size_t)pl.g.B * pl.g.T * 4, st));
+    return run_spatial(feats, p, pl, (char*)scratch - pl.norms, cover_level, frame_counts, spatial_sims, st);
 }
 
 sttm_status sttm_temporal(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,

@@ -3,4 +3,4 @@
 ``inputs`` (seeded synthetic videos) imports nothing from the CUDA side.  ``binding``
 loads the library lazily and raises when it is missing: there is no CPU fallback.
 """
-__all__ = ["inputs", "binding", "build"]
+__all__ = ["inputs", "binding", "build", "shard"]

@@ -78,7 +78,7 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     f->NA = (f->S + 127) / 128;
     f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
     f->slot_bytes = 16 * f->row_bytes;
-    const size_t fixed = (size_t)2 * f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
+    const size_t fixed = (size_t)f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
                          16 * 32 * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) +
                          (2 * kMaxRing + 6 * kRecRing + 4) * 8;
     int R = (int)((kMaxSmem - fixed) / f->slot_bytes);

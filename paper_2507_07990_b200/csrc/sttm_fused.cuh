@@ -369,7 +369,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* ring = smem;
     size_t off = (size_t)p.R * p.slot_bytes;
-    float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)2 * p.NM * kGramVals * 4;   // two frames
+    float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)p.NM * kGramVals * 4;
     float* redsum = reinterpret_cast<float*>(smem + off);    off += kGramVals * 4;
     float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * p.C * kSumVals * 4;
     float* wtab = reinterpret_cast<float*>(smem + off);      off += 16 * 32 * 4;      // [shape][W1 x16, W2 x16]
@@ -478,11 +478,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     mma_bf16(c0, a, b[0], b[2]);
                     mma_bf16(c1, a, b[1], b[3]);
                 }
-                const int gb = q & 1;
-                if (q >= 2 && !mbar_wait(gempty_bar + 8 * gb, q / 2 - 1, timed_out)) break;
+                // the combine warps have taken the previous frame's parts out of the buffer?
+                if (q >= 1 && !mbar_wait(gempty_bar, q - 1, timed_out)) break;
                 __syncwarp();
                 {
-                    float* r = red + (gb * p.NM + warp) * kGramVals;
+                    float* r = red + warp * kGramVals;
                     const int gr = lane >> 2, gc = (lane & 3) * 2;
                     *reinterpret_cast<float2*>(r + gr * 16 + gc) = make_float2(g0[0] + h0[0], g0[1] + h0[1]);
                     *reinterpret_cast<float2*>(r + (gr + 8) * 16 + gc) = make_float2(g0[2] + h0[2], g0[3] + h0[3]);
@@ -496,7 +496,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 }
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(gfull_bar + 8 * gb);
+                    mbar_arrive(gfull_bar);
                     // done with the previous frame's slot (the current one stays for the next frame)
                     if (q >= 1) mbar_arrive(empty_bar + 8 * sp);
                 }
@@ -521,21 +521,20 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             if (skip) continue;
             const uint32_t W1s = smem_u32(wtab + it.cls * 32), W2s = W1s + 64;
             for (int j = 0; j < it.n; j++, q++) {
-                const int gb = q & 1;
                 // the first combine warp waits; the named barriers hand the outcome to the others
-                if (warp == w_comb) mbar_wait(gfull_bar + 8 * gb, q / 2, timed_out);
+                if (warp == w_comb) mbar_wait(gfull_bar, q, timed_out);
                 if (named_sync_or(3, nthr, timed_out)) { timed_out = true; break; }
                 // add the Gram warps' parts, each thread a share of the 512 entries
                 for (int i = ctid * 4; i < kGramVals; i += nthr * 4) {
-                    float4 sum = lds_f32x4(red_a + (gb * p.NM * kGramVals + i) * 4);
+                    float4 sum = lds_f32x4(red_a + i * 4);
                     for (int w = 1; w < p.NM; w++) {
-                        const float4 v = lds_f32x4(red_a + ((gb * p.NM + w) * kGramVals + i) * 4);
+                        const float4 v = lds_f32x4(red_a + (w * kGramVals + i) * 4);
                         sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
                     }
                     *reinterpret_cast<float4*>(redsum + i) = sum;
                 }
                 named_sync(1, nthr);
-                if (lane == 0) mbar_arrive(gempty_bar + 8 * gb);
+                if (lane == 0) mbar_arrive(gempty_bar);
                 // contract to 8 numbers per cell and send this CTA's share to every CTA of the cluster
                 const int xb = q % kRecRing;
                 if (warp == w_comb && q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);

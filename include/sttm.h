@@ -188,7 +188,8 @@ void sttm_set_stage_events(void** events);
  * Benchmark and test knobs; 0 leaves a choice to the library.
  *   path             1: always the three-pass kernels, 2 or 0: the fused single-read kernel
  *                    wherever it applies (bf16 input, D a multiple of 16, at most 64 tiles of
- *                    4x4 cells per frame, D / cluster_size <= 1024)
+ *                    4x4 cells per frame, D / cluster_size <= 1024), 3: the same without
+ *                    packing the partial border tiles of a frame together
  *   cluster_size     CTAs that share one tile's channels (1, 2, 4 or 8)
  *   frames_per_item  frames of one tile that one cluster processes in a row
  * Not thread safe; affects later calls of every entry point.

@@ -8,6 +8,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 #include "sttm_kernels.cuh"
 #include "sttm_fused.cuh"
@@ -38,7 +39,7 @@ struct FusedPlan {
     bool ok;
     int C, S, NM, NA, R, row_bytes, slot_bytes, F, nseg, nitems, ntiles, Wt;
     size_t smem;
-    unsigned char tile_order[kMaxTiles];
+    TileDesc tiles[kMaxTiles];      // most cells first
 };
 
 struct Plan {
@@ -54,17 +55,73 @@ struct Plan {
 };
 
 // benchmark / test knobs (sttm_set_tuning): 0 = choose automatically
-int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0;
+int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0, g_tune_pack = 0;
 
 constexpr size_t kMaxSmem = 232448;   // 227 KB per CTA on sm_100
+
+// Cuts the grid into the kernel's tiles.  Full 4x4 tiles map one to one.  The partial tiles of
+// the right and bottom border are packed several to a tile: a partial tile of r x c cells sits
+// at an offset (oy, ox) of the 4x4 lane grid that keeps its own 2x2 blocks on lane pairs
+// (ox even when c >= 2, ox = 0 when c > 2, the same for rows), and every lane records which
+// neighbour lanes belong to its block and its coarsest node, so packed tiles never mix.
+int fused_resident_clusters(const FusedPlan& f);
+
+bool build_tiles(const Geo& g, FusedPlan* f) {
+    struct Part { int y0, x0, r, c; };
+    std::vector<Part> full, part;
+    for (int y0 = 0; y0 < g.H; y0 += 4)
+        for (int x0 = 0; x0 < g.W; x0 += 4) {
+            Part pt{y0, x0, std::min(4, g.H - y0), std::min(4, g.W - x0)};
+            (pt.r == 4 && pt.c == 4 ? full : part).push_back(pt);
+        }
+    std::vector<TileDesc> tiles;
+    auto blank = [] { TileDesc t; std::memset(t.y, 255, 16); std::memset(t.x, 0, 16); std::memset(t.bits, 0, 16); return t; };
+    auto place = [&](TileDesc& t, const Part& pt, int oy, int ox) {
+        const int qb = (pt.c >= 2 ? 1 : 0) | (pt.r >= 2 ? 4 : 0);
+        const int tb = qb | (pt.c > 2 ? 2 : 0) | (pt.r > 2 ? 8 : 0);
+        for (int dy = 0; dy < pt.r; dy++)
+            for (int dx = 0; dx < pt.c; dx++) {
+                const int l = (oy + dy) * 4 + ox + dx;
+                t.y[l] = (unsigned char)(pt.y0 + dy);
+                t.x[l] = (unsigned char)(pt.x0 + dx);
+                t.bits[l] = (unsigned char)(qb | (tb << 4));
+            }
+    };
+    if (g.H > 254 || g.W > 254) return false;
+    for (const Part& pt : full) { TileDesc t = blank(); place(t, pt, 0, 0); tiles.push_back(t); }
+    std::vector<TileDesc> packed;
+    std::stable_sort(part.begin(), part.end(), [](const Part& a, const Part& b) { return a.r * a.c > b.r * b.c; });
+    for (const Part& pt : part) {
+        bool done = false;
+        for (size_t k = 0; k < packed.size() && !done; k++) {
+            if (g_tune_pack == 1) break;
+            for (int oy = 0; oy + pt.r <= 4 && !done; oy++) {
+                if ((pt.r >= 2 && (oy & 1)) || (pt.r > 2 && oy != 0)) continue;
+                for (int ox = 0; ox + pt.c <= 4 && !done; ox++) {
+                    if ((pt.c >= 2 && (ox & 1)) || (pt.c > 2 && ox != 0)) continue;
+                    bool free_ = true;
+                    for (int dy = 0; dy < pt.r; dy++)
+                        for (int dx = 0; dx < pt.c; dx++)
+                            if (packed[k].y[(oy + dy) * 4 + ox + dx] != 255) free_ = false;
+                    if (free_) { place(packed[k], pt, oy, ox); done = true; }
+                }
+            }
+        }
+        if (!done) { TileDesc t = blank(); place(t, pt, 0, 0); packed.push_back(t); }
+    }
+    for (const TileDesc& t : packed) tiles.push_back(t);
+    if ((int)tiles.size() > kMaxTiles) return false;
+    f->ntiles = (int)tiles.size();
+    for (int t = 0; t < f->ntiles; t++) f->tiles[t] = tiles[t];
+    return true;
+}
 
 void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     f->ok = false;
     if (g_tune_path == 1) return;
     if (p->in_dtype != STTM_BF16 || g.D % 16 != 0) return;
     f->Wt = (g.W + 3) / 4;
-    f->ntiles = ((g.H + 3) / 4) * f->Wt;
-    if (f->ntiles > kMaxTiles) return;
+    if (!build_tiles(g, f)) return;
     int C = 0;
     for (int c = 1; c <= kMaxCluster; c *= 2) {
         if (g_tune_cluster && c != g_tune_cluster) continue;
@@ -86,23 +143,29 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     if (R < 4) return;
     f->R = R;
     f->smem = (size_t)R * f->slot_bytes + fixed;
-    // frames per item: about four items per resident cluster, counted in full tiles
-    const double tiles_equiv = (double)g.HW / 16.0;
-    const double want = (double)g.B * g.T * tiles_equiv / (4.0 * (kSmCount / C));
-    int F = g_tune_seg > 0 ? g_tune_seg : std::max(8, std::min((int)std::ceil(want), 256));
-    F = std::min(F, g.T);
-    f->F = F;
-    f->nseg = (g.T + F - 1) / F;
-    f->nitems = g.B * f->ntiles * f->nseg;
-    // tiles with more cells inside the grid first
-    int cells[kMaxTiles];
-    for (int t = 0; t < f->ntiles; t++) {
-        const int y0 = (t / f->Wt) * 4, x0 = (t % f->Wt) * 4;
-        cells[t] = std::min(4, g.H - y0) * std::min(4, g.W - x0);
-        f->tile_order[t] = (unsigned char)t;
+    // frames per item: about four items per resident cluster, with the number of items as close
+    // below a multiple of the cluster count as the frame count allows (the items are dealt out
+    // statically, and every item of a cluster costs about the same)
+    if (g_tune_seg > 0) {
+        f->F = std::min(g_tune_seg, g.T);
+    } else {
+        const int ncl = fused_resident_clusters(*f);
+        const long long tiles_all = (long long)g.B * f->ntiles;
+        const int lo = std::max(1, (int)(g.T / 256)), hi = std::max(lo, std::min(g.T, std::max(1, g.T / 8)));
+        double best_cost = 1e300;
+        int best_nseg = lo;
+        for (int nseg = lo; nseg <= hi; nseg++) {
+            const int F = (g.T + nseg - 1) / nseg;
+            if ((g.T + F - 1) / F != nseg) continue;
+            const long long items = tiles_all * nseg;
+            const long long rounds = (items + ncl - 1) / ncl;
+            const double cost = (double)rounds * (F + 1 + 6);        // frames + the frame before + pipeline fill
+            if (cost < best_cost - 1e-9) { best_cost = cost; best_nseg = nseg; }
+        }
+        f->F = (g.T + best_nseg - 1) / best_nseg;
     }
-    std::stable_sort(f->tile_order, f->tile_order + f->ntiles,
-                     [&](unsigned char a, unsigned char b) { return cells[a] > cells[b]; });
+    f->nseg = (g.T + f->F - 1) / f->F;
+    f->nitems = g.B * f->ntiles * f->nseg;
     f->ok = true;
 }
 
@@ -338,7 +401,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.pieces = (float*)(ws + pl.pieces);
     fp.piece_meta = (int2*)(ws + pl.piece_meta);
     fp.status = device_status;
-    std::memcpy(fp.tile_order, f.tile_order, sizeof(fp.tile_order));
+    std::memcpy(fp.tiles, f.tiles, sizeof(fp.tiles));
     Taus taus;
     fill_taus(p, &taus);
 
@@ -475,7 +538,8 @@ int sttm_fused_launch_shape(const sttm_params* p, int* shape) {
 void sttm_set_stage_events(void** events) { g_stage_events = (cudaEvent_t*)events; }
 
 void sttm_set_tuning(int path, int cluster_size, int frames_per_item) {
-    g_tune_path = path;
+    g_tune_path = path == 3 ? 2 : path;
+    g_tune_pack = path == 3 ? 1 : 0;
     g_tune_cluster = cluster_size;
     g_tune_seg = frames_per_item;
 }

@@ -4,7 +4,10 @@
 // Decomposition.  A frame is cut into 4x4-cell tiles (the region of a coarsest quadtree
 // node when the tree has three levels; four / sixteen independent regions when it has two
 // / one).  Everything that touches features stays inside one tile through time, so a work
-// item is (video, tile, run of consecutive frames).  A thread-block cluster of C CTAs owns
+// item is (video, tile, run of consecutive frames).  The partial tiles at the right and
+// bottom border of a grid whose sides are not multiples of four are packed, several at a
+// time, into the 16 rows of one "tile" of the kernel (they never interact: every lane knows
+// which of its neighbours belong to its own 2x2 block and coarsest node).  A thread-block cluster of C CTAs owns
 // a fixed list of items; each CTA owns D/C channels of the tile and streams them frame by
 // frame through a shared-memory ring filled by bulk asynchronous copies (one per cell).
 //
@@ -65,6 +68,14 @@ struct FrameRec {
     uint16_t wmat[256];
 };
 
+// One tile of the kernel: up to 16 cells of a frame, row l of the tile = lane l of the
+// decision warps.  y == 255: no cell.  bits: low nibble = which lane-index bits join the lanes
+// of one 2x2 block (1: the lane to the right, 4: the lane below), high nibble = the same for
+// the coarsest node (1, 2: along the row, 4, 8: down the column).  A full tile has 0xf5.
+struct TileDesc {
+    unsigned char y[16], x[16], bits[16];
+};
+
 struct FusedParams {
     const __nv_bfloat16* feats;
     int B, T, H, W, D, L;
@@ -81,7 +92,7 @@ struct FusedParams {
     float* pieces;           // [nitems][kPieceSlots][D]
     int2* piece_meta;        // [nitems][kPieceSlots] {key cell id or -1, weight}
     int* status;
-    unsigned char tile_order[kMaxTiles];
+    TileDesc tiles[kMaxTiles];   // most cells first
 };
 
 // ---------------------------------------------------------------------------------
@@ -226,14 +237,47 @@ __device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
     return v;
 }
 
-// tile-local cell c = dy*4 + dx; top-left cell of the level-lv node that holds c
-__device__ __forceinline__ int tile_anchor(int c, int lv) {
-    const int m = ~((1 << lv) - 1);
-    return (((c >> 2) & m) << 2) | ((c & 3) & m);
+// What lane c of a decision warp knows about its cell: the lanes of its 2x2 block and of its
+// coarsest node (bit masks over the 16 lanes, cells inside the grid only), the averaging
+// weights (w1: of a cell in its block; w2: of a cell in the coarsest node = mean of the
+// existing blocks' means), its position in the frame.
+struct LaneGeo {
+    bool valid;
+    int qbits, tbits;
+    uint32_t qmask, tmask;
+    float w1, w2;
+    int cell;               // y * W + x
+};
+// Pure function of the tile description: any thread can ask for any lane.
+__device__ __forceinline__ LaneGeo lane_geo(const TileDesc& td, int c, int L, int W) {
+    LaneGeo g;
+    g.valid = td.y[c] != 255;
+    g.qbits = L >= 2 ? (td.bits[c] & 15) : 0;
+    g.tbits = L == 3 ? (td.bits[c] >> 4) : 0;
+    g.qmask = 0;
+    g.tmask = 0;
+    int blocks = 0;
+    for (int l = 0; l < 16; l++) {
+        if (td.y[l] == 255) continue;
+        const int ql = L >= 2 ? (td.bits[l] & 15) : 0, tl = L == 3 ? (td.bits[l] >> 4) : 0;
+        if ((l & ~ql) == (c & ~g.qbits)) g.qmask |= 1u << l;
+        if ((l & ~tl) == (c & ~g.tbits)) {
+            g.tmask |= 1u << l;
+            blocks += (l & ~ql) == l ? 1 : 0;         // top-left cells of the blocks of the node
+        }
+    }
+    if (!g.valid) { g.qmask = 0; g.tmask = 0; }
+    g.w1 = g.valid && L >= 2 ? 1.f / (float)__popc(g.qmask) : 0.f;
+    g.w2 = g.valid && L == 3 ? g.w1 / (float)blocks : 0.f;
+    g.cell = g.valid ? td.y[c] * W + td.x[c] : 0;
+    return g;
 }
-__device__ __forceinline__ uint32_t quad_mask(int c) { return 0x33u << (8 * (c >> 3) + 2 * ((c >> 1) & 1)); }
-__device__ __forceinline__ uint32_t region_mask(int c, int lv) {
-    return lv == 0 ? (1u << c) : (lv == 1 ? quad_mask(c) : 0xffffu);
+// top-left lane of the level-lv node of lane c
+__device__ __forceinline__ int lane_anchor(const LaneGeo& g, int c, int lv) {
+    return lv == 0 ? c : (lv == 1 ? (c & ~g.qbits) : (c & ~g.tbits));
+}
+__device__ __forceinline__ uint32_t lane_region(const LaneGeo& g, int c, int lv) {
+    return lv == 0 ? (g.valid ? 1u << c : 0u) : (lv == 1 ? g.qmask : g.tmask);
 }
 // position of the k-th (0-based) set bit of a 16-bit mask that has more than k bits set
 __device__ __forceinline__ int kth_set_bit16(uint32_t m, int k) {
@@ -254,16 +298,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float x, float y) {
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// sum over lanes that share (lane & 16): every lane of a half gets its half's total
-__device__ __forceinline__ float half_warp_sum(float v) {
+// sum over the lanes of the lane's coarsest node (lanes 0..15 and 16..31 separately): a butterfly
+// over the lane-index bits that stay inside the node
+__device__ __forceinline__ float top_sum(float v, int tbits) {
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    for (int o = 8; o > 0; o >>= 1) {
+        const float t = __shfl_xor_sync(0xffffffffu, v, o);
+        v += (tbits & o) ? t : 0.f;
+    }
     return v;
 }
-// sum over the four cells of the lane's 2x2 block (lane = cell, or cell + 16)
-__device__ __forceinline__ float quad_sum(float v) {
-    v += __shfl_xor_sync(0xffffffffu, v, 1);
-    v += __shfl_xor_sync(0xffffffffu, v, 4);
+// sum over the lanes of the lane's 2x2 block
+__device__ __forceinline__ float quad_sum(float v, int qbits) {
+    float t = __shfl_xor_sync(0xffffffffu, v, 1);
+    v += (qbits & 1) ? t : 0.f;
+    t = __shfl_xor_sync(0xffffffffu, v, 4);
+    v += (qbits & 4) ? t : 0.f;
     return v;
 }
 // cos(a, b) > tau from a.b, |a|^2, |b|^2 without a division; a zero vector has cosine 0
@@ -279,8 +329,8 @@ __device__ __forceinline__ bool cos_above(float dot, float na, float nb, float t
 
 struct ItemGeo {
     int item, b, tstart, n, halo, last_seg;
-    int y0, x0, cls;
-    uint32_t vmask;     // bit c: cell c of the tile lies inside the grid
+    int tile;           // index into FusedParams::tiles
+    uint32_t vmask;     // bit l: row l of the tile holds a cell
     int nvalid;
 };
 
@@ -298,18 +348,16 @@ __device__ __forceinline__ bool next_item(const FusedParams& p, int round, uint3
     const int seg = it.item % p.nseg;
     const int tb = it.item / p.nseg;
     it.b = tb % p.B;
-    const int tile = p.tile_order[tb / p.B];
+    it.tile = tb / p.B;
     const int t0 = seg * p.F, t1 = min(p.T, t0 + p.F);
     it.halo = t0 > 0;
     it.tstart = t0 - it.halo;
     it.n = t1 - it.tstart;
     it.last_seg = t1 == p.T;
-    it.y0 = (tile / p.Wt) * 4;
-    it.x0 = (tile % p.Wt) * 4;
-    const int rows = min(4, p.H - it.y0), cols = min(4, p.W - it.x0);
-    it.cls = (rows - 1) * 4 + (cols - 1);
-    it.vmask = (0xfu >> (4 - cols)) * (0x1111u >> (4 * (4 - rows)));
-    it.nvalid = rows * cols;
+    it.vmask = 0;
+    for (int l = 0; l < 16; l++)
+        if (p.tiles[it.tile].y[l] != 255) it.vmask |= 1u << l;
+    it.nvalid = __popc(it.vmask);
     return true;
 }
 
@@ -319,37 +367,44 @@ __device__ __forceinline__ bool next_item(const FusedParams& p, int round, uint3
 //   k=0  |x_c|^2                       k=1  x_c . parent(c)            k=2  x_c . top
 //   k=3  x_c(t) . x_c(t-1)             k=4  x_c(t) . parent(c)(t-1)    k=5  x_c(t) . top(t-1)
 //   k=6  parent(c)(t) . x_c(t-1)       k=7  top(t) . x_c(t-1)
-// Ring rows of cells outside the grid hold stale finite data: such columns are masked or
-// get weight 0 here, and the similarity warp drops the numbers of such cells.
-__device__ __forceinline__ float combine_sums(uint32_t G, int c, int k, uint32_t vmask, uint32_t W1s, uint32_t W2s) {
+// Ring rows without a cell hold stale finite data: such columns are masked here, and the
+// similarity warp drops the numbers of such rows.  W2s: the 16 lanes' weights w2 in shared memory.
+__device__ __forceinline__ float combine_sums(uint32_t G, int c, int k, const LaneGeo& g, uint32_t W2s) {
     const uint32_t Cm = G + 256 * 4;
-    const int qb = tile_anchor(c, 1);
-    const float m0 = (vmask >> qb) & 1u ? 1.f : 0.f, m1 = (vmask >> (qb + 1)) & 1u ? 1.f : 0.f;
-    const float m2 = (vmask >> (qb + 4)) & 1u ? 1.f : 0.f, m3 = (vmask >> (qb + 5)) & 1u ? 1.f : 0.f;
     float v = 0.f;
     if (k == 0) {
         v = lds_f32(G + (c * 16 + c) * 4);
     } else if (k == 3) {
         v = lds_f32(Cm + (c * 16 + c) * 4);
     } else if (k == 1 || k == 4 || k == 6) {
-        // the four cells of the 2x2 block: along the row of c (k = 1, 4) or down its column (k = 6)
+        // the (up to) four cells of the 2x2 block: along the row of c (k = 1, 4) or down its column (k = 6)
         const uint32_t M = k == 1 ? G : Cm;
+        const int qb = c & ~g.qbits;
         const int step = k == 6 ? 16 : 1;
         const uint32_t a = M + (k == 6 ? (qb * 16 + c) : (c * 16 + qb)) * 4;
+        const float m0 = (g.qmask >> qb) & 1u ? 1.f : 0.f, m1 = (g.qbits & 1) && ((g.qmask >> (qb + 1)) & 1u) ? 1.f : 0.f;
+        const float m2 = (g.qbits & 4) && ((g.qmask >> (qb + 4)) & 1u) ? 1.f : 0.f;
+        const float m3 = (g.qbits & 5) == 5 && ((g.qmask >> (qb + 5)) & 1u) ? 1.f : 0.f;
         const float x0 = lds_f32(a), x1 = lds_f32(a + step * 4), x2 = lds_f32(a + 4 * step * 4),
                     x3 = lds_f32(a + 5 * step * 4);
-        v = ((m0 * x0 + m1 * x1) + (m2 * x2 + m3 * x3)) * lds_f32(W1s + c * 4);
+        v = ((m0 * x0 + m1 * x1) + (m2 * x2 + m3 * x3)) * g.w1;
     } else {
-        // weighted sum over all 16 cells: along the row of c (k = 2, 5) or down its column (k = 7)
+        // weighted sum over the cells of the coarsest node: along the row of c (k = 2, 5) or down its column (k = 7)
         const uint32_t M = k == 2 ? G : Cm;
         if (k == 7) {
 #pragma unroll
-            for (int i = 0; i < 16; i++) v = fmaf(lds_f32(W2s + i * 4), lds_f32(M + (i * 16 + c) * 4), v);
+            for (int i = 0; i < 16; i++) {
+                const float w = (g.tmask >> i) & 1u ? lds_f32(W2s + i * 4) : 0.f;
+                v = fmaf(w, lds_f32(M + (i * 16 + c) * 4), v);
+            }
         } else {
 #pragma unroll
             for (int i = 0; i < 16; i += 4) {
                 const float4 w = lds_f32x4(W2s + i * 4), x = lds_f32x4(M + (c * 16 + i) * 4);
-                v = fmaf(w.x, x.x, v); v = fmaf(w.y, x.y, v); v = fmaf(w.z, x.z, v); v = fmaf(w.w, x.w, v);
+                v = fmaf((g.tmask >> i) & 1u ? w.x : 0.f, x.x, v);
+                v = fmaf((g.tmask >> (i + 1)) & 1u ? w.y : 0.f, x.y, v);
+                v = fmaf((g.tmask >> (i + 2)) & 1u ? w.z : 0.f, x.z, v);
+                v = fmaf((g.tmask >> (i + 3)) & 1u ? w.w : 0.f, x.w, v);
             }
         }
     }
@@ -389,7 +444,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     const uint32_t ring_base = smem_u32(ring);
     const int w_comb = p.NM, w_sum = p.NM + kCombineWarps, w_sim = w_sum + p.NA, w_chain = w_sim + 1, w_prod = w_sim + 2;
 
-    // set-up: barriers, a ring without NaN patterns, the pooling weights of all 16 tile shapes
+    // set-up: barriers, a ring without NaN patterns
     if (tid == 0) {
         for (int s = 0; s < p.R; s++) {
             mbar_init(full_bar + 8 * s, 1);
@@ -411,17 +466,6 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     }
     for (int k = tid * 16; k < p.R * p.slot_bytes; k += blockDim.x * 16)
         *reinterpret_cast<uint4*>(ring + k) = make_uint4(0u, 0u, 0u, 0u);
-    for (int i = tid; i < 256; i += blockDim.x) {
-        const int cls = i >> 4, c = i & 15;
-        const int rows = (cls >> 2) + 1, cols = (cls & 3) + 1;
-        const uint32_t vm = (0xfu >> (4 - cols)) * (0x1111u >> (4 * (4 - rows)));
-        const int nq = __popc(vm & quad_mask(c));
-        int quads = 0;
-        for (int qd = 0; qd < 4; qd++) quads += (vm & (0x33u << (8 * (qd >> 1) + 2 * (qd & 1)))) ? 1 : 0;
-        const float inv1 = nq ? 1.f / (float)nq : 0.f;
-        wtab[cls * 32 + c] = p.L >= 2 ? inv1 : 0.f;                                        // per 2x2 block
-        wtab[cls * 32 + 16 + c] = p.L == 3 && ((vm >> c) & 1u) ? inv1 * (1.f / (float)quads) : 0.f;
-    }
     __syncthreads();
     cluster_arrive();
     cluster_wait();         // every CTA of the cluster has its barriers before anyone signals them
@@ -519,7 +563,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         }
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
-            const uint32_t W1s = smem_u32(wtab + it.cls * 32), W2s = W1s + 64;
+            // this thread's cell and the weights of all 16 lanes for the sums over the coarsest node
+            const LaneGeo lg = lane_geo(p.tiles[it.tile], ctid & 15, p.L, p.W);
+            const uint32_t W2s = smem_u32(wtab);
+            named_sync(1, nthr);                       // the previous item's weights are not read any more
+            if (ctid < 16) wtab[ctid] = lg.w2;
+            named_sync(1, nthr);
             for (int j = 0; j < it.n; j++, q++) {
                 // the first combine warp waits; the named barriers hand the outcome to the others
                 if (warp == w_comb) mbar_wait(gfull_bar, q, timed_out);
@@ -540,7 +589,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (warp == w_comb && q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
                 if (named_sync_or(2, nthr, timed_out)) { timed_out = true; break; }
                 {
-                    const float sum = combine_sums(redsum_a, ctid & 15, ctid >> 4, it.vmask, W1s, W2s);
+                    const float sum = combine_sums(redsum_a, ctid & 15, ctid >> 4, lg, W2s);
                     const uint32_t xo = xb * p.C * kSumVals * 4, bo = 8 * xb;
 #pragma unroll
                     for (int r = 0; r < kMaxCluster; r++)
@@ -643,13 +692,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const int c = lane & 15, half = lane >> 4;
         const int L = p.L;
         const uint32_t xchg_a = smem_u32(xchg);
-        const uint32_t qm = quad_mask(c);
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             const float tau_s = taus.s[it.b], tau_t = taus.t[it.b];
-            const float w1 = wtab[it.cls * 32 + c], w2 = wtab[it.cls * 32 + 16 + c];
-            const bool valid = (it.vmask >> c) & 1u;
-            const bool quad_exists = (it.vmask & qm) != 0;
+            const LaneGeo lg = lane_geo(p.tiles[it.tile], c, L, p.W);
+            const float w1 = lg.w1, w2 = lg.w2;
+            const bool valid = lg.valid;
             int carry_lv = 0;               // cover level / squared norm of the node covering cell c in the
             float carry_nk = 0.f;           // last frame of the previous pass
             for (int j = 0; j < it.n; j += 2) {
@@ -682,18 +730,18 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
 
                 // Section 3.2: cosine of every node with its parent, then the coarse-to-fine search
                 const float n0 = v[0], d0 = v[1], rr = v[2];
-                const float n1 = w1 * quad_sum(d0);              // |parent|^2
-                const float d1 = w1 * quad_sum(rr);              // parent . top
-                const float n2 = half_warp_sum(w2 * rr);         // |top|^2
+                const float n1 = w1 * quad_sum(d0, lg.qbits);    // |parent|^2
+                const float d1 = w1 * quad_sum(rr, lg.qbits);    // parent . top
+                const float n2 = top_sum(w2 * rr, lg.tbits);     // |top|^2
                 int lv = 0;
                 if (L >= 2) {
                     const bool p0 = !valid || cos_above(d0, n0, n1, tau_s);
                     const uint32_t pm0 = (__ballot_sync(full, p0) >> (16 * half)) & 0xffffu;
-                    const bool quad_pass = (pm0 & qm) == qm;
+                    const bool quad_pass = (pm0 & lg.qmask) == lg.qmask;
                     if (L == 3) {
-                        const bool p1 = !quad_exists || cos_above(d1, n1, n2, tau_s);
+                        const bool p1 = !valid || cos_above(d1, n1, n2, tau_s);
                         const uint32_t pm1 = (__ballot_sync(full, p1) >> (16 * half)) & 0xffffu;
-                        lv = pm1 == 0xffffu ? 2 : (quad_pass ? 1 : 0);
+                        lv = (pm1 & lg.tmask) == lg.tmask ? 2 : (quad_pass ? 1 : 0);
                     } else {
                         lv = quad_pass ? 1 : 0;
                     }
@@ -709,20 +757,20 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const float pnk = half ? nk_lo : carry_nk;
                 int link_local = -1;
                 {
-                    const float t11 = w1 * quad_sum(v[4]), t12 = w1 * quad_sum(v[5]);
-                    const float t21 = w1 * quad_sum(v[7]), t22 = half_warp_sum(w2 * v[5]);
+                    const float t11 = w1 * quad_sum(v[4], lg.qbits), t12 = w1 * quad_sum(v[5], lg.qbits);
+                    const float t21 = w1 * quad_sum(v[7], lg.qbits), t22 = top_sum(w2 * v[5], lg.tbits);
                     float dot;
                     if (lv == 0) dot = lu == 0 ? v[3] : (lu == 1 ? v[4] : v[5]);
                     else if (lv == 1) dot = lu == 0 ? v[6] : (lu == 1 ? t11 : t12);
                     else dot = lu == 0 ? v[7] : (lu == 1 ? t21 : t22);
                     const bool has_prev = j + half > 0;
-                    const bool rep = valid && has_prev && tile_anchor(c, min(lv, lu)) == c;
+                    const bool rep = valid && has_prev && lane_anchor(lg, c, min(lv, lu)) == c;
                     const bool pass = rep && cos_above(dot, nk, pnk, tau_t);
                     const uint32_t passm = (__ballot_sync(full, pass) >> (16 * half)) & 0xffffu;
-                    const uint32_t cand = passm & region_mask(c, lv);
+                    const uint32_t cand = passm & lane_region(lg, c, lv);
                     const int cstar = cand ? __ffs(cand) - 1 : 0;     // first in row-major order: the top-left one
                     const int lu_star = __shfl_sync(full, lu, 16 * half + cstar);
-                    link_local = cand ? tile_anchor(cstar, lu_star) : -1;
+                    link_local = cand ? lane_anchor(lg, cstar, lu_star) : -1;      // same sub-tile: same bits
                 }
                 carry_lv = two ? lv_hi : lv_lo;
                 carry_nk = two ? nk_hi : nk_lo;
@@ -752,8 +800,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         uint32_t carry_mask = 0;
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
-            const bool valid = (it.vmask >> c) & 1u;
-            const float w1 = wtab[it.cls * 32 + c], w2 = wtab[it.cls * 32 + 16 + c];
+            const LaneGeo lg = lane_geo(p.tiles[it.tile], c, p.L, p.W);
+            const bool valid = lg.valid;
+            const float w1 = lg.w1, w2 = lg.w2;
             if (rank == 0) p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
             int prev_slot = 0;
             uint32_t active_slots = 0;
@@ -774,7 +823,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
 
                 // nodes with a link join the chain of their target; chains without a member in this
                 // frame have ended; the remaining nodes start new chains in free slots
-                const bool anchor = valid && tile_anchor(c, lv) == c;
+                const bool anchor = valid && lane_anchor(lg, c, lv) == c;
                 const bool linked = anchor && link_local >= 0;
                 const bool fresh = anchor && link_local < 0;
                 const int slot_linked = __shfl_sync(full, prev_slot, link_local < 0 ? 0 : link_local);
@@ -784,11 +833,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const uint32_t freshm = __ballot_sync(full, fresh && low);
                 const int slot_fresh = kth_set_bit16(freem, __popc(freshm & ((1u << c) - 1)));
                 const int node_slot = linked ? slot_linked : slot_fresh;
-                const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + tile_anchor(c, lv));
-                const uint32_t cells = it.vmask & region_mask(c, lv);
+                const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + lane_anchor(lg, c, lv));
+                const uint32_t cells = lane_region(lg, c, lv);
                 const int wint = p.weight_mode ? __popc(cells) : 1;
-                const long long gc =
-                    (long long)it.b * p.N + (long long)t * p.HW + (it.y0 + (c >> 2)) * p.W + it.x0 + (c & 3);
+                const long long gc = (long long)it.b * p.N + (long long)t * p.HW + lg.cell;
+                const int link_cell = __shfl_sync(full, lg.cell, link_local < 0 ? 0 : link_local);
 
                 // chains that ended: lane s looks at slot s (before the slot is given away again); at
                 // the first frame of an item nothing of the item runs yet and the list is the carry
@@ -816,7 +865,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (low && linked) atomicAdd(&tab->weight[slot_linked], wint);
                 // the frame's weight matrix: row = chain slot, column = cell
                 reinterpret_cast<uint4*>(rec->wmat)[lane] = make_uint4(0u, 0u, 0u, 0u);
-                const int wnode = __shfl_sync(full, wint, (lane & 16) + tile_anchor(c, lv));
+                const int wnode = __shfl_sync(full, wint, (lane & 16) + lane_anchor(lg, c, lv));
                 __syncwarp();
                 if (low && valid && !is_halo) {
                     const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
@@ -827,9 +876,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
 
                 if (rank == 0 && !is_halo && low && valid) {
                     p.cover[gc] = (int8_t)lv;
-                    p.link[gc] = link_local < 0 ? -1
-                                                : (t - 1) * p.HW + (it.y0 + (link_local >> 2)) * p.W + it.x0 +
-                                                      (link_local & 3);
+                    p.link[gc] = link_local < 0 ? -1 : (t - 1) * p.HW + link_cell;
                     p.chain_key[gc] = tab->key[cur_slot] - it.b * p.N;
                 }
                 if (is_last) {
@@ -879,7 +926,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 __syncwarp();
                 if (lane < 16 && ((it.vmask >> lane) & 1u)) {
                     const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
-                                           (it.y0 + (lane >> 2)) * p.W + it.x0 + (lane & 3);
+                                           p.tiles[it.tile].y[lane] * p.W + p.tiles[it.tile].x[lane];
                     bulk_g2s(ring_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
                              (uint32_t)(p.S * 2), bar);
                 }

@@ -14,9 +14,10 @@ from tests import helpers
 pytestmark = pytest.mark.gpu
 
 # (path, cluster size, frames per item) for sttm_set_tuning: the library's own choice, the
-# three-pass kernels, and fused launches that force clusters and many item borders
+# three-pass kernels, fused launches that force clusters and many item borders, and the fused
+# kernel without packing of partial border tiles
 TUNINGS = {"auto": (0, 0, 0), "threepass": (1, 0, 0), "c1f3": (2, 1, 3), "c2f2": (2, 2, 2), "c4f5": (2, 4, 5),
-           "c8f1": (2, 8, 1)}
+           "c8f1": (2, 8, 1), "nopack": (3, 0, 0)}
 
 
 @pytest.fixture(params=list(TUNINGS), ids=list(TUNINGS))

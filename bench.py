@@ -169,7 +169,10 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    binding.load_library().sttm_set_tuning(*[int(v) for v in args.tuning.split(",")])
+    tuning = [int(v) for v in args.tuning.split(",")]
+    binding.load_library().sttm_set_tuning(*tuning[:3])
+    if len(tuning) > 3:
+        binding.load_library().sttm_set_ring_split(*(tuning[3:5] + [0])[:2])
 
     cfg, spec, th, key = workload_setup(args.workload)
     N = spec.tokens
@@ -300,7 +303,8 @@ def main():
                     help="frames per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tuning", default="0,0,0",
-                    help="path,cluster_size,frames_per_item for sttm_set_tuning (0 = library's choice)")
+                    help="path,cluster_size,frames_per_item for sttm_set_tuning, optionally followed by "
+                         "sum_slots,lead_frames for sttm_set_ring_split (0 = library's choice)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

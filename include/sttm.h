@@ -196,14 +196,26 @@ void sttm_set_stage_events(void** events);
  */
 void sttm_set_tuning(int path, int cluster_size, int frames_per_item);
 
+/*
+ * Second benchmark knob of the fused kernel.  The kernel reads every frame from HBM once for
+ * the similarity products and, because the frame would otherwise sit in shared memory until
+ * its merge decisions exist, a second time (an L2 hit) for the chain sums.
+ *   sum_slots    shared-memory slots of the second ring (the rest go to the first); 0: default
+ *   lead_frames  the second copy of frame q starts once the similarity warp has finished frame
+ *                q - lead_frames; 0: right after the frame's own decisions
+ * Not thread safe; affects later calls of every entry point.
+ */
+void sttm_set_ring_split(int sum_slots, int lead_frames);
+
 /* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 fused. */
 int sttm_last_path(void);
 
 /*
  * Launch shape the fused kernel would get for these params (host pointers; queries the
- * current device for the number of clusters that fit).  shape[10] = {cluster size, channels
- * per CTA, threads per CTA, ring slots, dynamic shared memory bytes, frames per item, items,
- * clusters that can be resident, clusters launched, tensor-core (Gram) warps}.  Returns 1, or 0
+ * current device for the number of clusters that fit).  shape[12] = {cluster size, channels
+ * per CTA, threads per CTA, slots of the first ring, dynamic shared memory bytes, frames per
+ * item, items, clusters that can be resident, clusters launched, tensor-core (Gram) warps,
+ * slots of the second ring, lead_frames}.  Returns 1, or 0
  * when the fused kernel does not apply to the params.
  */
 int sttm_fused_launch_shape(const sttm_params* p, int* shape);

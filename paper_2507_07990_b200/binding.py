@@ -25,7 +25,7 @@ STATUS_NAMES = ["ok", "bad argument", "unsupported shape", "workspace too small"
 EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame", "sttm_spatial",
            "sttm_temporal", "sttm_merge_ex", "sttm_merge", "sttm_merge_host", "sttm_release_cache",
            "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
-           "sttm_set_stage_events", "sttm_set_tuning", "sttm_last_path",
+           "sttm_set_stage_events", "sttm_set_tuning", "sttm_set_ring_split", "sttm_last_path",
            "sttm_fused_launch_shape", "sttm_spatial_static"]
 
 
@@ -87,6 +87,8 @@ def load_library(path: Optional[str] = None):
     lib.sttm_set_stage_events.restype = None
     lib.sttm_set_tuning.argtypes = [C.c_int, C.c_int, C.c_int]
     lib.sttm_set_tuning.restype = None
+    lib.sttm_set_ring_split.argtypes = [C.c_int, C.c_int]
+    lib.sttm_set_ring_split.restype = None
     lib.sttm_last_path.argtypes = []
     lib.sttm_last_path.restype = C.c_int
     lib.sttm_fused_launch_shape.argtypes = [pp, C.POINTER(C.c_int)]
@@ -157,11 +159,11 @@ def sttm_workspace_bytes(problem: Problem) -> int:
 
 def sttm_fused_launch_shape(problem: Problem) -> Optional[dict]:
     """Launch shape of the fused kernel for a problem, or None when it does not apply."""
-    arr = (C.c_int * 10)()
+    arr = (C.c_int * 12)()
     if not load_library().sttm_fused_launch_shape(C.byref(problem.params), arr):
         return None
     names = ["cluster_size", "channels_per_cta", "threads", "ring_slots", "smem_bytes", "frames_per_item", "items",
-             "resident_clusters", "clusters", "mma_warps"]
+             "resident_clusters", "clusters", "mma_warps", "sum_ring_slots", "lead_frames"]
     return dict(zip(names, list(arr)))
 
 

@@ -37,7 +37,7 @@ inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 // Launch shape of the fused kernel for one problem; ok == false: the three-pass kernels run.
 struct FusedPlan {
     bool ok;
-    int C, S, NM, NA, R, row_bytes, slot_bytes, F, nseg, nitems, ntiles, Wt;
+    int C, S, NM, NA, R, RB, lead, row_bytes, slot_bytes, F, nseg, nitems, ntiles, Wt;
     size_t smem;
     TileDesc tiles[kMaxTiles];      // most cells first
 };
@@ -55,7 +55,7 @@ struct Plan {
 };
 
 // benchmark / test knobs (sttm_set_tuning): 0 = choose automatically
-int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0, g_tune_pack = 0;
+int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0, g_tune_pack = 0, g_tune_sum_slots = 0, g_tune_lead = 0;
 
 constexpr size_t kMaxSmem = 232448;   // 227 KB per CTA on sm_100
 
@@ -136,13 +136,19 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
     f->slot_bytes = 16 * f->row_bytes;
     const size_t fixed = (size_t)f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
-                         16 * 32 * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) +
-                         (2 * kMaxRing + 6 * kRecRing + 4) * 8;
-    int R = (int)((kMaxSmem - fixed) / f->slot_bytes);
-    R = std::min(R, kMaxRing);
-    if (R < 4) return;
-    f->R = R;
-    f->smem = (size_t)R * f->slot_bytes + fixed;
+                         16 * 32 * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) + 16 +
+                         (4 * kMaxRing + 6 * kRecRing + 4) * 8;
+    // the slots that fit, shared out between the Gram warps' ring (a frame stays for its own
+    // products and the next frame's, plus the time its copy takes to arrive) and the sum
+    // warps' ring (filled from L2 shortly before use)
+    const int slots = std::min((int)((kMaxSmem - fixed) / f->slot_bytes), 2 * kMaxRing);
+    if (slots < 5) return;
+    int RB = g_tune_sum_slots > 0 ? g_tune_sum_slots : (slots * 3 + 3) / 7;
+    RB = std::max(2, std::min(RB, std::min(slots - 3, kMaxRing)));
+    f->RB = RB;
+    f->R = std::min(slots - RB, kMaxRing);
+    f->lead = std::max(0, g_tune_lead);
+    f->smem = (size_t)(f->R + f->RB) * f->slot_bytes + fixed;
     // frames per item: about four items per resident cluster, with the number of items as close
     // below a multiple of the cluster count as the frame count allows (the items are dealt out
     // statically, and every item of a cluster costs about the same)
@@ -353,7 +359,7 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
 int fused_resident_clusters(const FusedPlan& f) {
     static int cached[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
     static size_t cached_smem[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
-    const int warps = f.NM + kCombineWarps + f.NA + 3;
+    const int warps = f.NM + kCombineWarps + f.NA + kTailWarps;
     int& slot = cached[f.C][warps];
     if (slot > 0 && cached_smem[f.C][warps] == f.smem) return slot;
     int n = 0;
@@ -390,7 +396,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.HW = g.HW; fp.N = g.N;
     fp.Wt = f.Wt; fp.ntiles = f.ntiles;
     fp.C = f.C; fp.S = f.S; fp.NM = f.NM; fp.NA = f.NA;
-    fp.row_bytes = f.row_bytes; fp.slot_bytes = f.slot_bytes; fp.R = f.R;
+    fp.row_bytes = f.row_bytes; fp.slot_bytes = f.slot_bytes; fp.R = f.R; fp.RB = f.RB; fp.lead = f.lead;
     fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
     fp.weight_mode = (int)p->wt;
     fp.out_f32 = p->out_dtype == STTM_F32;
@@ -408,7 +414,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     const int nclusters = std::min(f.nitems, fused_resident_clusters(f));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nclusters * f.C);
-    cfg.blockDim = dim3((f.NM + kCombineWarps + f.NA + 3) * 32);
+    cfg.blockDim = dim3((f.NM + kCombineWarps + f.NA + kTailWarps) * 32);
     cfg.dynamicSmemBytes = f.smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -529,8 +535,8 @@ int sttm_fused_launch_shape(const sttm_params* p, int* shape) {
     if (shape == nullptr || make_plan(p, &pl) != STTM_OK || !pl.f.ok) return 0;
     const FusedPlan& f = pl.f;
     const int resident = fused_resident_clusters(f);
-    const int v[10] = {f.C, f.S, (f.NM + kCombineWarps + f.NA + 3) * 32, f.R, (int)f.smem, f.F, f.nitems, resident,
-                       std::min(f.nitems, resident), f.NM};
+    const int v[12] = {f.C, f.S, (f.NM + kCombineWarps + f.NA + kTailWarps) * 32, f.R, (int)f.smem, f.F, f.nitems, resident,
+                       std::min(f.nitems, resident), f.NM, f.RB, f.lead};
     std::memcpy(shape, v, sizeof(v));
     return 1;
 }
@@ -542,6 +548,11 @@ void sttm_set_tuning(int path, int cluster_size, int frames_per_item) {
     g_tune_pack = path == 3 ? 1 : 0;
     g_tune_cluster = cluster_size;
     g_tune_seg = frames_per_item;
+}
+
+void sttm_set_ring_split(int sum_slots, int lead_frames) {
+    g_tune_sum_slots = sum_slots;
+    g_tune_lead = lead_frames;
 }
 
 sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,

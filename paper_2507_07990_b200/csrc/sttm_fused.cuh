@@ -50,20 +50,22 @@ constexpr int kMaxRing = 12;
 constexpr int kMaxGramWarps = 4;
 constexpr int kCombineWarps = 4;
 constexpr int kMaxSumWarps = 8;         // 128 channels each: at most 1024 channels per CTA
-constexpr int kFusedMaxThreads = (kMaxGramWarps + kCombineWarps + kMaxSumWarps + 3) * 32;
+constexpr int kTailWarps = 4;           // similarity, chain, two producers
+constexpr int kFusedMaxThreads = (kMaxGramWarps + kCombineWarps + kMaxSumWarps + kTailWarps) * 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after two seconds
 constexpr uint32_t kWaitHintNs = 100000u;    // one try may sleep this long before it reports "not yet"
 
 enum : int { kStatusWaitTimeout = 1 << 6 };
 
 struct FlushCmd { int slot, kind, dst; float weight; };     // kind 0: finished row, 1: piece
-// Commands of one frame for the sum warps: first write out and clear the listed chain sums
-// (chains that got no member in this frame; at the first frame of an item: everything the
-// previous item left), then add W X to the running sums, W[slot][cell] (bf16; the weights
+// Commands of one frame for the sum warps: first write out and clear the chain sums of the
+// slots in flush_mask, flush[s] saying where slot s goes (chains that got no member in this
+// frame; at the first frame of an item: everything the previous item left; all of them are
+// written in one go, each slot by the lanes that hold it), then add W X to the running sums, W[slot][cell] (bf16; the weights
 // are small integers times powers of two, hence exact) = weight of the cell in its kept node
 // if that node belongs to the chain in `slot`, else 0.
 struct FrameRec {
-    int n_flush, pad0, pad1, pad2;
+    uint32_t flush_mask, pad0, pad1, pad2;
     FlushCmd flush[16];
     uint16_t wmat[256];
 };
@@ -82,7 +84,8 @@ struct FusedParams {
     int HW, N;
     int Wt, ntiles;
     int C, S, NM, NA;        // cluster size, channels per CTA, Gram warps, sum warps
-    int row_bytes, slot_bytes, R;
+    int row_bytes, slot_bytes;
+    int R, RB, lead;         // slots of the Gram warps' ring and of the sum warps' ring; see the second producer
     int F, nseg, nitems;
     int weight_mode, out_f32;
     int8_t* cover;
@@ -145,6 +148,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, int use, bool& timed_out
             timed_out = true;
             return false;
         }
+    }
+    return true;
+}
+// waits until a progress counter in shared memory (written by another warp of the CTA; only
+// a timing hint, no data hangs on it) has reached `target`; time-bounded like mbar_wait
+__device__ __forceinline__ bool hint_wait(const int* counter, int target, bool& timed_out) {
+    if (timed_out) return false;
+    const volatile int* c = counter;
+    if (*c >= target) return true;
+    const unsigned long long t0 = global_timer_ns();
+    while (*c < target) {
+        __nanosleep(64);
+        if (global_timer_ns() - t0 > kWaitLimitNs) { timed_out = true; return false; }
     }
     return true;
 }
@@ -417,13 +433,13 @@ struct SlotTable {
 };
 
 // ---------------------------------------------------------------------------------
-// The kernel.  Warps: [0, NM) Gram, [NM, NM+NA) sum, then similarity, chain, producer.
+// The kernel.  Warps: [0, NM) Gram, then 4 combine, NA sum, similarity, chain, two producers.
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kFusedMaxThreads, 1)
 k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* ring = smem;
-    size_t off = (size_t)p.R * p.slot_bytes;
+    size_t off = (size_t)(p.R + p.RB) * p.slot_bytes;
     float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)p.NM * kGramVals * 4;
     float* redsum = reinterpret_cast<float*>(smem + off);    off += kGramVals * 4;
     float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * p.C * kSumVals * 4;
@@ -431,25 +447,32 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     int* hand = reinterpret_cast<int*>(smem + off);          off += kRecRing * 16 * 4;
     SlotTable* tab = reinterpret_cast<SlotTable*>(smem + off); off += sizeof(SlotTable);
     FrameRec* recs = reinterpret_cast<FrameRec*>(smem + off); off += kRecRing * sizeof(FrameRec);
+    int* hint = reinterpret_cast<int*>(smem + off);          off += 16;               // frames the similarity warp has finished
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + off);
     const uint32_t bar0 = smem_u32(bars);
     const uint32_t full_bar = bar0, empty_bar = bar0 + 8 * kMaxRing;
-    const uint32_t xfull_bar = bar0 + 16 * kMaxRing, xempty_bar = xfull_bar + 8 * kRecRing;
+    const uint32_t fullb_bar = bar0 + 16 * kMaxRing, emptyb_bar = bar0 + 24 * kMaxRing;
+    const uint32_t xfull_bar = bar0 + 32 * kMaxRing, xempty_bar = xfull_bar + 8 * kRecRing;
     const uint32_t hfull_bar = xempty_bar + 8 * kRecRing, hempty_bar = hfull_bar + 8 * kRecRing;
     const uint32_t rfull_bar = hempty_bar + 8 * kRecRing, rempty_bar = rfull_bar + 8 * kRecRing;
     const uint32_t gfull_bar = rempty_bar + 8 * kRecRing, gempty_bar = gfull_bar + 16;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank(), cid = cluster_id(), ncl = cluster_count();
-    const uint32_t ring_base = smem_u32(ring);
+    const uint32_t ring_base = smem_u32(ring), ringb_base = ring_base + p.R * p.slot_bytes;
     const int w_comb = p.NM, w_sum = p.NM + kCombineWarps, w_sim = w_sum + p.NA, w_chain = w_sim + 1, w_prod = w_sim + 2;
 
     // set-up: barriers, a ring without NaN patterns
     if (tid == 0) {
         for (int s = 0; s < p.R; s++) {
             mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, p.NM + p.NA);
+            mbar_init(empty_bar + 8 * s, p.NM);
         }
+        for (int s = 0; s < p.RB; s++) {
+            mbar_init(fullb_bar + 8 * s, 1);
+            mbar_init(emptyb_bar + 8 * s, p.NA);
+        }
+        *hint = 0;
         for (int s = 0; s < kRecRing; s++) {
             mbar_init(xfull_bar + 8 * s, 1);
             mbar_init(xempty_bar + 8 * s, p.C);
@@ -464,7 +487,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int k = tid * 16; k < p.R * p.slot_bytes; k += blockDim.x * 16)
+    for (int k = tid * 16; k < (p.R + p.RB) * p.slot_bytes; k += blockDim.x * 16)
         *reinterpret_cast<uint4*>(ring + k) = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     cluster_arrive();
@@ -625,19 +648,21 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         for (; q <= total; q++) {
             const int rk = q % kRecRing;
             if (!mbar_wait(rfull_bar + 8 * rk, q / kRecRing, timed_out)) break;
-            if (q < total && !mbar_wait(full_bar + 8 * s, use, timed_out)) break;
+            if (q < total && !mbar_wait(fullb_bar + 8 * s, use, timed_out)) break;
             __syncwarp();
             const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
-            const int n_flush = (int)lds_u32x4(rec).x;
+            const uint32_t flush_mask = lds_u32x4(rec).x;
+            // Slots g and g + 8 live in the four lanes of group g: all slots of one half of the
+            // fragment are written in the same pass, every group following its own command.  One
+            // loop per kind of destination and per half keeps register indices and offsets static.
 #pragma unroll 1
-            for (int i = 0; i < n_flush; i++) {
-                const uint4 fc = lds_u32x4(rec + 16 + i * 16);       // slot, kind, dst, weight
-                const int slot = (int)fc.x;
-                const bool hi = slot >= 8;
-                const float inv = fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
+            for (int hi = 0; hi < 2; hi++) {
+                const uint32_t m8 = (flush_mask >> (8 * hi)) & 0xffu;
+                if (m8 == 0) continue;
+                const bool mine = (m8 >> g) & 1u;
+                const uint4 fc = lds_u32x4(rec + 16 + (g + 8 * hi) * 16);       // slot, kind, dst, weight
+                const float inv = mine && fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
                 const long long row = (long long)(int)fc.z * p.D + chan;
-                // only the four lanes that hold the slot's rows work; one loop per kind of destination
-                // and per half of the fragment keeps every register index and store offset static
 #define STTM_FLUSH_LOOP(I0, I1, STORE)                                        \
     _Pragma("unroll") for (int nt = 0; nt < 16; nt++) {                       \
         const float x = sums[nt][I0] * inv, y = sums[nt][I1] * inv;           \
@@ -656,7 +681,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.staging) + row;                               \
         STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<uint32_t*>(dst + nt * 8) = pack_bf16x2(x, y))               \
     }
-                if (g == (slot & 7)) {
+                if (mine) {
                     if (hi) { STTM_FLUSH_KINDS(2, 3) } else { STTM_FLUSH_KINDS(0, 1) }
                 }
 #undef STTM_FLUSH_KINDS
@@ -666,7 +691,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             if (q < total) {
                 uint32_t wa[4];
                 ldmatrix_x4(rec + woff, wa);
-                const uint32_t xb = ring_base + s * p.slot_bytes + xoff;
+                const uint32_t xb = ringb_base + s * p.slot_bytes + xoff;
 #pragma unroll
                 for (int pr = 0; pr < 8; pr++) {
                     if (ch0 + pr * 16 < p.S) {
@@ -680,9 +705,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(rempty_bar + 8 * rk);
-                if (q < total) mbar_arrive(empty_bar + 8 * s);
+                if (q < total) mbar_arrive(emptyb_bar + 8 * s);
             }
-            if (++s == p.R) { s = 0; use++; }
+            if (++s == p.RB) { s = 0; use++; }
         }
     } else if (warp == w_sim) {
         // --------------------------------- similarity warp ---------------------------------
@@ -788,6 +813,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     if (two) mbar_arrive(hfull_bar + 8 * ((q + 1) % kRecRing));
                 }
                 q += two ? 2 : 1;
+                if (lane == 0) *reinterpret_cast<volatile int*>(hint) = q;
             }
         }
     } else if (warp == w_chain) {
@@ -842,18 +868,17 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 // chains that ended: lane s looks at slot s (before the slot is given away again); at
                 // the first frame of an item nothing of the item runs yet and the list is the carry
                 if (low && ((dead >> lane) & 1u)) {
-                    const int at = __popc(dead & ((1u << lane) - 1));
                     if (tab->virt[lane]) {
                         const int pc = it.item * kPieceSlots + tab->cell[lane];
-                        rec->flush[at] = FlushCmd{lane, 1, pc, 0.f};
+                        rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
                         if (rank == 0) p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
                     } else {
-                        rec->flush[at] = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
+                        rec->flush[lane] = FlushCmd{lane, 0, tab->key[lane], (float)tab->weight[lane]};
                     }
                 }
-                if (low && ((carry_mask >> lane) & 1u))
-                    rec->flush[__popc(dead) + __popc(carry_mask & ((1u << lane) - 1))] = carry;
-                const int n_flush = __popc(dead) + __popc(carry_mask);
+                // (nothing of the item runs at its first frame: dead and the carry never meet)
+                if (low && ((carry_mask >> lane) & 1u)) rec->flush[lane] = carry;
+                const uint32_t flush_mask = dead | carry_mask;
                 carry_mask = 0;
                 __syncwarp();
                 if (low && fresh) {
@@ -892,9 +917,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                         }
                     }
                 }
-                if (lane == 0) {
-                    rec->n_flush = n_flush;
-                }
+                if (lane == 0) rec->flush_mask = flush_mask;
                 active_slots = is_last ? 0u : active;
                 prev_slot = cur_slot;
                 __syncwarp();
@@ -906,10 +929,8 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             const int hb = q % kRecRing;
             __syncwarp();
             FrameRec* rec = recs + hb;
-            if (low && ((carry_mask >> lane) & 1u)) rec->flush[__popc(carry_mask & ((1u << lane) - 1))] = carry;
-            if (lane == 0) {
-                rec->n_flush = __popc(carry_mask);
-            }
+            if (low && ((carry_mask >> lane) & 1u)) rec->flush[lane] = carry;
+            if (lane == 0) rec->flush_mask = carry_mask;
             __syncwarp();
             if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
         }
@@ -938,6 +959,37 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         for (int qq = max(0, q - p.R); qq < q; qq++) {
             bool late = false;
             mbar_wait(full_bar + 8 * (qq % p.R), qq / p.R, late);
+            timed_out |= late;
+        }
+    } else if (warp == w_prod + 1) {
+        // ---------------------------------- second producer ----------------------------------
+        // The sum warps need a frame only once its record exists, long after the Gram warps are
+        // done with it.  Holding the frame in shared memory all that time would let too few frames
+        // be in flight, so it is fetched a second time (from L2, where the first copy left it) into
+        // a ring of its own, timed by the similarity warp's progress so that it lands about when
+        // the chain warp posts the record.
+        int s = 0, use = 0;
+        for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
+            if (skip) continue;
+            for (int j = 0; j < it.n; j++, q++) {
+                const uint32_t bar = fullb_bar + 8 * s;
+                if (!hint_wait(hint, q + 1 - p.lead, timed_out)) break;
+                if (use >= 1 && !mbar_wait(emptyb_bar + 8 * s, use - 1, timed_out)) break;
+                __syncwarp();
+                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
+                __syncwarp();
+                if (lane < 16 && ((it.vmask >> lane) & 1u)) {
+                    const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
+                                           p.tiles[it.tile].y[lane] * p.W + p.tiles[it.tile].x[lane];
+                    bulk_g2s(ringb_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
+                             (uint32_t)(p.S * 2), bar);
+                }
+                if (++s == p.RB) { s = 0; use++; }
+            }
+        }
+        for (int qq = max(0, q - p.RB); qq < q; qq++) {
+            bool late = false;
+            mbar_wait(fullb_bar + 8 * (qq % p.RB), qq / p.RB, late);
             timed_out |= late;
         }
     }

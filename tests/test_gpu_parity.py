@@ -13,18 +13,23 @@ from tests import helpers
 
 pytestmark = pytest.mark.gpu
 
-# (path, cluster size, frames per item) for sttm_set_tuning: the library's own choice, the
-# three-pass kernels, fused launches that force clusters and many item borders, and the fused
-# kernel without packing of partial border tiles
-TUNINGS = {"auto": (0, 0, 0), "threepass": (1, 0, 0), "c1f3": (2, 1, 3), "c2f2": (2, 2, 2), "c4f5": (2, 4, 5),
-           "c8f1": (2, 8, 1), "nopack": (3, 0, 0)}
+# (path, cluster size, frames per item) for sttm_set_tuning, then (sum slots, lead frames) for
+# sttm_set_ring_split: the library's own choice, the three-pass kernels, fused launches that
+# force clusters and many item borders, the fused kernel without packing of partial border
+# tiles, and two other ways to share out the shared-memory slots
+TUNINGS = {"auto": (0, 0, 0, 0, 0), "threepass": (1, 0, 0, 0, 0), "c1f3": (2, 1, 3, 0, 0), "c2f2": (2, 2, 2, 0, 0),
+           "c4f5": (2, 4, 5, 0, 0), "c8f1": (2, 8, 1, 0, 0), "nopack": (3, 0, 0, 0, 0), "sum2lead2": (2, 0, 0, 2, 2),
+           "sum4": (2, 0, 7, 4, 1)}
 
 
 @pytest.fixture(params=list(TUNINGS), ids=list(TUNINGS))
 def tuning(request):
-    binding.load_library().sttm_set_tuning(*TUNINGS[request.param])
+    lib = binding.load_library()
+    lib.sttm_set_tuning(*TUNINGS[request.param][:3])
+    lib.sttm_set_ring_split(*TUNINGS[request.param][3:])
     yield request.param
-    binding.load_library().sttm_set_tuning(0, 0, 0)
+    lib.sttm_set_tuning(0, 0, 0)
+    lib.sttm_set_ring_split(0, 0)
 
 
 def run_and_compare(video_np, tau_s, tau_t, lv1=4, out_dtype=torch.float32, wt=binding.W_NODE,

@@ -197,10 +197,12 @@ void sttm_set_stage_events(void** events);
 void sttm_set_tuning(int path, int cluster_size, int frames_per_item);
 
 /*
- * Second benchmark knob of the fused kernel.  The kernel reads every frame from HBM once for
- * the similarity products and, because the frame would otherwise sit in shared memory until
- * its merge decisions exist, a second time (an L2 hit) for the chain sums.
- *   sum_slots    shared-memory slots of the second ring (the rest go to the first); 0: default
+ * Second benchmark knob of the fused kernel.  By default a frame stays in the kernel's
+ * shared-memory ring from its one read from HBM until its merge decisions exist and the chain
+ * sums have used it.  With sum_slots > 0 the ring is split: the frame leaves the first ring
+ * after the similarity products and is read a second time (an L2 hit) into a second ring of
+ * sum_slots slots for the chain sums, which lets more frames be in flight.
+ *   sum_slots    slots of the second ring (at least 2; the rest go to the first); 0: one ring
  *   lead_frames  the second copy of frame q starts once the similarity warp has finished frame
  *                q - lead_frames; 0: right after the frame's own decisions
  * Not thread safe; affects later calls of every entry point.

@@ -138,13 +138,13 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     const size_t fixed = (size_t)f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
                          16 * 32 * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) + 16 +
                          (4 * kMaxRing + 6 * kRecRing + 4) * 8;
-    // the slots that fit, shared out between the Gram warps' ring (a frame stays for its own
-    // products and the next frame's, plus the time its copy takes to arrive) and the sum
-    // warps' ring (filled from L2 shortly before use)
+    // the slots that fit: one ring in which a frame stays until the sum warps have used it, or,
+    // on request, shared out between the Gram warps' ring (a frame stays for its own products and
+    // the next frame's) and a ring of the sum warps (filled from L2 shortly before use)
     const int slots = std::min((int)((kMaxSmem - fixed) / f->slot_bytes), 2 * kMaxRing);
     if (slots < 5) return;
-    int RB = g_tune_sum_slots > 0 ? g_tune_sum_slots : (slots * 3 + 3) / 7;
-    RB = std::max(2, std::min(RB, std::min(slots - 3, kMaxRing)));
+    int RB = 0;                                 // one ring for both unless asked otherwise
+    if (g_tune_sum_slots > 0) RB = std::max(2, std::min(g_tune_sum_slots, std::min(slots - 3, kMaxRing)));
     f->RB = RB;
     f->R = std::min(slots - RB, kMaxRing);
     f->lead = std::max(0, g_tune_lead);

@@ -466,7 +466,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     if (tid == 0) {
         for (int s = 0; s < p.R; s++) {
             mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, p.NM);
+            mbar_init(empty_bar + 8 * s, p.NM + (p.RB == 0 ? p.NA : 0));
         }
         for (int s = 0; s < p.RB; s++) {
             mbar_init(fullb_bar + 8 * s, 1);
@@ -643,12 +643,17 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         int total = 0;
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
             if (!skip) total += it.n;
+        // the frames come from a ring of their own, or (RB == 0) from the Gram warps' ring
+        const bool own = p.RB > 0;
+        const uint32_t sfull_bar = own ? fullb_bar : full_bar, sempty_bar = own ? emptyb_bar : empty_bar;
+        const uint32_t sbase = own ? ringb_base : ring_base;
+        const int SR = own ? p.RB : p.R;
         // one record per frame, and a last one that only writes out what the last item left
         int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before
         for (; q <= total; q++) {
             const int rk = q % kRecRing;
             if (!mbar_wait(rfull_bar + 8 * rk, q / kRecRing, timed_out)) break;
-            if (q < total && !mbar_wait(fullb_bar + 8 * s, use, timed_out)) break;
+            if (q < total && !mbar_wait(sfull_bar + 8 * s, use, timed_out)) break;
             __syncwarp();
             const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
             const uint32_t flush_mask = lds_u32x4(rec).x;
@@ -691,7 +696,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             if (q < total) {
                 uint32_t wa[4];
                 ldmatrix_x4(rec + woff, wa);
-                const uint32_t xb = ringb_base + s * p.slot_bytes + xoff;
+                const uint32_t xb = sbase + s * p.slot_bytes + xoff;
 #pragma unroll
                 for (int pr = 0; pr < 8; pr++) {
                     if (ch0 + pr * 16 < p.S) {
@@ -705,9 +710,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(rempty_bar + 8 * rk);
-                if (q < total) mbar_arrive(emptyb_bar + 8 * s);
+                if (q < total) mbar_arrive(sempty_bar + 8 * s);
             }
-            if (++s == p.RB) { s = 0; use++; }
+            if (++s == SR) { s = 0; use++; }
         }
     } else if (warp == w_sim) {
         // --------------------------------- similarity warp ---------------------------------
@@ -961,13 +966,14 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             mbar_wait(full_bar + 8 * (qq % p.R), qq / p.R, late);
             timed_out |= late;
         }
-    } else if (warp == w_prod + 1) {
+    } else if (warp == w_prod + 1 && p.RB > 0) {
         // ---------------------------------- second producer ----------------------------------
         // The sum warps need a frame only once its record exists, long after the Gram warps are
         // done with it.  Holding the frame in shared memory all that time would let too few frames
         // be in flight, so it is fetched a second time (from L2, where the first copy left it) into
         // a ring of its own, timed by the similarity warp's progress so that it lands about when
-        // the chain warp posts the record.
+        // the chain warp posts the record.  (With RB == 0 there is one ring for both and this warp
+        // has nothing to do.)
         int s = 0, use = 0;
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;

@@ -157,7 +157,7 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     } else {
         const int ncl = fused_resident_clusters(*f);
         const long long tiles_all = (long long)g.B * f->ntiles;
-        const int lo = std::max(1, (int)(g.T / 256)), hi = std::max(lo, std::min(g.T, std::max(1, g.T / 8)));
+        const int lo = 1, hi = std::max(lo, std::min(g.T, std::max(1, g.T / 8)));
         double best_cost = 1e300;
         int best_nseg = lo;
         for (int nseg = lo; nseg <= hi; nseg++) {
@@ -429,9 +429,12 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
 template <typename OutT>
 sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacity, cudaStream_t st) {
     const Geo g = pl.g;
-    // one warp per row; the row count is only known on the device, so the grid covers the most rows there can be
+    // one warp per row, striding; the row count is only known on the device, so the grid covers the
+    // most rows there can be, up to a few waves of blocks (most tokens merge: few rows, and blocks
+    // without a row would only cost their launch)
     const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
-    k_gather<OutT><<<blocks_for(max_rows, 8), 256, 0, st>>>(g, (const long long*)(ws + pl.vid_off),
+    const unsigned blocks = std::min<unsigned>(blocks_for(max_rows, 8), kSmCount * 16);
+    k_gather<OutT><<<blocks, 256, 0, st>>>(g, (const long long*)(ws + pl.vid_off),
                                                  (const int32_t*)(ws + pl.row_anchor),
                                                  (const int32_t*)(ws + pl.row_head),
                                                  (const int32_t*)(ws + pl.piece_next),

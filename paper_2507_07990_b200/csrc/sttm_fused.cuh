@@ -1086,23 +1086,26 @@ k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict
                 }
             }
         } else {
-            // the row's pieces in increasing index order; lists are short (a few per item border),
-            // so the first eight are found once and kept in registers
+            // the row's pieces in increasing index order; lists are short (a few per item border):
+            // one walk that keeps the first eight sorted in registers
             constexpr int kMaxList = 8;
             int ids[kMaxList];
-            int n = 0, last = -1;
+            int n = 0;
             bool longer = false;
-            while (true) {
-                int best = 0x7fffffff;
-                for (int pc = head; pc >= 0; pc = piece_next[pc])
-                    if (pc > last && pc < best) best = pc;
-                if (best == 0x7fffffff) break;
+            for (int pc = head; pc >= 0; pc = piece_next[pc]) {
                 if (n == kMaxList) { longer = true; break; }
+                int v = pc;
 #pragma unroll
-                for (int k = 0; k < kMaxList; k++)
-                    if (k == n) ids[k] = best;
+                for (int k = 0; k < kMaxList; k++) {
+                    if (k < n) {
+                        const int lo = min(ids[k], v);
+                        v = max(ids[k], v);
+                        ids[k] = lo;
+                    } else if (k == n) {
+                        ids[k] = v;
+                    }
+                }
                 n++;
-                last = best;
             }
             const float wsum = (float)row_weight[r];
             // four 128-channel groups per trip, so that 4 x n loads are in flight

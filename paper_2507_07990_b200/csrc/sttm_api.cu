@@ -286,6 +286,26 @@ inline sttm_status launched() {
     return cudaPeekAtLastError() == cudaSuccess ? STTM_OK : STTM_ERR_CUDA;
 }
 
+// Launch with programmatic stream serialization: the kernel's blocks may be set up while the
+// kernel before it in the stream drains; every kernel launched this way begins with
+// wait_for_prior_kernel(), so it touches nothing before that kernel has completed.
+template <typename... KArgs, typename... Args>
+sttm_status launch_after(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+    g_launches++;
+    return e == cudaSuccess ? STTM_OK : STTM_ERR_CUDA;
+}
+
 inline unsigned blocks_for(long long items, int per_block) { return (unsigned)((items + per_block - 1) / per_block); }
 
 sttm_status run_spatial(const void* feats, const sttm_params* p, const Plan& pl, char* ws, int8_t* cover,
@@ -434,13 +454,10 @@ sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacit
     // without a row would only cost their launch)
     const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
     const unsigned blocks = std::min<unsigned>(blocks_for(max_rows, 8), kSmCount * 16);
-    k_gather<OutT><<<blocks, 256, 0, st>>>(g, (const long long*)(ws + pl.vid_off),
-                                                 (const int32_t*)(ws + pl.row_anchor),
-                                                 (const int32_t*)(ws + pl.row_head),
-                                                 (const int32_t*)(ws + pl.piece_next),
-                                                 (const int32_t*)(ws + pl.row_weight), (const OutT*)(ws + pl.staging),
-                                                 (const float*)(ws + pl.pieces), (OutT*)out, capacity);
-    return launched();
+    return launch_after(k_gather<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
+                        (const int32_t*)(ws + pl.row_anchor), (const int32_t*)(ws + pl.row_head),
+                        (const int32_t*)(ws + pl.piece_next), (const int32_t*)(ws + pl.row_weight),
+                        (const OutT*)(ws + pl.staging), (const float*)(ws + pl.pieces), (OutT*)out, capacity);
 }
 
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
@@ -634,32 +651,36 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
         s = run_fused(feats, p, pl, ws, device_status, st);
         if (s != STTM_OK) return s;
         mark_stage(1, st);
-        k_resolve_roots<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, pl.f.nseg + 1, (const int32_t*)(ws + pl.cell_row),
-                                                                  root, device_status);
-        if ((s = launched()) != STTM_OK) return s;
+        s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, pl.f.nseg + 1,
+                         (const int32_t*)(ws + pl.cell_row), root, device_status);
+        if (s != STTM_OK) return s;
         mark_stage(2, st);
         int32_t* frame_roots = (int32_t*)(ws + pl.frame_roots);
         int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
         long long* vid_off = (long long*)(ws + pl.vid_off);
         int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
         int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
-        k_frame_roots<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_roots);
-        if ((s = launched()) != STTM_OK) return s;
-        k_scan_frames<<<1, 1024, 0, st>>>(g, frame_roots, frame_base, out_count, vid_off, out_offsets);
-        if ((s = launched()) != STTM_OK) return s;
-        k_rows<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_base, vid_off, row_at_root, row_anchor, out_pos,
-                                          p->out_capacity_rows, (int)p->pos, device_status);
-        if ((s = launched()) != STTM_OK) return s;
+        s = launch_after(k_frame_roots, (unsigned)(g.B * g.T), 256, st, g, (const int8_t*)cover, (const int32_t*)link,
+                         frame_roots);
+        if (s != STTM_OK) return s;
+        s = launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)frame_roots, frame_base, out_count, vid_off,
+                         out_offsets);
+        if (s != STTM_OK) return s;
+        s = launch_after(k_rows, (unsigned)(g.B * g.T), 256, st, g, (const int8_t*)cover, (const int32_t*)link,
+                         (const int32_t*)frame_base, (const long long*)vid_off, row_at_root, row_anchor, out_pos,
+                         (long long)p->out_capacity_rows, (int)p->pos, device_status);
+        if (s != STTM_OK) return s;
         if (merge_map != nullptr) {
-            k_merge_map<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, root, row_at_root, merge_map);
-            if ((s = launched()) != STTM_OK) return s;
+            s = launch_after(k_merge_map, blocks_for(pl.cells, 256), 256, st, g, (const int32_t*)root,
+                             (const int32_t*)row_at_root, merge_map);
+            if (s != STTM_OK) return s;
         }
         const int npieces = pl.f.nitems * kPieceSlots;
-        k_piece_link<<<blocks_for(npieces, 256), 256, 0, st>>>(g, npieces, (const int2*)(ws + pl.piece_meta), root,
-                                                              row_at_root, vid_off, (int32_t*)(ws + pl.row_head),
-                                                              (int32_t*)(ws + pl.piece_next),
-                                                              (int32_t*)(ws + pl.row_weight));
-        if ((s = launched()) != STTM_OK) return s;
+        s = launch_after(k_piece_link, blocks_for(npieces, 256), 256, st, g, npieces,
+                         (const int2*)(ws + pl.piece_meta), (const int32_t*)root, (const int32_t*)row_at_root,
+                         (const long long*)vid_off, (int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.piece_next),
+                         (int32_t*)(ws + pl.row_weight));
+        if (s != STTM_OK) return s;
         mark_stage(3, st);
         s = p->out_dtype == STTM_BF16 ? launch_gather<__nv_bfloat16>(pl, ws, out_feats, p->out_capacity_rows, st)
                                       : launch_gather<float>(pl, ws, out_feats, p->out_capacity_rows, st);

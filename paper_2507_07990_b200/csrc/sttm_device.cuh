@@ -58,6 +58,11 @@ struct Col {
     }
 };
 
+// First statement of a kernel that may be launched with programmatic stream serialization
+// (its blocks may become resident while the kernel before it in the stream still runs): waits
+// until that kernel has completed and its writes are visible.  Returns at once otherwise.
+__device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

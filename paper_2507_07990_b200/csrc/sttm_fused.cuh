@@ -1015,6 +1015,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
 __global__ void __launch_bounds__(256)
 k_resolve_roots(Geo g, int max_hops, const int32_t* __restrict__ chain_key, int32_t* __restrict__ root,
                 int32_t* status) {
+    wait_for_prior_kernel();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (long long)g.B * g.N) return;
     const long long vb = i / g.N * g.N;
@@ -1040,6 +1041,7 @@ __global__ void __launch_bounds__(256)
 k_piece_link(Geo g, int npieces, const int2* __restrict__ piece_meta, const int32_t* __restrict__ root,
              const int32_t* __restrict__ row_at_root, const long long* __restrict__ vid_off,
              int32_t* __restrict__ row_head, int32_t* __restrict__ piece_next, int32_t* __restrict__ row_weight) {
+    wait_for_prior_kernel();
     const int pc = blockIdx.x * blockDim.x + threadIdx.x;
     if (pc >= npieces) return;
     const int2 m = piece_meta[pc];
@@ -1060,6 +1062,7 @@ k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict
          const int32_t* __restrict__ row_head, const int32_t* __restrict__ piece_next,
          const int32_t* __restrict__ row_weight, const OutT* __restrict__ staging, const float* __restrict__ pieces,
          OutT* __restrict__ out, long long capacity) {
+    wait_for_prior_kernel();
     const int lane = threadIdx.x & 31;
     const long long nrows = min(vid_off[g.B], capacity);
     const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
@@ -1167,6 +1170,7 @@ k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict
 __global__ void __launch_bounds__(256)
 k_merge_map(Geo g, const int32_t* __restrict__ root, const int32_t* __restrict__ row_at_root,
             int32_t* __restrict__ merge_map) {
+    wait_for_prior_kernel();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (long long)g.B * g.N) return;
     const long long vb = i / g.N * g.N;

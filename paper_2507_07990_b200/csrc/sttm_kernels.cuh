@@ -341,6 +341,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int& total, int* smem
 __global__ void __launch_bounds__(256)
 k_frame_roots(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__ link,
               int32_t* __restrict__ frame_roots) {
+    wait_for_prior_kernel();
     const long long bt = blockIdx.x;
     int n = 0;
     for (int cell = threadIdx.x; cell < g.HW; cell += blockDim.x)
@@ -355,6 +356,7 @@ k_frame_roots(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict
 __global__ void __launch_bounds__(1024)
 k_scan_frames(Geo g, const int32_t* __restrict__ frame_roots, int32_t* __restrict__ frame_base,
               int32_t* __restrict__ out_count, long long* __restrict__ vid_off, int64_t* out_offsets) {
+    wait_for_prior_kernel();
     __shared__ int sm[33];
     __shared__ long long running_rows;
     if (threadIdx.x == 0) running_rows = 0;
@@ -390,6 +392,7 @@ k_rows(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__ link
        const int32_t* __restrict__ frame_base, const long long* __restrict__ vid_off,
        int32_t* __restrict__ row_at_root, int32_t* __restrict__ row_anchor, int32_t* __restrict__ out_pos,
        long long capacity, int pos_mode, int32_t* status) {
+    wait_for_prior_kernel();
     __shared__ int sm[33];
     const long long bt = blockIdx.x;
     const int b = (int)(bt / g.T), t = (int)(bt % g.T);

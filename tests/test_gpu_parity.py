@@ -210,3 +210,25 @@ def test_bad_arguments_are_rejected_on_the_host():
                              C.c_void_p(dev.data_ptr()), C.c_void_p(dev.data_ptr()), None,
                              C.c_void_p(dev.data_ptr()), None, None, None)
     assert code == 3
+
+
+# Shapes of the paper's other set-ups at their real feature widths: the 14x14 grid of
+# LLaVA-Video (Section 3.2), a non-square dynamic-resolution grid (three levels: grids up to 16 cells a side), and D = 8192 of the 72B
+# model (eight CTAs per cluster, eight sum warps per CTA).
+@pytest.mark.parametrize("shape", [(6, 14, 14, 3584), (4, 16, 12, 3584), (5, 13, 13, 8192), (3, 16, 16, 8192)],
+                         ids=lambda s: "T%dH%dW%dD%d" % s)
+def test_other_workload_shapes_full_width(shape):
+    T, H, W, D = shape
+    done = 0
+    for seed in range(3):
+        spec = helpers.small_spec(300 + seed, T, H, W, D, sigma=0.05)
+        video = inputs.make_video(spec)
+        taus = helpers.safe_thresholds(video, 0.5, 0.5)
+        if taus is None:
+            continue
+        for out_dtype in (torch.float32, torch.bfloat16):
+            run_and_compare(video, taus[0], taus[1], out_dtype=out_dtype)
+        assert binding.load_library().sttm_last_path() == 1          # the fused kernel took it
+        done += 1
+        break
+    assert done >= 1, "no seed gave thresholds with a margin"

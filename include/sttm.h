@@ -55,6 +55,10 @@ typedef enum { STTM_POS_SURVIVED = 0, STTM_POS_REASSIGNED = 1 } sttm_pos_mode;
 /* Averaging weights inside a chain (the paper does not fix them): one per node, or the
  * number of grid cells the node covers. */
 typedef enum { STTM_W_NODE = 0, STTM_W_AREA = 1 } sttm_weight_mode;
+/* Which of several overlapping nodes of frame t-1 above tau_t a node is linked to (Section 3.3):
+ * the top-left one (the paper's choice), or the most similar one (the "optimal" destination of
+ * the paper's ablation; equal similarities: the top-left of them). */
+typedef enum { STTM_MATCH_TOPLEFT = 0, STTM_MATCH_BEST = 1 } sttm_match_mode;
 
 typedef struct sttm_params {
     int B, T, H, W, D;            /* videos, frames, grid, channels                      */
@@ -67,10 +71,11 @@ typedef struct sttm_params {
     sttm_pos_mode pos;
     sttm_weight_mode wt;
     long long out_capacity_rows;  /* rows available in out_feats / out_pos (all videos)   */
+    sttm_match_mode match;        /* destination rule of the temporal link                */
 } sttm_params;
 
 /* Fills *p with defaults: B=1, bf16 in and out, lv1=4, survived ids, node weights,
- * capacity B*T*H*W.  Host only. */
+ * top-left destination, capacity B*T*H*W.  Host only. */
 void sttm_default_params(sttm_params* p, int T, int H, int W, int D, float tau_s, float tau_t);
 
 /* Bytes of device workspace the calls below need for these params (0 on bad params). */

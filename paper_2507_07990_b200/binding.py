@@ -19,6 +19,7 @@ from . import build as _build
 BF16, F32 = 0, 1
 POS_SURVIVED, POS_REASSIGNED = 0, 1
 W_NODE, W_AREA = 0, 1
+MATCH_TOPLEFT, MATCH_BEST = 0, 1
 STATUS_NAMES = ["ok", "bad argument", "unsupported shape", "workspace too small",
                 "output capacity exceeded", "root search did not converge", "CUDA error"]
 
@@ -34,7 +35,7 @@ class SttmParams(C.Structure):
                 ("in_dtype", C.c_int), ("out_dtype", C.c_int), ("lv1", C.c_int),
                 ("tau_s", C.c_float), ("tau_t", C.c_float),
                 ("tau_s_per_video", C.POINTER(C.c_float)), ("tau_t_per_video", C.POINTER(C.c_float)),
-                ("pos", C.c_int), ("wt", C.c_int), ("out_capacity_rows", C.c_longlong)]
+                ("pos", C.c_int), ("wt", C.c_int), ("out_capacity_rows", C.c_longlong), ("match", C.c_int)]
 
 
 class SttmError(RuntimeError):
@@ -130,7 +131,8 @@ class Problem:
 
 def make_params(shape: Sequence[int], in_dtype: torch.dtype, tau_s: Union[float, Sequence[float]],
                 tau_t: Union[float, Sequence[float]], lv1: int = 4, out_dtype: torch.dtype = torch.bfloat16,
-                pos: int = POS_SURVIVED, wt: int = W_NODE, capacity: Optional[int] = None) -> Problem:
+                pos: int = POS_SURVIVED, wt: int = W_NODE, capacity: Optional[int] = None,
+                match: int = MATCH_TOPLEFT) -> Problem:
     B, T, H, W, D = shape
     p = SttmParams()
     p.B, p.T, p.H, p.W, p.D = B, T, H, W, D
@@ -148,7 +150,7 @@ def make_params(shape: Sequence[int], in_dtype: torch.dtype, tau_s: Union[float,
         arr = (C.c_float * B)(*[float(v) for v in tau_t])
         p.tau_t_per_video = C.cast(arr, C.POINTER(C.c_float))
         keep.append(arr)
-    p.pos, p.wt = pos, wt
+    p.pos, p.wt, p.match = pos, wt, match
     p.out_capacity_rows = B * T * H * W if capacity is None else capacity
     return Problem(p, tuple(keep))
 
@@ -219,12 +221,12 @@ def sttm_spatial_static(feats: torch.Tensor, tau_s, cover: torch.Tensor, counts:
 
 
 def sttm_temporal(feats: torch.Tensor, cover: torch.Tensor, tau_s, tau_t, ws: torch.Tensor, lv1: int = 4,
-                  want_sims: bool = False):
+                  want_sims: bool = False, match: int = MATCH_TOPLEFT):
     """Temporal stage alone, on a workspace sttm_spatial has filled.  Returns (link, root,
     temporal_sims or None, device_status)."""
     feats = _as5d(feats)
     B, T, H, W, D = feats.shape
-    prob = make_params(feats.shape, feats.dtype, tau_s, tau_t, lv1)
+    prob = make_params(feats.shape, feats.dtype, tau_s, tau_t, lv1, match=match)
     link = torch.empty((B, T * H * W), dtype=torch.int32, device=feats.device)
     root = torch.empty((B, T * H * W), dtype=torch.int32, device=feats.device)
     tsim = torch.empty((B, T * H * W), dtype=torch.float32, device=feats.device) if want_sims else None
@@ -250,8 +252,8 @@ class MergePlan:
     """Pre-allocated buffers for repeated sttm_merge_ex calls on one problem shape."""
 
     def __init__(self, shape, in_dtype, tau_s, tau_t, lv1=4, out_dtype=torch.bfloat16, pos=POS_SURVIVED,
-                 wt=W_NODE, capacity=None, want_map=False, device="cuda"):
-        self.problem = make_params(shape, in_dtype, tau_s, tau_t, lv1, out_dtype, pos, wt, capacity)
+                 wt=W_NODE, capacity=None, want_map=False, device="cuda", match=MATCH_TOPLEFT):
+        self.problem = make_params(shape, in_dtype, tau_s, tau_t, lv1, out_dtype, pos, wt, capacity, match)
         p = self.problem.params
         B, T, H, W, D = shape
         self.ws = alloc_workspace(self.problem, device)
@@ -275,11 +277,11 @@ class MergePlan:
 
 def sttm_merge_ex(feats: torch.Tensor, tau_s, tau_t, lv1: int = 4, out_dtype: torch.dtype = torch.bfloat16,
                   pos: int = POS_SURVIVED, wt: int = W_NODE, capacity: Optional[int] = None,
-                  want_map: bool = True) -> MergeOutput:
+                  want_map: bool = True, match: int = MATCH_TOPLEFT) -> MergeOutput:
     """The whole path for ``[B, T, H, W, D]`` (or one video ``[T, H, W, D]``)."""
     feats = _as5d(feats)
     plan = MergePlan(tuple(feats.shape), feats.dtype, tau_s, tau_t, lv1, out_dtype, pos, wt, capacity, want_map,
-                     feats.device)
+                     feats.device, match)
     return plan.run(feats)
 
 

@@ -194,6 +194,7 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
     if (p->D % 4 != 0) return STTM_ERR_ARG;
     if (p->in_dtype != STTM_BF16 && p->in_dtype != STTM_F32) return STTM_ERR_ARG;
     if (p->out_dtype != STTM_BF16 && p->out_dtype != STTM_F32) return STTM_ERR_ARG;
+    if (p->match != STTM_MATCH_TOPLEFT && p->match != STTM_MATCH_BEST) return STTM_ERR_ARG;
     if (p->B > kMaxBatch) return STTM_ERR_UNSUPPORTED;
     if ((long long)p->B * p->T * p->H * p->W >= (1ll << 31)) return STTM_ERR_UNSUPPORTED;
     Geo& g = pl->g;
@@ -336,7 +337,7 @@ sttm_status run_temporal(const void* feats, const sttm_params* p, const Plan& pl
         using T = std::remove_const_t<std::remove_pointer_t<decltype(tag)>>;
         constexpr int LV = decltype(lv)::value;
         k_temporal<LV, T><<<blocks_for(warps, kWarpsPerBlock), kWarpsPerBlock * 32, 0, st>>>(
-            (const T*)feats, g, taus, cover, norms, link, tsim);
+            (const T*)feats, g, taus, cover, norms, link, tsim, p->match == STTM_MATCH_BEST ? 1 : 0);
         sttm_status s = launched();
         if (s != STTM_OK) return s;
         k_roots<LV><<<g.B * g.ncol, 256, 0, st>>>(g, cover, link, root, status, max_rounds);
@@ -419,6 +420,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.row_bytes = f.row_bytes; fp.slot_bytes = f.slot_bytes; fp.R = f.R; fp.RB = f.RB; fp.lead = f.lead;
     fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
     fp.weight_mode = (int)p->wt;
+    fp.match_best = p->match == STTM_MATCH_BEST ? 1 : 0;
     fp.out_f32 = p->out_dtype == STTM_F32;
     fp.cover = (int8_t*)(ws + pl.cover);
     fp.link = (int32_t*)(ws + pl.link);
@@ -525,7 +527,7 @@ void sttm_default_params(sttm_params* p, int T, int H, int W, int D, float tau_s
     p->in_dtype = STTM_BF16; p->out_dtype = STTM_BF16;
     p->lv1 = 4;
     p->tau_s = tau_s; p->tau_t = tau_t;
-    p->pos = STTM_POS_SURVIVED; p->wt = STTM_W_NODE;
+    p->pos = STTM_POS_SURVIVED; p->wt = STTM_W_NODE; p->match = STTM_MATCH_TOPLEFT;
     p->out_capacity_rows = (long long)T * H * W;
 }
 

@@ -87,7 +87,7 @@ struct FusedParams {
     int row_bytes, slot_bytes;
     int R, RB, lead;         // slots of the Gram warps' ring and of the sum warps' ring; see the second producer
     int F, nseg, nitems;
-    int weight_mode, out_f32;
+    int weight_mode, out_f32, match_best;
     int8_t* cover;
     int32_t* link;
     int32_t* chain_key;      // [B*N] per cell: root cell id of its chain as far as the item knows it
@@ -798,7 +798,18 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     const bool pass = rep && cos_above(dot, nk, pnk, tau_t);
                     const uint32_t passm = (__ballot_sync(full, pass) >> (16 * half)) & 0xffffu;
                     const uint32_t cand = passm & lane_region(lg, c, lv);
-                    const int cstar = cand ? __ffs(cand) - 1 : 0;     // first in row-major order: the top-left one
+                    int cstar = cand ? __ffs(cand) - 1 : 0;           // first in row-major order: the top-left one
+                    if (p.match_best) {
+                        // the most similar of them instead (equal ones: the first); the cosine itself is
+                        // needed here, every lane looks at the 16 lanes of its half
+                        const float cosv = pass ? dot / (sqrtf(nk) * sqrtf(pnk)) : -2.f;
+                        float best = -2.f;
+#pragma unroll
+                        for (int i = 0; i < 16; i++) {
+                            const float si = __shfl_sync(full, cosv, 16 * half + i);
+                            if (((cand >> i) & 1u) && si > best) { best = si; cstar = i; }
+                        }
+                    }
                     const int lu_star = __shfl_sync(full, lu, 16 * half + cstar);
                     link_local = cand ? lane_anchor(lg, cstar, lu_star) : -1;      // same sub-tile: same bits
                 }

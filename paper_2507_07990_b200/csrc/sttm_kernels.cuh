@@ -156,7 +156,8 @@ k_spatial(const T* __restrict__ feats, Geo g, Taus taus, int8_t* __restrict__ co
 template <int LEVELS, typename T>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 k_temporal(const T* __restrict__ feats, Geo g, Taus taus, const int8_t* __restrict__ cover,
-           const float* __restrict__ norms, int32_t* __restrict__ link, float* __restrict__ tsim) {
+           const float* __restrict__ norms, int32_t* __restrict__ link, float* __restrict__ tsim,
+           int match_best) {
     using C = Col<LEVELS>;
     const int lane = threadIdx.x & 31;
     const long long w = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
@@ -228,8 +229,10 @@ k_temporal(const T* __restrict__ feats, Geo g, Taus taus, const int8_t* __restri
     const float* np = nc - (long long)g.ncol * C::NN;
     const float tau = taus.t[b];
     // lane a keeps the link of the node of frame t anchored at cell a; pairs are visited
-    // in row-major order of their finer node, so the first passing one is the top-left
+    // in row-major order of their finer node, so the first passing one is the top-left (and
+    // with match_best a later one only replaces it when it is strictly more similar)
     int my_link = -1;
+    float my_best = 0.f;
     float my_sim = __int_as_float(0x7fc00000);
 #pragma unroll
     for (int c = 0; c < C::NC; c++) {
@@ -241,7 +244,10 @@ k_temporal(const T* __restrict__ feats, Geo g, Taus taus, const int8_t* __restri
             const int mv = ~((1 << lv) - 1), mu = ~((1 << lu) - 1);
             const int anchor_v = (C::dy(c) & mv) * C::SIDE + (C::dx(c) & mv);
             const int anchor_u = (t - 1) * g.HW + (y0 + (C::dy(c) & mu)) * g.W + x0 + (C::dx(c) & mu);
-            if (lane == anchor_v && my_link < 0 && s > tau) my_link = anchor_u;
+            if (lane == anchor_v && s > tau && (my_link < 0 || (match_best && s > my_best))) {
+                my_link = anchor_u;
+                my_best = s;
+            }
         }
     }
     const int mvm = ~((1 << lc_mine) - 1);

@@ -33,12 +33,13 @@ def tuning(request):
 
 
 def run_and_compare(video_np, tau_s, tau_t, lv1=4, out_dtype=torch.float32, wt=binding.W_NODE,
-                    pos=binding.POS_SURVIVED, stages=True):
+                    pos=binding.POS_SURVIVED, stages=True, match=binding.MATCH_TOPLEFT):
     T, H, W, D = video_np.shape
     N = T * H * W
-    ref = oracle.merge(video_np, tau_s, tau_t, lv1=lv1, weight_mode=wt, pos_mode=pos, want_sims=True, want_pairs=True)
+    ref = oracle.merge(video_np, tau_s, tau_t, lv1=lv1, weight_mode=wt, pos_mode=pos, match_mode=match,
+                       want_sims=True, want_pairs=True)
     dev = helpers.to_torch(video_np)
-    out = binding.sttm_merge_ex(dev, tau_s, tau_t, lv1=lv1, out_dtype=out_dtype, wt=wt, pos=pos)
+    out = binding.sttm_merge_ex(dev, tau_s, tau_t, lv1=lv1, out_dtype=out_dtype, wt=wt, pos=pos, match=match)
     torch.cuda.synchronize()
     assert int(out.device_status.item()) == 0
     count = int(out.out_count[0].item())
@@ -50,7 +51,8 @@ def run_and_compare(video_np, tau_s, tau_t, lv1=4, out_dtype=torch.float32, wt=b
                                   out_dtype == torch.bfloat16)
     if stages:
         cover, counts, sims, ws = binding.sttm_spatial(dev, tau_s, lv1=lv1, want_sims=True)
-        link, root, tsim, status = binding.sttm_temporal(dev, cover, tau_s, tau_t, ws, lv1=lv1, want_sims=True)
+        link, root, tsim, status = binding.sttm_temporal(dev, cover, tau_s, tau_t, ws, lv1=lv1, want_sims=True,
+                                                         match=match)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         np.testing.assert_array_equal(cover[0].cpu().numpy(), ref.cover_level)
@@ -232,3 +234,36 @@ def test_other_workload_shapes_full_width(shape):
         done += 1
         break
     assert done >= 1, "no seed gave thresholds with a margin"
+
+
+def test_most_similar_destination(tuning):
+    """Section 3.3's other destination rule: among the overlapping nodes above tau_t the most
+    similar one instead of the top-left one.  Both sides pick a maximum, so the inputs are
+    chosen such that the two best candidates of every node are at least 1e-4 apart."""
+    assert binding.MATCH_BEST == oracle.MATCH_BEST
+    checked = differs = 0
+    for shape in [(6, 13, 13, 256), (5, 16, 16, 384), (4, 8, 8, 64)]:
+        T, H, W, D = shape
+        for seed in range(4):
+            spec = helpers.small_spec(400 + seed, T, H, W, D, dtype="f32" if D == 64 else "bf16",
+                                      sigma=0.3 if D < 200 else 0.05, p_static=0.5)
+            video = inputs.make_video(spec)
+            taus = helpers.safe_thresholds(video, 0.6, 0.15)
+            if taus is None:
+                continue
+            ref = oracle.merge(video, taus[0], taus[1], match_mode=oracle.MATCH_BEST, want_pairs=True, want_feats=False)
+            above = {}
+            for v, sim in zip(ref.tsim_v.tolist(), ref.tsim.tolist()):
+                if sim > taus[1]:
+                    above.setdefault(v, []).append(sim)
+            gaps = [sorted(c)[-1] - sorted(c)[-2] for c in above.values() if len(c) > 1]
+            if gaps and min(gaps) < 1e-4:
+                continue
+            topleft = oracle.merge(video, taus[0], taus[1], want_feats=False)
+            differs += int((topleft.link != ref.link).sum())
+            run_and_compare(video, taus[0], taus[1], match=binding.MATCH_BEST)
+            run_and_compare(video, taus[0], taus[1], out_dtype=torch.bfloat16, stages=False, match=binding.MATCH_BEST)
+            checked += 1
+            break
+    assert checked >= 2, "no input with a margin between the best candidates"
+    assert differs > 0, "the rule never chose another destination than the top-left one"

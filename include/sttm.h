@@ -171,6 +171,27 @@ sttm_status sttm_merge_host(const void* h_feats, const sttm_params* p,
                             void* h_out_feats, int32_t* h_out_pos, int32_t* h_merge_map,
                             int32_t* h_out_count, int64_t* h_out_offsets, int32_t* h_device_status);
 
+/*
+ * "Merged" position strategy of Section 3.4 (the first of its three ways to give a merged token a
+ * rotary position): the position of an output row is the average of the positions of the tokens
+ * merged into it.  Reading taken here: the position of an input token is its index t*H*W + y*W + x
+ * inside its video (the numbering of the survived ids), every cell of the video counts once, and the
+ * average is returned as a number (a rotary embedding evaluated at it is left to the caller).
+ *   merge_map     [B, N] int32, N = T*H*W: row (inside its video) of every cell, as written by
+ *                 sttm_merge_ex
+ *   out_offsets   [B + 1] int64: first row of every video in the packed output, as written by
+ *                 sttm_merge_ex
+ *   ws            at least sttm_merged_positions_workspace(capacity_rows) bytes, 256-byte aligned
+ *   out_pos_mean  [capacity_rows] float32: sum of the member indices (exact, 64-bit) divided by their
+ *                 number in double precision, rounded once to float; rows at or beyond capacity_rows
+ *                 are dropped and (1 << STTM_ERR_CAPACITY) is OR-ed into *device_status (may be NULL)
+ * Asynchronous on `stream`.
+ */
+size_t sttm_merged_positions_workspace(long long capacity_rows);
+sttm_status sttm_merged_positions(const int32_t* merge_map, const int64_t* out_offsets, int B, long long N,
+                                  void* ws, size_t ws_bytes, float* out_pos_mean, long long capacity_rows,
+                                  int32_t* device_status, void* stream);
+
 /* Frees the cached buffers of sttm_merge / sttm_merge_host on the current device. */
 void sttm_release_cache(void);
 

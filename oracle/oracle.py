@@ -151,3 +151,17 @@ def merge(feats: np.ndarray, tau_s: float, tau_t: float, lv1: int = 4,
     return OracleResult(count, sims, cover, link, root, mmap,
                         out[:count] if out is not None else None, pos[:count], members[:count],
                         tv, tu, ts, int(counters[0]), int(counters[1]))
+
+
+def merged_positions(merge_map: np.ndarray, count: int) -> np.ndarray:
+    """Section 3.4, "merged" position strategy, read as: the position of an output row is the mean
+    of the indices (t*H*W + y*W + x) of the cells merged into it.  ``merge_map`` holds the row of
+    every cell of one video.  Plain definition: integer sums, one division in double precision,
+    one rounding to float32."""
+    merge_map = np.asarray(merge_map).reshape(-1)
+    sums = np.zeros(count, dtype=np.int64)
+    cnts = np.zeros(count, dtype=np.int64)
+    for i, r in enumerate(merge_map.tolist()):
+        sums[r] += i
+        cnts[r] += 1
+    return (sums.astype(np.float64) / cnts.astype(np.float64)).astype(np.float32)

@@ -27,7 +27,8 @@ EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame",
            "sttm_temporal", "sttm_merge_ex", "sttm_merge", "sttm_merge_host", "sttm_release_cache",
            "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
            "sttm_set_stage_events", "sttm_set_tuning", "sttm_set_ring_split", "sttm_last_path",
-           "sttm_fused_launch_shape", "sttm_spatial_static"]
+           "sttm_fused_launch_shape", "sttm_spatial_static", "sttm_merged_positions",
+           "sttm_merged_positions_workspace"]
 
 
 class SttmParams(C.Structure):
@@ -88,6 +89,11 @@ def load_library(path: Optional[str] = None):
     lib.sttm_set_stage_events.restype = None
     lib.sttm_set_tuning.argtypes = [C.c_int, C.c_int, C.c_int]
     lib.sttm_set_tuning.restype = None
+    lib.sttm_merged_positions_workspace.argtypes = [C.c_longlong]
+    lib.sttm_merged_positions_workspace.restype = C.c_size_t
+    lib.sttm_merged_positions.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_longlong, C.c_void_p, C.c_size_t,
+                                          C.c_void_p, C.c_longlong, C.c_void_p, C.c_void_p]
+    lib.sttm_merged_positions.restype = C.c_int
     lib.sttm_set_ring_split.argtypes = [C.c_int, C.c_int]
     lib.sttm_set_ring_split.restype = None
     lib.sttm_last_path.argtypes = []
@@ -283,6 +289,22 @@ def sttm_merge_ex(feats: torch.Tensor, tau_s, tau_t, lv1: int = 4, out_dtype: to
     plan = MergePlan(tuple(feats.shape), feats.dtype, tau_s, tau_t, lv1, out_dtype, pos, wt, capacity, want_map,
                      feats.device, match)
     return plan.run(feats)
+
+
+def sttm_merged_positions(merge_map: torch.Tensor, out_offsets: torch.Tensor, rows: int):
+    """Mean member index of every output row ("merged" positions of Section 3.4) from the merge map and
+    the video offsets that sttm_merge_ex wrote.  Returns (float32 [rows], device_status)."""
+    if merge_map.dim() != 2 or merge_map.dtype != torch.int32 or not merge_map.is_cuda or not merge_map.is_contiguous():
+        raise ValueError("merge_map must be a contiguous int32 CUDA tensor [B, N]")
+    B, N = merge_map.shape
+    lib = load_library()
+    ws = torch.empty(int(lib.sttm_merged_positions_workspace(rows)) + 256, dtype=torch.uint8, device=merge_map.device)
+    ws = ws[(-ws.data_ptr()) % 256:]
+    out = torch.empty((rows,), dtype=torch.float32, device=merge_map.device)
+    status = torch.zeros(1, dtype=torch.int32, device=merge_map.device)
+    _check(lib.sttm_merged_positions(_ptr(merge_map), _ptr(out_offsets), B, N, _ptr(ws), ws.numel(), _ptr(out), rows,
+                                     _ptr(status), _stream()), "sttm_merged_positions")
+    return out, status
 
 
 def sttm_merge(feats: torch.Tensor, tau_s: float, tau_t: float):

@@ -752,6 +752,32 @@ sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_
                          stream);
 }
 
+size_t sttm_merged_positions_workspace(long long capacity_rows) {
+    if (capacity_rows <= 0) return 0;
+    return ((size_t)capacity_rows * 8 + 255) / 256 * 256 + (size_t)capacity_rows * 4;
+}
+
+sttm_status sttm_merged_positions(const int32_t* merge_map, const int64_t* out_offsets, int B, long long N, void* ws,
+                                  size_t ws_bytes, float* out_pos_mean, long long capacity_rows,
+                                  int32_t* device_status, void* stream) {
+    if (!merge_map || !out_offsets || !ws || !out_pos_mean) return STTM_ERR_ARG;
+    if (B < 1 || N < 1 || capacity_rows < 1 || misaligned(ws, 256)) return STTM_ERR_ARG;
+    if (B > kMaxBatch || (long long)B * N >= (1ll << 31)) return STTM_ERR_UNSUPPORTED;
+    const size_t need = sttm_merged_positions_workspace(capacity_rows);
+    if (ws_bytes < need) return STTM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long* sum = (unsigned long long*)ws;
+    unsigned int* cnt = (unsigned int*)((char*)ws + ((size_t)capacity_rows * 8 + 255) / 256 * 256);
+    STTM_CUDA_TRY(cudaMemsetAsync(ws, 0, need, st));
+    k_pos_accumulate<<<blocks_for((long long)B * N, 256), 256, 0, st>>>(B, N, merge_map, out_offsets, sum, cnt,
+                                                                       capacity_rows, device_status);
+    sttm_status s = launched();
+    if (s != STTM_OK) return s;
+    const long long rows_max = std::min<long long>(capacity_rows, (long long)B * N);
+    k_pos_finish<<<blocks_for(rows_max, 256), 256, 0, st>>>(rows_max, out_offsets, B, sum, cnt, out_pos_mean);
+    return launched();
+}
+
 sttm_status sttm_merge_host(const void* h_feats, const sttm_params* p, void* h_out_feats, int32_t* h_out_pos,
                             int32_t* h_merge_map, int32_t* h_out_count, int64_t* h_out_offsets,
                             int32_t* h_device_status) {

@@ -607,4 +607,33 @@ k_combine(Geo g, int Tc, const long long* __restrict__ vid_off, const int32_t* _
     }
 }
 
+// ---------------------------------------------------------------------------------
+// "Merged" positions (Section 3.4): per output row the mean of its member cells' indices.
+// Integer sums (exact), one division per row.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_pos_accumulate(int B, long long N, const int32_t* __restrict__ merge_map, const int64_t* __restrict__ out_offsets,
+                 unsigned long long* __restrict__ sum, unsigned int* __restrict__ cnt, long long capacity,
+                 int32_t* status) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)B * N) return;
+    const int b = (int)(i / N);
+    const long long row = out_offsets[b] + merge_map[i];
+    if (row >= capacity) {
+        if (status != nullptr) atomicOr(status, kStatusCapacity);
+        return;
+    }
+    atomicAdd(sum + row, (unsigned long long)(i - (long long)b * N));
+    atomicAdd(cnt + row, 1u);
+}
+
+__global__ void __launch_bounds__(256)
+k_pos_finish(long long rows_max, const int64_t* __restrict__ out_offsets, int B,
+             const unsigned long long* __restrict__ sum, const unsigned int* __restrict__ cnt,
+             float* __restrict__ out_pos_mean) {
+    const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows_max || r >= out_offsets[B]) return;
+    out_pos_mean[r] = cnt[r] ? (float)((double)sum[r] / (double)cnt[r]) : 0.f;
+}
+
 }  // namespace sttm

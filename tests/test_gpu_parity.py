@@ -267,3 +267,32 @@ def test_most_similar_destination(tuning):
             break
     assert checked >= 2, "no input with a margin between the best candidates"
     assert differs > 0, "the rule never chose another destination than the top-left one"
+
+
+def test_merged_positions():
+    """The "merged" position output (Section 3.4) from the library's own merge map, bit for bit
+    against the oracle's definition; a batch of two videos, and the capacity condition."""
+    specs = [helpers.small_spec(500 + v, 6, 13, 13, 256, p_static=p) for v, p in enumerate((0.9, 0.4))]
+    videos, taus = [], []
+    for spec in specs:
+        video = inputs.make_video(spec)
+        t = helpers.safe_thresholds(video, 0.5, 0.5)
+        assert t is not None
+        videos.append(video)
+        taus.append(t)
+    dev = helpers.to_torch(np.stack(videos))
+    out = binding.sttm_merge_ex(dev, [t[0] for t in taus], [t[1] for t in taus], out_dtype=torch.bfloat16)
+    rows = int(out.out_offsets[-1].item())
+    pos, status = binding.sttm_merged_positions(out.merge_map, out.out_offsets, rows)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    offs = out.out_offsets.tolist()
+    got = pos.cpu().numpy()
+    for v, (video, t) in enumerate(zip(videos, taus)):
+        ref = oracle.merge(video, t[0], t[1], want_feats=False)
+        np.testing.assert_array_equal(out.merge_map[v].cpu().numpy(), ref.merge_map)
+        np.testing.assert_array_equal(got[offs[v]:offs[v + 1]], oracle.merged_positions(ref.merge_map, ref.count))
+    short, status = binding.sttm_merged_positions(out.merge_map, out.out_offsets, rows - 5)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1 << 4                      # capacity exceeded, reported, not fatal
+    np.testing.assert_array_equal(short.cpu().numpy()[:offs[1] - 5], got[:offs[1] - 5])

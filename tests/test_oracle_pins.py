@@ -300,3 +300,19 @@ def test_generator_margins_match_the_stored_thresholds():
     assert r.count == fixed["count"]
     m = min(np.abs(r.spatial_sims - fixed["tau_s"]).min(), np.abs(r.tsim - fixed["tau_t"]).min())
     assert m >= 1e-4
+
+
+def test_merged_positions_closed_forms():
+    """Section 3.4, merged strategy: mean member index per row.  Hand values, the identity when
+    nothing merges, and the arithmetic-series mean when everything merges into one row."""
+    got = oracle.merged_positions(np.array([0, 0, 1, 2, 2, 2, 1]), 3)
+    assert got.dtype == np.float32
+    np.testing.assert_array_equal(got, np.array([0.5, 4.0, 4.0], dtype=np.float32))      # (0+1)/2, (2+6)/2, (3+4+5)/3
+    np.testing.assert_array_equal(oracle.merged_positions(np.arange(37), 37), np.arange(37, dtype=np.float32))
+    n = 1001
+    np.testing.assert_array_equal(oracle.merged_positions(np.zeros(n, dtype=np.int32), 1),
+                                  np.array([(n - 1) / 2.0], dtype=np.float32))
+    # against the merge itself: with tau >= 1 nothing merges, so the mean is the survived id
+    video = np.random.default_rng(5).standard_normal((3, 4, 4, 8)).astype(np.float32)
+    ref = oracle.merge(video, 2.0, 2.0, want_feats=False)
+    np.testing.assert_array_equal(oracle.merged_positions(ref.merge_map, ref.count), ref.out_pos.astype(np.float32))

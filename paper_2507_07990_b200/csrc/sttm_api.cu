@@ -451,15 +451,19 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
 template <typename OutT>
 sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacity, cudaStream_t st) {
     const Geo g = pl.g;
-    // one warp per row, striding; the row count is only known on the device, so the grid covers the
-    // most rows there can be, up to a few waves of blocks (most tokens merge: few rows, and blocks
-    // without a row would only cost their launch)
+    // kGatherParts warps per row, striding; the row count is only known on the device, so the grid
+    // covers the most rows there can be, up to a few waves of blocks (most tokens merge: few rows,
+    // and blocks without a row would only cost their launch)
     const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
-    const unsigned blocks = std::min<unsigned>(blocks_for(max_rows, 8), kSmCount * 16);
-    return launch_after(k_gather<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
-                        (const int32_t*)(ws + pl.row_anchor), (const int32_t*)(ws + pl.row_head),
-                        (const int32_t*)(ws + pl.piece_next), (const int32_t*)(ws + pl.row_weight),
-                        (const OutT*)(ws + pl.staging), (const float*)(ws + pl.pieces), (OutT*)out, capacity);
+    const unsigned blocks = std::min<unsigned>(blocks_for(max_rows * kGatherParts, 8), kSmCount * 16);
+    sttm_status s = launch_after(k_gather_rows<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
+                                 (const int32_t*)(ws + pl.row_anchor), (const int32_t*)(ws + pl.row_head),
+                                 (const OutT*)(ws + pl.staging), (OutT*)out, capacity);
+    if (s != STTM_OK) return s;
+    return launch_after(k_gather_pieces<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
+                        (const int32_t*)(ws + pl.row_head), (const int32_t*)(ws + pl.piece_next),
+                        (const int32_t*)(ws + pl.row_weight), (const float*)(ws + pl.pieces), (OutT*)out, capacity,
+                        pl.f.nitems * kPieceSlots);
 }
 
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }

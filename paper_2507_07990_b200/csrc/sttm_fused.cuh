@@ -1065,114 +1065,136 @@ k_piece_link(Geo g, int npieces, const int2* __restrict__ piece_meta, const int3
     atomicAdd(row_weight + row, m.y);
 }
 
-// One warp per output row: copy the staged row, or add the row's pieces in the order of
-// their index (a fixed order, so the result does not depend on scheduling).
+// Gather: kGatherParts warps per output row, each a contiguous share of the channels.  Two
+// kernels over the same rows, because the two kinds of row want different register budgets:
+// k_gather_rows copies the rows that are one finished staging row (bandwidth: many warps, few
+// registers), k_gather_pieces adds the pieces of the rows whose chains were cut by item borders,
+// in the order of their index (a fixed order, so the result does not depend on scheduling).  A row
+// of pieces is bound by the latency of its dependent loads (list head -> piece ids -> data), so
+// every warp issues all loads of its share before it adds anything.
+constexpr int kGatherParts = 4;
 template <typename OutT>
 __global__ void __launch_bounds__(256)
-k_gather(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict__ row_anchor,
-         const int32_t* __restrict__ row_head, const int32_t* __restrict__ piece_next,
-         const int32_t* __restrict__ row_weight, const OutT* __restrict__ staging, const float* __restrict__ pieces,
-         OutT* __restrict__ out, long long capacity) {
+k_gather_rows(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict__ row_anchor,
+              const int32_t* __restrict__ row_head, const OutT* __restrict__ staging, OutT* __restrict__ out,
+              long long capacity) {
     wait_for_prior_kernel();
     const int lane = threadIdx.x & 31;
-    const long long nrows = min(vid_off[g.B], capacity);
+    const long long nunits = min(vid_off[g.B], capacity) * kGatherParts;
     const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
-    const int n16 = (int)((size_t)g.D * sizeof(OutT) / 16);
-    for (long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < nrows; r += nwarps) {
+    const int n16 = (int)((size_t)g.D * sizeof(OutT) / 16);         // 16-byte pieces of a row
+    for (long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); unit < nunits; unit += nwarps) {
+        const long long r = unit / kGatherParts;
+        const int part = (int)(unit % kGatherParts);
+        if (row_head[r] >= 0) continue;                 // a row of pieces
+        int b = 0;                                      // video of the row: vid_off is short, walk it
+        while (b + 1 < g.B && vid_off[b + 1] <= r) b++;
+        const long long src = (long long)b * g.N + row_anchor[r];
+        const uint4* s4 = reinterpret_cast<const uint4*>(staging + src * g.D);
+        uint4* d4 = reinterpret_cast<uint4*>(out + r * g.D);
+        const int lo = (int)((long long)n16 * part / kGatherParts), hi = (int)((long long)n16 * (part + 1) / kGatherParts);
+        for (int i0 = lo; i0 < hi; i0 += 4 * 32) {      // four loads in flight per lane
+            uint4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                const int i = i0 + k * 32 + lane;
+                if (i < hi) v[k] = __ldcs(s4 + i);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                const int i = i0 + k * 32 + lane;
+                if (i < hi) __stcs(d4 + i, v[k]);
+            }
+        }
+    }
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+k_gather_pieces(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict__ row_head,
+                const int32_t* __restrict__ piece_next, const int32_t* __restrict__ row_weight,
+                const float* __restrict__ pieces, OutT* __restrict__ out, long long capacity, int max_pieces) {
+    wait_for_prior_kernel();
+    const int lane = threadIdx.x & 31;
+    const long long nunits = min(vid_off[g.B], capacity) * kGatherParts;
+    const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+    const int nf4 = g.D / VEC;                                      // 4-channel groups of a row
+    for (long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); unit < nunits; unit += nwarps) {
+        const long long r = unit / kGatherParts;
+        const int part = (int)(unit % kGatherParts);
         const int head = row_head[r];
-        if (head < 0) {
-            int b = 0;                                  // video of the row: vid_off is short, walk it
-            while (b + 1 < g.B && vid_off[b + 1] <= r) b++;
-            const long long src = (long long)b * g.N + row_anchor[r];
-            const uint4* s4 = reinterpret_cast<const uint4*>(staging + src * g.D);
-            uint4* d4 = reinterpret_cast<uint4*>(out + r * g.D);
-            for (int i0 = 0; i0 < n16; i0 += 8 * 32) {  // eight loads in flight per lane
-                uint4 v[8];
+        if (head < 0) continue;                         // a finished staging row
+        // the row's pieces in increasing index order; lists are short (a few per item border):
+        // one walk that keeps the first eight sorted in registers (the walk also stops after as
+        // many steps as there are pieces at all, whatever the list holds)
+        constexpr int kMaxList = 8;
+        int ids[kMaxList];
+        int n = 0, steps = 0;
+        bool longer = false;
+        for (int pc = head; pc >= 0 && steps < max_pieces; pc = piece_next[pc], steps++) {
+            if (n == kMaxList) { longer = true; break; }
+            int v = pc;
 #pragma unroll
-                for (int k = 0; k < 8; k++) {
-                    const int i = i0 + k * 32 + lane;
-                    if (i < n16) v[k] = __ldcs(s4 + i);
-                }
-#pragma unroll
-                for (int k = 0; k < 8; k++) {
-                    const int i = i0 + k * 32 + lane;
-                    if (i < n16) __stcs(d4 + i, v[k]);
+            for (int k = 0; k < kMaxList; k++) {
+                if (k < n) {
+                    const int lo = min(ids[k], v);
+                    v = max(ids[k], v);
+                    ids[k] = lo;
+                } else if (k == n) {
+                    ids[k] = v;
                 }
             }
-        } else {
-            // the row's pieces in increasing index order; lists are short (a few per item border):
-            // one walk that keeps the first eight sorted in registers
-            constexpr int kMaxList = 8;
-            int ids[kMaxList];
-            int n = 0;
-            bool longer = false;
-            for (int pc = head; pc >= 0; pc = piece_next[pc]) {
-                if (n == kMaxList) { longer = true; break; }
-                int v = pc;
+            n++;
+        }
+        const float wsum = (float)row_weight[r];
+        const int lo = (int)((long long)nf4 * part / kGatherParts), hi = (int)((long long)nf4 * (part + 1) / kGatherParts);
+        // eight groups per trip (a quarter of a 3584-channel row is seven): 8 x n loads in flight
+        for (int f0 = lo + lane; f0 < hi; f0 += 8 * 32) {
+            float sum[8][VEC];
+#pragma unroll
+            for (int u = 0; u < 8; u++)
+#pragma unroll
+                for (int v = 0; v < VEC; v++) sum[u][v] = 0.f;
+            if (!longer) {
 #pragma unroll
                 for (int k = 0; k < kMaxList; k++) {
                     if (k < n) {
-                        const int lo = min(ids[k], v);
-                        v = max(ids[k], v);
-                        ids[k] = lo;
-                    } else if (k == n) {
-                        ids[k] = v;
+                        const float4* src = reinterpret_cast<const float4*>(pieces + (long long)ids[k] * g.D);
+                        float4 v[8];
+#pragma unroll
+                        for (int u = 0; u < 8; u++)
+                            if (f0 + u * 32 < hi) v[u] = __ldcs(src + f0 + u * 32);
+#pragma unroll
+                        for (int u = 0; u < 8; u++)
+                            if (f0 + u * 32 < hi) {
+                                sum[u][0] += v[u].x; sum[u][1] += v[u].y; sum[u][2] += v[u].z; sum[u][3] += v[u].w;
+                            }
                     }
                 }
-                n++;
-            }
-            const float wsum = (float)row_weight[r];
-            // four 128-channel groups per trip, so that 4 x n loads are in flight
-            for (int d0 = lane * VEC; d0 < g.D; d0 += 4 * kSliceCh) {
-                float sum[4][VEC];
+            } else {
+                int lst = -1;
+                for (int round = 0; round < max_pieces; round++) {
+                    int best = 0x7fffffff, hops = 0;
+                    for (int pc = head; pc >= 0 && hops < max_pieces; pc = piece_next[pc], hops++)
+                        if (pc > lst && pc < best) best = pc;
+                    if (best == 0x7fffffff) break;
+                    const float4* src = reinterpret_cast<const float4*>(pieces + (long long)best * g.D);
 #pragma unroll
-                for (int u = 0; u < 4; u++)
-#pragma unroll
-                    for (int v = 0; v < VEC; v++) sum[u][v] = 0.f;
-                if (!longer) {
-#pragma unroll
-                    for (int k = 0; k < kMaxList; k++) {
-                        if (k < n) {
-                            const float* src = pieces + (long long)ids[k] * g.D;
-#pragma unroll
-                            for (int u = 0; u < 4; u++) {
-                                const int d = d0 + u * kSliceCh;
-                                if (d < g.D) {
-                                    const float4 v = __ldcs(reinterpret_cast<const float4*>(src + d));
-                                    sum[u][0] += v.x; sum[u][1] += v.y; sum[u][2] += v.z; sum[u][3] += v.w;
-                                }
-                            }
+                    for (int u = 0; u < 8; u++)
+                        if (f0 + u * 32 < hi) {
+                            const float4 v = src[f0 + u * 32];
+                            sum[u][0] += v.x; sum[u][1] += v.y; sum[u][2] += v.z; sum[u][3] += v.w;
                         }
-                    }
-                } else {
-                    int lst = -1;
-                    while (true) {
-                        int best = 0x7fffffff;
-                        for (int pc = head; pc >= 0; pc = piece_next[pc])
-                            if (pc > lst && pc < best) best = pc;
-                        if (best == 0x7fffffff) break;
-                        const float* src = pieces + (long long)best * g.D;
-#pragma unroll
-                        for (int u = 0; u < 4; u++) {
-                            const int d = d0 + u * kSliceCh;
-                            if (d < g.D) {
-                                const float4 v = *reinterpret_cast<const float4*>(src + d);
-                                sum[u][0] += v.x; sum[u][1] += v.y; sum[u][2] += v.z; sum[u][3] += v.w;
-                            }
-                        }
-                        lst = best;
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; u++) {
-                    const int d = d0 + u * kSliceCh;
-                    if (d < g.D) {
-#pragma unroll
-                        for (int v = 0; v < VEC; v++) sum[u][v] = sum[u][v] / wsum;
-                        store4(out + r * g.D + d, sum[u]);
-                    }
+                    lst = best;
                 }
             }
+#pragma unroll
+            for (int u = 0; u < 8; u++)
+                if (f0 + u * 32 < hi) {
+#pragma unroll
+                    for (int v = 0; v < VEC; v++) sum[u][v] = sum[u][v] / wsum;
+                    store4(out + r * g.D + (long long)(f0 + u * 32) * VEC, sum[u]);
+                }
         }
     }
 }

@@ -424,6 +424,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.out_f32 = p->out_dtype == STTM_F32;
     fp.cover = (int8_t*)(ws + pl.cover);
     fp.link = (int32_t*)(ws + pl.link);
+    fp.frame_roots = (int32_t*)(ws + pl.frame_counts);   // inside the region that is cleared before every call
     fp.chain_key = (int32_t*)(ws + pl.cell_row);       // the three-pass kernels' cell_row array is free here
     fp.staging = ws + pl.staging;
     fp.pieces = (float*)(ws + pl.pieces);
@@ -661,14 +662,11 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
                          (const int32_t*)(ws + pl.cell_row), root, device_status);
         if (s != STTM_OK) return s;
         mark_stage(2, st);
-        int32_t* frame_roots = (int32_t*)(ws + pl.frame_roots);
+        int32_t* frame_roots = (int32_t*)(ws + pl.frame_counts);     // counted by the fused kernel
         int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
         long long* vid_off = (long long*)(ws + pl.vid_off);
         int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
         int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
-        s = launch_after(k_frame_roots, (unsigned)(g.B * g.T), 256, st, g, (const int8_t*)cover, (const int32_t*)link,
-                         frame_roots);
-        if (s != STTM_OK) return s;
         s = launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)frame_roots, frame_base, out_count, vid_off,
                          out_offsets);
         if (s != STTM_OK) return s;

@@ -91,6 +91,7 @@ struct FusedParams {
     int8_t* cover;
     int32_t* link;
     int32_t* chain_key;      // [B*N] per cell: root cell id of its chain as far as the item knows it
+    int32_t* frame_roots;    // [B*T] chains that start in a frame (= its output rows), zero on entry
     void* staging;           // [B*N][D] rows of the output dtype
     float* pieces;           // [nitems][kPieceSlots][D]
     int2* piece_meta;        // [nitems][kPieceSlots] {key cell id or -1, weight}
@@ -873,6 +874,8 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const uint32_t dead = active_slots & ~memb;
                 const uint32_t freem = ~memb & 0xffffu;
                 const uint32_t freshm = __ballot_sync(full, fresh && low);
+                // every new chain is an output row of this frame (the ordering needs the count per frame)
+                if (rank == 0 && lane == 0 && !is_halo && freshm != 0) atomicAdd(p.frame_roots + it.b * p.T + t, __popc(freshm));
                 const int slot_fresh = kth_set_bit16(freem, __popc(freshm & ((1u << c) - 1)));
                 const int node_slot = linked ? slot_linked : slot_fresh;
                 const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + lane_anchor(lg, c, lv));

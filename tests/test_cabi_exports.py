@@ -35,3 +35,18 @@ def test_host_only_entry_points():
     assert binding.sttm_workspace_bytes(bad) == 0
     lib = binding.load_library()
     assert lib.sttm_status_string(2) == b"unsupported shape"
+
+
+def test_merged_positions_argument_checks_need_no_gpu():
+    import ctypes as C
+    lib = binding.load_library()
+    assert lib.sttm_merged_positions_workspace(0) == 0
+    need = lib.sttm_merged_positions_workspace(1000)
+    assert need >= 1000 * 12 and need % 4 == 0
+    # null pointers, bad sizes, a workspace that is too small: refused on the host, nothing launched
+    assert lib.sttm_merged_positions(None, None, 1, 10, None, 0, None, 10, None, None) == 1       # STTM_ERR_ARG
+    buf = (C.c_char * 4096)()
+    addr = (C.addressof(buf) + 255) // 256 * 256
+    assert lib.sttm_merged_positions(addr, addr, 0, 10, addr, 2048, addr, 10, None, None) == 1
+    assert lib.sttm_merged_positions(addr, addr, 1, 10, addr + 4, 2048, addr, 10, None, None) == 1   # misaligned ws
+    assert lib.sttm_merged_positions(addr, addr, 1, 10, addr, 16, addr, 10, None, None) == 3        # STTM_ERR_WORKSPACE

@@ -953,8 +953,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             __syncwarp();
             if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
         }
-    } else if (warp == w_prod) {
-        // ----------------------------------- producer warp -----------------------------------
+    } else if (warp == w_prod || (warp == w_prod + 1 && p.RB == 0)) {
+        // ---------------------------------- producer warps ----------------------------------
+        // Issuing one bulk copy costs a warp some 80 cycles, and a frame is 16 of them, so two
+        // warps share the rows (with a second ring the second warp has that ring to fill, and
+        // this one issues all 16).
+        const int nprod = p.RB == 0 ? 2 : 1, which = warp - w_prod;
+        const int row = lane * nprod + which;              // the tile row this lane copies
         int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
@@ -962,12 +967,14 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const uint32_t bar = full_bar + 8 * s;
                 if (use >= 1 && !mbar_wait(empty_bar + 8 * s, use - 1, timed_out)) break;
                 __syncwarp();
-                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
+                // (one warp announces the bytes of the whole frame; a copy of the other warp that lands
+                // before that only makes the count run negative for a moment)
+                if (lane == 0 && which == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
                 __syncwarp();
-                if (lane < 16 && ((it.vmask >> lane) & 1u)) {
+                if (row < 16 && ((it.vmask >> row) & 1u)) {
                     const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
-                                           p.tiles[it.tile].y[lane] * p.W + p.tiles[it.tile].x[lane];
-                    bulk_g2s(ring_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
+                                           p.tiles[it.tile].y[row] * p.W + p.tiles[it.tile].x[row];
+                    bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * p.D + rank * p.S,
                              (uint32_t)(p.S * 2), bar);
                 }
                 if (++s == p.R) { s = 0; use++; }

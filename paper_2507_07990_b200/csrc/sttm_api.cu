@@ -136,7 +136,7 @@ void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
     f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
     f->slot_bytes = 16 * f->row_bytes;
     const size_t fixed = (size_t)f->NM * kGramVals * 4 + kGramVals * 4 + (size_t)kRecRing * C * kSumVals * 4 +
-                         16 * 32 * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) + 16 +
+                         128 + kRecRing * kSumVals * 4 + kRecRing * 16 * 4 + sizeof(SlotTable) + kRecRing * sizeof(FrameRec) + 16 +
                          (4 * kMaxRing + 6 * kRecRing + 4) * 8;
     // the slots that fit: one ring in which a frame stays until the sum warps have used it, or,
     // on request, shared out between the Gram warps' ring (a frame stays for its own products and

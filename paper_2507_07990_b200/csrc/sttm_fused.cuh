@@ -849,6 +849,17 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     mbar_arrive(hfull_bar + 8 * (q % kRecRing));
                     if (two) mbar_arrive(hfull_bar + 8 * ((q + 1) % kRecRing));
                 }
+                // cover map and links go out from here, after the hand-over: this warp has more slack
+                // than the chain warp, whose time per frame weighs most on the pipeline
+                {
+                    const int lcell = __shfl_sync(full, lg.cell, 16 * half + (link_local < 0 ? 0 : link_local));
+                    const int tt = it.tstart + j + half;
+                    if (rank == 0 && mine && valid && !(it.halo && j + half == 0)) {
+                        const long long gcc = (long long)it.b * p.N + (long long)tt * p.HW + lg.cell;
+                        p.cover[gcc] = (int8_t)lv;
+                        p.link[gcc] = link_local < 0 ? -1 : (tt - 1) * p.HW + lcell;
+                    }
+                }
                 q += two ? 2 : 1;
                 if (lane == 0) *reinterpret_cast<volatile int*>(hint) = q;
             }
@@ -902,7 +913,6 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const uint32_t cells = lane_region(lg, c, lv);
                 const int wint = p.weight_mode ? __popc(cells) : 1;
                 const long long gc = (long long)it.b * p.N + (long long)t * p.HW + lg.cell;
-                const int link_cell = __shfl_sync(full, lg.cell, link_local < 0 ? 0 : link_local);
 
                 // chains that ended: lane s looks at slot s (before the slot is given away again); at
                 // the first frame of an item nothing of the item runs yet and the list is the carry
@@ -943,8 +953,6 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
 
                 if (rank == 0 && !is_halo && low && valid) {
-                    p.cover[gc] = (int8_t)lv;
-                    p.link[gc] = link_local < 0 ? -1 : (t - 1) * p.HW + link_cell;
                     p.chain_key[gc] = tab->key[cur_slot] - it.b * p.N;
                 }
                 if (is_last) {

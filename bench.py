@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on the qwen workload;
 # a streaming kernel's traffic grows in proportion to the bytes it must move, so the ratio is
 # applied to the benchmark workload's algorithmic bytes).  Absent = no capture of the current kernel.
-NCU_TRAFFIC_RATIO = {"fused": 0.944}
+NCU_TRAFFIC_RATIO = {"fused": 0.946}
 
 
 def workload_setup(name: str):

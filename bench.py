@@ -185,9 +185,14 @@ def run_ours(args):
     view = h_feats.view(torch.int16).numpy().view(np.uint16) if spec.dtype == "bf16" else h_feats.numpy()
     inputs.make_video(spec, out=view[0])
     d_feats = h_feats.cuda()
-    plan = binding.MergePlan((1, spec.T, spec.H, spec.W, spec.D), tdtype, th["tau_s"], th["tau_t"],
-                             out_dtype=torch.bfloat16, want_map=False,
-                             match=binding.MATCH_BEST if args.match == "best" else binding.MATCH_TOPLEFT)
+    if args.budget_rows > 0:
+        # budget mode: tau_t chosen on the device for this many rows (two passes of the fused kernel)
+        plan = binding.BudgetPlan((1, spec.T, spec.H, spec.W, spec.D), tdtype, th["tau_s"], args.budget_rows,
+                                  out_dtype=torch.bfloat16, want_map=False)
+    else:
+        plan = binding.MergePlan((1, spec.T, spec.H, spec.W, spec.D), tdtype, th["tau_s"], th["tau_t"],
+                                 out_dtype=torch.bfloat16, want_map=False,
+                                 match=binding.MATCH_BEST if args.match == "best" else binding.MATCH_TOPLEFT)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
 
     def barrier():
@@ -307,7 +312,7 @@ def run_ours(args):
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": dict(workload_config(args.workload, spec, th, key),
-                               match=args.match,
+                               match=args.match, budget_rows=args.budget_rows,
                                launch=("3 of 4 steps replay a CUDA graph of the library call, every 4th is the call "
                                        "itself with stage events") if graph is not None else "library calls"),
                 "out_rows": count,
@@ -335,6 +340,8 @@ def main():
                     help="frames per step of the --impl reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="every timed step is a direct library call")
+    ap.add_argument("--budget-rows", type=int, default=0,
+                    help="time the budget mode (sttm_merge_budget) with this row budget instead of fixed thresholds")
     ap.add_argument("--match", default="topleft", choices=["topleft", "best"],
                     help="destination rule of the temporal link (the paper's default, or its most-similar variant)")
     ap.add_argument("--tuning", default="0,0,0",

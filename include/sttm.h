@@ -172,6 +172,28 @@ sttm_status sttm_merge_host(const void* h_feats, const sttm_params* p,
                             int32_t* h_out_count, int64_t* h_out_offsets, int32_t* h_device_status);
 
 /*
+ * Budget mode (the adaptive thresholds the paper leaves to future work in its limitations): tau_s
+ * as given in *p, tau_t chosen per video on the device so that the video keeps at most
+ * budget_rows[v] rows.  With the cover maps fixed, a kept node is merged into the frame before iff
+ * the largest cosine to its candidates exceeds tau_t, so the row count is nodes - #{best cosine >
+ * tau_t}; the threshold returned is the middle of the gap between the k-th and the (k+1)-th largest
+ * best cosine, k = nodes - budget (2.0 when the spatial stage alone meets the budget; -2.0, and
+ * more rows than asked for, when even linking every node that has a candidate does not).  Equal
+ * best cosines at the cut leave the count off by their number.  Runs the fused kernel twice
+ * (once to collect the best cosines, once to merge); only for shapes the fused kernel covers
+ * (STTM_ERR_UNSUPPORTED otherwise); tau_t / tau_t_per_video of *p are ignored.
+ *   budget_rows  host, [B]: rows allowed per video (>= 1)
+ *   ws           at least sttm_budget_workspace_bytes(p) bytes, 256-byte aligned
+ *   tau_t_out    [B] float32, may be NULL: the thresholds chosen
+ * Other arguments as sttm_merge_ex.  Asynchronous on `stream`.
+ */
+size_t sttm_budget_workspace_bytes(const sttm_params* p);
+sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const long long* budget_rows, void* ws,
+                              size_t ws_bytes, void* out_feats, int32_t* out_pos, int32_t* merge_map,
+                              int32_t* out_count, int64_t* out_offsets, float* tau_t_out, int32_t* device_status,
+                              void* stream);
+
+/*
  * "Merged" position strategy of Section 3.4 (the first of its three ways to give a merged token a
  * rotary position): the position of an output row is the average of the positions of the tokens
  * merged into it.  Reading taken here: the position of an input token is its index t*H*W + y*W + x

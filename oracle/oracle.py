@@ -165,3 +165,31 @@ def merged_positions(merge_map: np.ndarray, count: int) -> np.ndarray:
         sums[r] += i
         cnts[r] += 1
     return (sums.astype(np.float64) / cnts.astype(np.float64)).astype(np.float32)
+
+
+def best_candidate_cosines(feats: np.ndarray, tau_s: float, lv1: int = 4):
+    """(number of kept nodes, descending array with, for every kept node that has candidates in
+    the frame before it, the largest cosine to them) under the cover maps that ``tau_s`` gives."""
+    base = merge(feats, tau_s, 2.0, lv1=lv1, want_feats=False, want_pairs=True)
+    best = {}
+    for v, sim in zip(base.tsim_v.tolist(), base.tsim.tolist()):
+        best[v] = max(best.get(v, -2.0), sim)
+    return base.count, np.sort(np.array(list(best.values()), dtype=np.float64))[::-1]
+
+
+def budget_tau_t(feats: np.ndarray, tau_s: float, budget_rows: int, lv1: int = 4):
+    """Budget mode (the adaptive threshold the paper names as future work): with the cover maps
+    fixed by ``tau_s``, a kept node is merged into the frame before iff the largest cosine to its
+    candidates exceeds tau_t, so the row count is nodes - #{best cosine > tau_t}.  Returns
+    (tau_t, gap): the middle of the gap between the k-th and the (k+1)-th largest best cosine,
+    k = nodes - budget, and the width of that gap; (2.0, inf) when no temporal merging is needed,
+    (-2.0, 0) when the budget cannot be met.  Plain definition on top of ``merge``."""
+    nodes, m = best_candidate_cosines(feats, tau_s, lv1)
+    k = nodes - int(budget_rows)
+    if k <= 0:
+        return 2.0, float("inf")
+    if k > len(m):
+        return -2.0, 0.0
+    mk = m[k - 1]
+    mk1 = m[k] if k < len(m) else mk - 2e-3
+    return 0.5 * (mk + mk1), float(mk - mk1)

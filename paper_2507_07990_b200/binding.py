@@ -28,7 +28,7 @@ EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame",
            "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
            "sttm_set_stage_events", "sttm_set_tuning", "sttm_set_ring_split", "sttm_last_path",
            "sttm_fused_launch_shape", "sttm_spatial_static", "sttm_merged_positions",
-           "sttm_merged_positions_workspace"]
+           "sttm_merged_positions_workspace", "sttm_merge_budget", "sttm_budget_workspace_bytes"]
 
 
 class SttmParams(C.Structure):
@@ -89,6 +89,11 @@ def load_library(path: Optional[str] = None):
     lib.sttm_set_stage_events.restype = None
     lib.sttm_set_tuning.argtypes = [C.c_int, C.c_int, C.c_int]
     lib.sttm_set_tuning.restype = None
+    lib.sttm_budget_workspace_bytes.argtypes = [pp]
+    lib.sttm_budget_workspace_bytes.restype = C.c_size_t
+    lib.sttm_merge_budget.argtypes = [C.c_void_p, pp, C.POINTER(C.c_longlong), C.c_void_p, C.c_size_t, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.sttm_merge_budget.restype = C.c_int
     lib.sttm_merged_positions_workspace.argtypes = [C.c_longlong]
     lib.sttm_merged_positions_workspace.restype = C.c_size_t
     lib.sttm_merged_positions.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_longlong, C.c_void_p, C.c_size_t,
@@ -289,6 +294,50 @@ def sttm_merge_ex(feats: torch.Tensor, tau_s, tau_t, lv1: int = 4, out_dtype: to
     plan = MergePlan(tuple(feats.shape), feats.dtype, tau_s, tau_t, lv1, out_dtype, pos, wt, capacity, want_map,
                      feats.device, match)
     return plan.run(feats)
+
+
+class BudgetPlan:
+    """Pre-allocated buffers for repeated sttm_merge_budget calls on one problem shape."""
+
+    def __init__(self, shape, in_dtype, tau_s, budget_rows, lv1=4, out_dtype=torch.bfloat16, want_map=False,
+                 device="cuda"):
+        B, T, H, W, D = shape
+        self.problem = make_params(shape, in_dtype, tau_s, 2.0, lv1, out_dtype)
+        p = self.problem.params
+        lib = load_library()
+        need = int(lib.sttm_budget_workspace_bytes(C.byref(p)))
+        if need == 0:
+            raise SttmError(2, "sttm_budget_workspace_bytes")
+        ws = torch.empty(need + 256, dtype=torch.uint8, device=device)
+        self.ws = ws[(-ws.data_ptr()) % 256:]
+        cap = int(p.out_capacity_rows)
+        self.out_feats = torch.empty((cap, D), dtype=out_dtype, device=device)
+        self.out_pos = torch.empty((cap,), dtype=torch.int32, device=device)
+        self.out_count = torch.empty((B,), dtype=torch.int32, device=device)
+        self.out_offsets = torch.empty((B + 1,), dtype=torch.int64, device=device)
+        self.merge_map = torch.empty((B, T * H * W), dtype=torch.int32, device=device) if want_map else None
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.tau = torch.empty((B,), dtype=torch.float32, device=device)
+        rows = budget_rows if hasattr(budget_rows, "__len__") else [budget_rows] * B
+        self.budgets = (C.c_longlong * B)(*[int(v) for v in rows])
+
+    def run(self, feats: torch.Tensor) -> MergeOutput:
+        lib = load_library()
+        _check(lib.sttm_merge_budget(_ptr(feats), C.byref(self.problem.params), self.budgets, _ptr(self.ws),
+                                     self.ws.numel(), _ptr(self.out_feats), _ptr(self.out_pos), _ptr(self.merge_map),
+                                     _ptr(self.out_count), _ptr(self.out_offsets), _ptr(self.tau), _ptr(self.status),
+                                     _stream()), "sttm_merge_budget")
+        return MergeOutput(self.out_feats, self.out_pos, self.out_count, self.out_offsets, self.merge_map,
+                           self.status, int(lib.sttm_last_launch_count()))
+
+
+def sttm_merge_budget(feats: torch.Tensor, tau_s: float, budget_rows, lv1: int = 4,
+                      out_dtype: torch.dtype = torch.bfloat16, want_map: bool = True):
+    """Budget mode: tau_s as given, tau_t chosen per video on the device so that video v keeps at
+    most ``budget_rows[v]`` rows.  Returns (MergeOutput, tau_t [B] float32 on the device)."""
+    feats = _as5d(feats)
+    plan = BudgetPlan(tuple(feats.shape), feats.dtype, tau_s, budget_rows, lv1, out_dtype, want_map, feats.device)
+    return plan.run(feats), plan.tau
 
 
 def sttm_merged_positions(merge_map: torch.Tensor, out_offsets: torch.Tensor, rows: int):

@@ -20,6 +20,8 @@ using namespace sttm;
 constexpr int kSmCount = 148;   // B200; the library is built for sm_100a only
 
 thread_local int g_launches = 0;
+thread_local float* g_budget_tmax = nullptr;           // set by sttm_merge_budget around its two passes
+thread_local const float* g_budget_tau_dev = nullptr;
 thread_local cudaEvent_t* g_stage_events = nullptr;   // when set: event i is recorded after stage i-1
 
 constexpr int kStageCount = 5;
@@ -424,6 +426,8 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.out_f32 = p->out_dtype == STTM_F32;
     fp.cover = (int8_t*)(ws + pl.cover);
     fp.link = (int32_t*)(ws + pl.link);
+    fp.tmax = g_budget_tmax;
+    fp.tau_t_dev = g_budget_tau_dev;
     fp.frame_roots = (int32_t*)(ws + pl.frame_counts);   // inside the region that is cleared before every call
     fp.chain_key = (int32_t*)(ws + pl.cell_row);       // the three-pass kernels' cell_row array is free here
     fp.staging = ws + pl.staging;
@@ -658,6 +662,11 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
         s = run_fused(feats, p, pl, ws, device_status, st);
         if (s != STTM_OK) return s;
         mark_stage(1, st);
+        if (g_budget_tmax != nullptr) {
+            // first pass of the budget mode: only the node counts per video are needed
+            return launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)(ws + pl.frame_counts),
+                                (int32_t*)(ws + pl.frame_base), out_count, (long long*)(ws + pl.vid_off), out_offsets);
+        }
         s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, pl.f.nseg + 1,
                          (const int32_t*)(ws + pl.cell_row), root, device_status);
         if (s != STTM_OK) return s;
@@ -752,6 +761,55 @@ sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_
     }
     return sttm_merge_ex(feats, &p, c.ws, c.ws_bytes, out_feats, out_pos, nullptr, out_count, nullptr, nullptr,
                          stream);
+}
+
+size_t sttm_budget_workspace_bytes(const sttm_params* p) {
+    Plan pl;
+    if (make_plan(p, &pl) != STTM_OK || !pl.f.ok) return 0;
+    return (pl.total + 255) / 256 * 256 + ((size_t)pl.cells * 4 + 255) / 256 * 256 + 256;
+}
+
+sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const long long* budget_rows, void* ws,
+                              size_t ws_bytes, void* out_feats, int32_t* out_pos, int32_t* merge_map,
+                              int32_t* out_count, int64_t* out_offsets, float* tau_t_out, int32_t* device_status,
+                              void* stream) {
+    Plan pl;
+    sttm_status s = make_plan(p, &pl);
+    if (s != STTM_OK) return s;
+    if (!pl.f.ok) return STTM_ERR_UNSUPPORTED;
+    if (!budget_rows || !ws || !out_count) return STTM_ERR_ARG;
+    for (int b = 0; b < p->B; b++)
+        if (budget_rows[b] < 1) return STTM_ERR_ARG;
+    if (ws_bytes < sttm_budget_workspace_bytes(p)) return STTM_ERR_WORKSPACE;
+    char* base = (char*)ws;
+    const size_t main_bytes = (pl.total + 255) / 256 * 256;
+    float* tmax = (float*)(base + main_bytes);
+    float* tau_dev = (float*)(base + main_bytes + ((size_t)pl.cells * 4 + 255) / 256 * 256);
+    cudaStream_t st = (cudaStream_t)stream;
+    // first pass: no temporal merging (tau_t = 2), every kept node reports its best candidate
+    sttm_params q = *p;
+    q.tau_t = 2.f;
+    q.tau_t_per_video = nullptr;
+    g_budget_tmax = tmax;
+    g_budget_tau_dev = nullptr;
+    s = sttm_merge_ex(feats, &q, ws, main_bytes, out_feats, out_pos, nullptr, out_count, out_offsets, device_status,
+                      stream);
+    g_budget_tmax = nullptr;
+    if (s != STTM_OK) return s;
+    Budgets bd = {};
+    for (int b = 0; b < p->B; b++) bd.rows[b] = budget_rows[b];
+    s = launch_after(k_budget_tau, (unsigned)p->B, 1024, st, (long long)pl.g.N, (const float*)tmax,
+                     (const int32_t*)out_count, bd, tau_dev);
+    if (s != STTM_OK) return s;
+    // second pass: the whole path with the thresholds read from device memory
+    g_budget_tau_dev = tau_dev;
+    s = sttm_merge_ex(feats, p, ws, main_bytes, out_feats, out_pos, merge_map, out_count, out_offsets, device_status,
+                      stream);
+    g_budget_tau_dev = nullptr;
+    if (s != STTM_OK) return s;
+    if (tau_t_out != nullptr)
+        STTM_CUDA_TRY(cudaMemcpyAsync(tau_t_out, tau_dev, sizeof(float) * p->B, cudaMemcpyDeviceToDevice, st));
+    return STTM_OK;
 }
 
 size_t sttm_merged_positions_workspace(long long capacity_rows) {

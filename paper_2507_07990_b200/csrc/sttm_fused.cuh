@@ -94,6 +94,9 @@ struct FusedParams {
     int32_t* link;
     int32_t* chain_key;      // [B*N] per cell: root cell id of its chain as far as the item knows it
     int32_t* frame_roots;    // [B*T] chains that start in a frame (= its output rows), zero on entry
+    float* tmax;             // budget mode, may be null: [B*N] per cell, at the top-left cell of a kept node the
+                             // largest cosine to its candidates in the frame before, -2 elsewhere / without one
+    const float* tau_t_dev;  // budget mode, may be null: [B] temporal thresholds in device memory
     void* staging;           // [B*N][D] rows of the output dtype
     float* pieces;           // [nitems][kPieceSlots][D]
     int2* piece_meta;        // [nitems][kPieceSlots] {key cell id or -1, weight}
@@ -745,7 +748,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const uint32_t xchg_a = smem_u32(xchg);
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
-            const float tau_s = taus.s[it.b], tau_t = taus.t[it.b];
+            const float tau_s = taus.s[it.b], tau_t = p.tau_t_dev != nullptr ? p.tau_t_dev[it.b] : taus.t[it.b];
             const LaneGeo lg = lane_geo(p.tiles[it.tile], c, L, p.W);
             const float w1 = lg.w1, w2 = lg.w2;
             const bool valid = lg.valid;
@@ -830,6 +833,21 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                             const float si = __shfl_sync(full, cosv, 16 * half + i);
                             if (((cand >> i) & 1u) && si > best) { best = si; cstar = i; }
                         }
+                    }
+                    if (p.tmax != nullptr) {
+                        // budget mode: the number of rows as a function of tau_t only needs, per kept node,
+                        // the largest cosine to its candidates (the node is linked iff that exceeds tau_t)
+                        const float cosv = rep ? ((nk == 0.f || pnk == 0.f) ? 0.f : dot / (sqrtf(nk) * sqrtf(pnk))) : -2.f;
+                        const uint32_t candm = ((__ballot_sync(full, rep) >> (16 * half)) & 0xffffu) & lane_region(lg, c, lv);
+                        float most = -2.f;
+#pragma unroll
+                        for (int i = 0; i < 16; i++) {
+                            const float si = __shfl_sync(full, cosv, 16 * half + i);
+                            if (((candm >> i) & 1u) && si > most) most = si;
+                        }
+                        if (rank == 0 && mine && valid && !(it.halo && j + half == 0))
+                            p.tmax[(long long)it.b * p.N + (long long)(it.tstart + j + half) * p.HW + lg.cell] =
+                                lane_anchor(lg, c, lv) == c ? most : -2.f;
                     }
                     const int lu_star = __shfl_sync(full, lu, 16 * half + cstar);
                     link_local = cand ? lane_anchor(lg, cstar, lu_star) : -1;      // same sub-tile: same bits
@@ -1267,6 +1285,90 @@ k_merge_map(Geo g, const int32_t* __restrict__ root, const int32_t* __restrict__
     if (i >= (long long)g.B * g.N) return;
     const long long vb = i / g.N * g.N;
     merge_map[i] = row_at_root[vb + root[i]];
+}
+
+// ---------------------------------------------------------------------------------
+// Budget mode: the temporal threshold that leaves at most `budget` rows.  With the cover maps
+// fixed (tau_s), a kept node is merged into the frame before iff the largest cosine m to its
+// candidates exceeds tau_t, so rows(tau_t) = nodes - #{m > tau_t}: the threshold is put in the
+// middle of the gap between the k-th and the (k+1)-th largest m, k = nodes - budget.  One block
+// per video; the k-th largest value by three histogram passes over the order-preserving bit
+// pattern of the floats.
+// ---------------------------------------------------------------------------------
+struct Budgets { long long rows[kMaxBatch]; };
+
+__device__ __forceinline__ uint32_t float_key(float f) {
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// k-th largest (k >= 1) of the values > -1.5 among v[0..n); the caller made sure there are at least k
+__device__ float block_kth_largest(const float* __restrict__ v, long long n, long long k, uint32_t* hist) {
+    __shared__ uint32_t s_prefix, s_mask;
+    __shared__ long long s_k;
+    if (threadIdx.x == 0) { s_prefix = 0; s_mask = 0; s_k = k; }
+    __syncthreads();
+    const int shifts[3] = {21, 10, 0}, bits[3] = {11, 11, 10};
+    for (int pass = 0; pass < 3; pass++) {
+        const int nb = 1 << bits[pass];
+        for (int i = threadIdx.x; i < 2048; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix, mask = s_mask;
+        for (long long i = threadIdx.x; i < n; i += blockDim.x) {
+            const float f = v[i];
+            if (f > -1.5f) {
+                const uint32_t key = float_key(f);
+                if ((key & mask) == prefix) atomicAdd(&hist[(key >> shifts[pass]) & (nb - 1)], 1u);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            long long kk = s_k;
+            int b = nb - 1;
+            for (; b > 0; b--) {               // from the largest bin down
+                if ((long long)hist[b] >= kk) break;
+                kk -= hist[b];
+            }
+            s_k = kk;
+            s_prefix = prefix | ((uint32_t)b << shifts[pass]);
+            s_mask = mask | ((uint32_t)(nb - 1) << shifts[pass]);
+        }
+        __syncthreads();
+    }
+    return key_float(s_prefix);
+}
+
+__global__ void __launch_bounds__(1024)
+k_budget_tau(long long N, const float* __restrict__ tmax, const int32_t* __restrict__ nodes, Budgets budgets,
+             float* __restrict__ tau_t) {
+    wait_for_prior_kernel();
+    __shared__ uint32_t hist[2048];
+    __shared__ long long s_cand;
+    const int b = blockIdx.x;
+    const float* v = tmax + (long long)b * N;
+    if (threadIdx.x == 0) s_cand = 0;
+    __syncthreads();
+    long long mine = 0;
+    for (long long i = threadIdx.x; i < N; i += blockDim.x) mine += v[i] > -1.5f ? 1 : 0;
+    atomicAdd(reinterpret_cast<unsigned long long*>(&s_cand), (unsigned long long)mine);
+    __syncthreads();
+    const long long cand = s_cand;
+    const long long k = (long long)nodes[b] - budgets.rows[b];          // nodes that have to be merged away
+    float tau;
+    if (k <= 0) {
+        tau = 2.f;                                                      // fits without temporal merging
+    } else if (k > cand) {
+        tau = -2.f;                                                     // not reachable: link whatever can be linked
+    } else {
+        const float mk = block_kth_largest(v, N, k, hist);
+        __syncthreads();
+        const float mk1 = k + 1 <= cand ? block_kth_largest(v, N, k + 1, hist) : mk - 2e-3f;
+        tau = 0.5f * (mk + mk1);
+    }
+    if (threadIdx.x == 0) tau_t[b] = tau;
 }
 
 }  // namespace sttm

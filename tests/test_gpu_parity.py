@@ -296,3 +296,48 @@ def test_merged_positions():
     torch.cuda.synchronize()
     assert int(status.item()) == 1 << 4                      # capacity exceeded, reported, not fatal
     np.testing.assert_array_equal(short.cpu().numpy()[:offs[1] - 5], got[:offs[1] - 5])
+
+
+def test_budget_mode():
+    """tau_t chosen on the device for a row budget: the threshold agrees with the oracle's rule, the
+    count meets the budget exactly (budgets picked where the best cosines leave a clear gap at the
+    cut), and the whole output equals the oracle's at the returned threshold."""
+    checked = 0
+    for seed, shape in [(700, (8, 13, 13, 256)), (701, (6, 16, 16, 384)), (702, (10, 13, 13, 256))]:
+        T, H, W, D = shape
+        spec = helpers.small_spec(seed, T, H, W, D, p_static=0.6)
+        video = inputs.make_video(spec)
+        taus = helpers.safe_thresholds(video, 0.5, 0.5)
+        if taus is None:
+            continue
+        tau_s = taus[0]
+        nodes, m = oracle.best_candidate_cosines(video, tau_s)
+        gaps = m[:-1] - m[1:]                                   # gap below the k-th largest, k = index + 1
+        ks = [int(k) + 1 for k in np.argsort(-gaps)[:12] if gaps[k] >= 2e-4][:4]
+        dev = helpers.to_torch(video)
+        for k in ks:
+            budget = nodes - k
+            tau_ref, gap = oracle.budget_tau_t(video, tau_s, budget)
+            assert gap >= 2e-4
+            out, tau = binding.sttm_merge_budget(dev, tau_s, [budget], out_dtype=torch.float32)
+            torch.cuda.synchronize()
+            assert int(out.device_status.item()) == 0
+            tau_gpu = float(tau[0].item())
+            assert abs(tau_gpu - tau_ref) < 1e-5
+            count = int(out.out_count[0].item())
+            assert count == budget
+            ref = oracle.merge(video, tau_s, tau_gpu)
+            assert ref.count == count
+            np.testing.assert_array_equal(out.merge_map[0].cpu().numpy(), ref.merge_map)
+            np.testing.assert_array_equal(out.out_pos[:count].cpu().numpy(), ref.out_pos)
+            helpers.assert_features_close(out.out_feats[:count].float().cpu().numpy(), ref.out_feats, False)
+            checked += 1
+    assert checked >= 6, "too few budgets with a clear gap at the cut"
+    # a budget that needs no temporal merging, and one that cannot be met
+    out, tau = binding.sttm_merge_budget(dev, tau_s, [10 ** 9])
+    torch.cuda.synchronize()
+    assert float(tau[0].item()) == 2.0 and int(out.out_count[0].item()) == nodes
+    out, tau = binding.sttm_merge_budget(dev, tau_s, [1])
+    torch.cuda.synchronize()
+    assert float(tau[0].item()) == -2.0
+    assert int(out.out_count[0].item()) == oracle.merge(video, tau_s, -2.0, want_feats=False).count

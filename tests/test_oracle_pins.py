@@ -12,6 +12,7 @@ import torch
 
 from oracle import oracle
 from paper_2507_07990_b200 import inputs
+from tests import helpers
 from tests.bruteforce import sttm_bruteforce, level_sizes
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "quad_2x2.json")
@@ -316,3 +317,28 @@ def test_merged_positions_closed_forms():
     video = np.random.default_rng(5).standard_normal((3, 4, 4, 8)).astype(np.float32)
     ref = oracle.merge(video, 2.0, 2.0, want_feats=False)
     np.testing.assert_array_equal(oracle.merged_positions(ref.merge_map, ref.count), ref.out_pos.astype(np.float32))
+
+
+def test_budget_threshold_properties():
+    """Budget mode on the oracle: at the returned tau_t the row count is exactly the budget whenever
+    the gap at the cut is positive; a budget the spatial stage already meets needs no temporal
+    merging; an unreachable one links everything that has a candidate."""
+    spec = helpers.small_spec(600, 8, 13, 13, 64, dtype="f32", sigma=0.3, p_static=0.6)
+    video = inputs.make_video(spec)
+    base = oracle.merge(video, 0.9, 2.0, want_feats=False)
+    everything = oracle.merge(video, 0.9, -2.0, want_feats=False)
+    checked = 0
+    for frac in (0.95, 0.9, 0.8, 0.7, 0.6, 0.5):
+        budget = int(base.count * frac)
+        if budget < everything.count:
+            continue
+        tau, gap = oracle.budget_tau_t(video, 0.9, budget)
+        if gap > 0:
+            assert oracle.merge(video, 0.9, tau, want_feats=False).count == budget
+            checked += 1
+    assert checked >= 3
+    assert oracle.budget_tau_t(video, 0.9, base.count) == (2.0, float("inf"))
+    assert oracle.budget_tau_t(video, 0.9, base.count + 7)[0] == 2.0
+    assert oracle.budget_tau_t(video, 0.9, 1)[0] == -2.0
+    # one frame: no candidates at all
+    assert oracle.budget_tau_t(video[:1], 0.9, 1)[0] == -2.0

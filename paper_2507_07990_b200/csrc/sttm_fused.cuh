@@ -671,7 +671,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             if (q < total && !mbar_wait(sfull_bar + 8 * s, use, timed_out)) break;
             __syncwarp();
             const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
-            const uint32_t flush_mask = lds_u32x4(rec).x;
+            // (first pass of the budget mode: only the decisions are wanted, nothing is summed or written)
+            const bool dry = p.tmax != nullptr;
+            const uint32_t flush_mask = dry ? 0u : lds_u32x4(rec).x;
             // Slots g and g + 8 live in the four lanes of group g: all slots of one half of the
             // fragment are written in the same pass, every group following its own command.  One
             // loop per kind of destination and per half keeps register indices and offsets static.
@@ -717,7 +719,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
 #undef STTM_FLUSH_LOOP
             }
             __syncwarp();
-            if (q < total) {
+            if (q < total && !dry) {
                 uint32_t wa[4];
                 ldmatrix_x4(rec + woff, wa);
                 const uint32_t xb = sbase + s * p.slot_bytes + xoff;
@@ -1305,10 +1307,12 @@ __device__ __forceinline__ float key_float(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// k-th largest (k >= 1) of the values > -1.5 among v[0..n); the caller made sure there are at least k
-__device__ float block_kth_largest(const float* __restrict__ v, long long n, long long k, uint32_t* hist) {
+// One block: k-th largest (k >= 1) of the values > -1.5 among v[0..n), or -2 when there are fewer
+// than k; *cand receives their number.  Three histogram passes (11 + 11 + 10 bits of the key).
+__device__ float block_kth_largest(const float* __restrict__ v, long long n, long long k, uint32_t* hist,
+                                   long long* cand) {
     __shared__ uint32_t s_prefix, s_mask;
-    __shared__ long long s_k;
+    __shared__ long long s_k, s_total;
     if (threadIdx.x == 0) { s_prefix = 0; s_mask = 0; s_k = k; }
     __syncthreads();
     const int shifts[3] = {21, 10, 0}, bits[3] = {11, 11, 10};
@@ -1317,6 +1321,7 @@ __device__ float block_kth_largest(const float* __restrict__ v, long long n, lon
         for (int i = threadIdx.x; i < 2048; i += blockDim.x) hist[i] = 0;
         __syncthreads();
         const uint32_t prefix = s_prefix, mask = s_mask;
+#pragma unroll 8
         for (long long i = threadIdx.x; i < n; i += blockDim.x) {
             const float f = v[i];
             if (f > -1.5f) {
@@ -1326,6 +1331,11 @@ __device__ float block_kth_largest(const float* __restrict__ v, long long n, lon
         }
         __syncthreads();
         if (threadIdx.x == 0) {
+            if (pass == 0) {
+                long long total = 0;
+                for (int b = 0; b < nb; b++) total += hist[b];
+                s_total = total;
+            }
             long long kk = s_k;
             int b = nb - 1;
             for (; b > 0; b--) {               // from the largest bin down
@@ -1337,8 +1347,10 @@ __device__ float block_kth_largest(const float* __restrict__ v, long long n, lon
             s_mask = mask | ((uint32_t)(nb - 1) << shifts[pass]);
         }
         __syncthreads();
+        if (pass == 0 && s_total < k) break;    // fewer candidates than k (the same for every thread)
     }
-    return key_float(s_prefix);
+    *cand = s_total;
+    return s_total < k ? -2.f : key_float(s_prefix);
 }
 
 __global__ void __launch_bounds__(1024)
@@ -1346,27 +1358,44 @@ k_budget_tau(long long N, const float* __restrict__ tmax, const int32_t* __restr
              float* __restrict__ tau_t) {
     wait_for_prior_kernel();
     __shared__ uint32_t hist[2048];
-    __shared__ long long s_cand;
+    __shared__ unsigned long long s_above, s_equal;
+    __shared__ uint32_t s_below;            // key of the largest value below the k-th largest
     const int b = blockIdx.x;
     const float* v = tmax + (long long)b * N;
-    if (threadIdx.x == 0) s_cand = 0;
-    __syncthreads();
-    long long mine = 0;
-    for (long long i = threadIdx.x; i < N; i += blockDim.x) mine += v[i] > -1.5f ? 1 : 0;
-    atomicAdd(reinterpret_cast<unsigned long long*>(&s_cand), (unsigned long long)mine);
-    __syncthreads();
-    const long long cand = s_cand;
     const long long k = (long long)nodes[b] - budgets.rows[b];          // nodes that have to be merged away
     float tau;
     if (k <= 0) {
         tau = 2.f;                                                      // fits without temporal merging
-    } else if (k > cand) {
-        tau = -2.f;                                                     // not reachable: link whatever can be linked
     } else {
-        const float mk = block_kth_largest(v, N, k, hist);
-        __syncthreads();
-        const float mk1 = k + 1 <= cand ? block_kth_largest(v, N, k + 1, hist) : mk - 2e-3f;
-        tau = 0.5f * (mk + mk1);
+        long long cand;
+        const float mk = block_kth_largest(v, N, k, hist, &cand);
+        if (k > cand) {
+            tau = -2.f;                                                 // not reachable: link whatever can be linked
+        } else {
+            // the (k+1)-th largest: mk again if enough values equal it, else the largest value below it
+            if (threadIdx.x == 0) { s_above = 0; s_equal = 0; s_below = 0; }
+            __syncthreads();
+            unsigned long long above = 0, equal = 0;
+            uint32_t below = 0;
+#pragma unroll 8
+            for (long long i = threadIdx.x; i < N; i += blockDim.x) {
+                const float f = v[i];
+                if (f > -1.5f) {
+                    above += f > mk;
+                    equal += f == mk;
+                    if (f < mk) below = max(below, float_key(f));
+                }
+            }
+            atomicAdd(&s_above, above);
+            atomicAdd(&s_equal, equal);
+            atomicMax(&s_below, below);
+            __syncthreads();
+            float mk1;
+            if (k + 1 <= (long long)(s_above + s_equal)) mk1 = mk;
+            else if (k + 1 <= cand) mk1 = key_float(s_below);
+            else mk1 = mk - 2e-3f;
+            tau = 0.5f * (mk + mk1);
+        }
     }
     if (threadIdx.x == 0) tau_t[b] = tau;
 }

@@ -26,8 +26,11 @@
  *   - Layout: feats is [B, T, H, W, D] contiguous, D fastest; D must be a multiple of 4
  *     and the base pointer 16-byte aligned.  A token's cell id inside its video is
  *     c = t*H*W + y*W + x.  A quadtree node is named by the cell id of its top-left
- *     (anchor) cell.  Quadtrees deeper than 3 levels (coarsest node wider than 4 cells)
- *     are reported as STTM_ERR_UNSUPPORTED.
+ *     (anchor) cell.  Quadtrees of up to 3 levels (coarsest node at most 4 cells wide) run on
+ *     the tuned kernels; deeper ones (up to 8 levels) only through sttm_merge_ex / sttm_merge /
+ *     sttm_merge_host, on plain general kernels whose chain sums use floating-point atomics
+ *     (last bits may differ between runs); the stage calls and the budget mode report them
+ *     as STTM_ERR_UNSUPPORTED.
  */
 #ifndef STTM_H
 #define STTM_H
@@ -257,7 +260,8 @@ void sttm_set_tuning(int path, int cluster_size, int frames_per_item);
  */
 void sttm_set_ring_split(int sum_slots, int lead_frames);
 
-/* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 fused. */
+/* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 fused, 2 the
+ * general kernels for quadtrees of more than three levels. */
 int sttm_last_path(void);
 
 /*

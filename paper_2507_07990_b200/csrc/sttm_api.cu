@@ -12,6 +12,7 @@
 
 #include "sttm_kernels.cuh"
 #include "sttm_fused.cuh"
+#include "sttm_generic.cuh"
 
 namespace {
 
@@ -25,10 +26,11 @@ thread_local const float* g_budget_tau_dev = nullptr;
 thread_local cudaEvent_t* g_stage_events = nullptr;   // when set: event i is recorded after stage i-1
 
 constexpr int kStageCount = 5;
-const char* const kStageNames[2][kStageCount] = {
+const char* const kStageNames[3][kStageCount] = {
     {"spatial", "temporal+roots", "ordering", "accumulate", "combine"},
-    {"fused", "roots", "ordering", "gather", "-"}};
-thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: fused kernel
+    {"fused", "roots", "ordering", "gather", "-"},
+    {"-", "-", "-", "-", "general"}};
+thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: fused kernel, 2: general kernels
 
 inline void mark_stage(int boundary, cudaStream_t st) {
     if (g_stage_events != nullptr) cudaEventRecord(g_stage_events[boundary], st);
@@ -50,6 +52,9 @@ struct Plan {
     long long cells;          // B*N
     long long partial_slots;
     FusedPlan f;
+    bool generic;             // more than three quadtree levels: the plain kernels of sttm_generic.cuh
+    Pyr py;
+    size_t gen_pooled, gen_norms, gen_dots, gen_allpass, gen_acc;
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
         frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
@@ -202,7 +207,8 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
     Geo& g = pl->g;
     g.B = p->B; g.T = p->T; g.H = p->H; g.W = p->W; g.D = p->D;
     g.L = levels_of(p->H, p->W, p->lv1, &g.H1, &g.W1, &g.Hc, &g.Wc);
-    if (g.L > 3) return STTM_ERR_UNSUPPORTED;
+    if (g.L > kMaxLevels) return STTM_ERR_UNSUPPORTED;
+    pl->generic = g.L > 3;
     g.side = 1 << (g.L - 1);
     g.ncol = g.Hc * g.Wc;
     g.HW = p->H * p->W;
@@ -218,7 +224,21 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
     pl->Tc = (int)((g.T + nchunk - 1) / nchunk);
     pl->nchunk = (g.T + pl->Tc - 1) / pl->Tc;
     const int NC = g.side * g.side;
-    pl->partial_slots = 2ll * NC * g.ncol * pl->nchunk * g.B;
+    pl->partial_slots = pl->generic ? 0 : 2ll * NC * g.ncol * pl->nchunk * g.B;
+    {
+        Pyr& py = pl->py;
+        py = Pyr{};
+        py.L = g.L;
+        int h = g.H, w = g.W, no = 0, uo = 0;
+        for (int l = 0; l < g.L; l++) {
+            py.H[l] = h; py.W[l] = w;
+            py.noff[l] = no; no += h * w;
+            py.uoff[l] = l == 0 ? 0 : uo;
+            if (l >= 1) uo += h * w;
+            h = (h + 1) / 2; w = (w + 1) / 2;
+        }
+        py.nodes = no; py.upper = uo;
+    }
 
     const int NN = g.L == 3 ? 21 : (g.L == 2 ? 5 : 1);
     size_t o = 0;
@@ -243,7 +263,19 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
     pl->queue = take(4);
     pl->zero_end = o;
     pl->partial = take((size_t)pl->partial_slots * g.D * sizeof(float));
-    plan_fused(p, g, &pl->f);
+    pl->f.ok = false;
+    pl->gen_pooled = pl->gen_norms = pl->gen_dots = pl->gen_allpass = pl->gen_acc = o;
+    if (pl->generic) {
+        const long long frames = (long long)g.B * g.T;
+        const long long rows = std::min<long long>(pl->cells, std::max<long long>(p->out_capacity_rows, 1));
+        pl->gen_pooled = take((size_t)frames * pl->py.upper * g.D * sizeof(float));
+        pl->gen_norms = take((size_t)frames * pl->py.nodes * sizeof(float));
+        pl->gen_dots = take((size_t)frames * pl->py.nodes * sizeof(float));
+        pl->gen_allpass = take((size_t)frames * pl->py.nodes);
+        pl->gen_acc = take((size_t)rows * g.D * sizeof(float));
+    } else {
+        plan_fused(p, g, &pl->f);
+    }
     pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = pl->piece_next = o;
     if (pl->f.ok) {
         const size_t out_elt = p->out_dtype == STTM_BF16 ? 2 : 4;
@@ -471,6 +503,78 @@ sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacit
                         pl.f.nitems * kPieceSlots);
 }
 
+template <typename T, typename OutT>
+sttm_status run_generic(const T* feats, const sttm_params* p, const Plan& pl, char* ws, OutT* out_feats,
+                        int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
+                        int32_t* device_status, cudaStream_t st) {
+    const Geo g = pl.g;
+    const Pyr py = pl.py;
+    Taus taus;
+    fill_taus(p, &taus);
+    float* pooled = (float*)(ws + pl.gen_pooled);
+    float* norms = (float*)(ws + pl.gen_norms);
+    float* dots = (float*)(ws + pl.gen_dots);
+    int8_t* allpass = (int8_t*)(ws + pl.gen_allpass);
+    float* acc = (float*)(ws + pl.gen_acc);
+    int8_t* cover = (int8_t*)(ws + pl.cover);
+    int32_t* link = (int32_t*)(ws + pl.link);
+    int32_t* root = (int32_t*)(ws + pl.root);
+    const long long frames = (long long)g.B * g.T;
+    const long long rows = std::min<long long>(pl.cells, std::max<long long>(p->out_capacity_rows, 1));
+    sttm_status s;
+    STTM_CUDA_TRY(cudaMemsetAsync(link, 0xff, (size_t)pl.cells * 4, st));
+    STTM_CUDA_TRY(cudaMemsetAsync(acc, 0, (size_t)rows * g.D * sizeof(float), st));
+    for (int l = 1; l < py.L; l++) {
+        k_gen_pool<T><<<blocks_for(frames * py.H[l] * py.W[l] * 32, 256), 256, 0, st>>>(feats, pooled, g, py, l);
+        if ((s = launched()) != STTM_OK) return s;
+    }
+    k_gen_norm_dot<T><<<blocks_for(frames * py.nodes * 32, 256), 256, 0, st>>>(feats, pooled, g, py, norms, dots);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_allpass<<<blocks_for(frames * py.nodes, 256), 256, 0, st>>>(g, py, taus, norms, dots, allpass);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_cover<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, py, allpass, cover);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_temporal<T><<<blocks_for(pl.cells * 32, 256), 256, 0, st>>>(feats, pooled, g, py, taus, cover, norms, link,
+                                                                     p->match == STTM_MATCH_BEST ? 1 : 0);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_root_init<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, cover, link, root);
+    if ((s = launched()) != STTM_OK) return s;
+    int rounds = 1;
+    while ((1 << rounds) < g.T) rounds++;
+    for (int r = 0; r <= rounds; r++) {
+        k_gen_root_jump<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, root);
+        if ((s = launched()) != STTM_OK) return s;
+    }
+    k_gen_root_fill<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, cover, root);
+    if ((s = launched()) != STTM_OK) return s;
+
+    int32_t* frame_roots = (int32_t*)(ws + pl.frame_roots);
+    int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
+    long long* vid_off = (long long*)(ws + pl.vid_off);
+    int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
+    int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
+    k_frame_roots<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_roots);
+    if ((s = launched()) != STTM_OK) return s;
+    k_scan_frames<<<1, 1024, 0, st>>>(g, frame_roots, frame_base, out_count, vid_off, out_offsets);
+    if ((s = launched()) != STTM_OK) return s;
+    k_rows<<<g.B * g.T, 256, 0, st>>>(g, cover, link, frame_base, vid_off, row_at_root, row_anchor, out_pos,
+                                      p->out_capacity_rows, (int)p->pos, device_status);
+    if ((s = launched()) != STTM_OK) return s;
+    k_members<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, cover, root, row_at_root, vid_off,
+                                                        (int32_t*)(ws + pl.cell_row), merge_map,
+                                                        (int32_t*)(ws + pl.row_weight),
+                                                        (int32_t*)(ws + pl.row_last_t), (int)p->wt);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_accumulate<T><<<blocks_for(pl.cells * 32, 256), 256, 0, st>>>(feats, pooled, g, py, cover,
+                                                                       (const int32_t*)(ws + pl.cell_row), acc,
+                                                                       p->out_capacity_rows, (int)p->wt);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_finish<OutT><<<blocks_for(rows * (g.D / VEC), 256), 256, 0, st>>>(g, vid_off, acc,
+                                                                           (const int32_t*)(ws + pl.row_weight),
+                                                                           out_feats, p->out_capacity_rows);
+    return launched();
+}
+
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
 
 // Scratch of sttm_spatial_static: lives in the library image, so every GPU that loads the
@@ -591,6 +695,7 @@ sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size
     Plan pl;
     sttm_status s = make_plan(p, &pl);
     if (s != STTM_OK) return s;
+    if (pl.generic) return STTM_ERR_UNSUPPORTED;      // the stage calls cover up to three quadtree levels
     if (!feats || !ws || !cover_level || !frame_counts) return STTM_ERR_ARG;
     if (misaligned(feats, 16) || misaligned(ws, 256)) return STTM_ERR_ARG;
     if (ws_bytes < pl.total) return STTM_ERR_WORKSPACE;
@@ -605,6 +710,7 @@ sttm_status sttm_spatial_static(const void* feats, const sttm_params* p, int8_t*
     Plan pl;
     sttm_status s = make_plan(p, &pl);
     if (s != STTM_OK) return s;
+    if (pl.generic) return STTM_ERR_UNSUPPORTED;      // the stage calls cover up to three quadtree levels
     if (!feats || !cover_level || !frame_counts) return STTM_ERR_ARG;
     if (misaligned(feats, 16)) return STTM_ERR_ARG;
     // the only scratch of the spatial stage: one squared norm per quadtree node
@@ -627,6 +733,7 @@ sttm_status sttm_temporal(const void* feats, const sttm_params* p, void* ws, siz
     Plan pl;
     sttm_status s = make_plan(p, &pl);
     if (s != STTM_OK) return s;
+    if (pl.generic) return STTM_ERR_UNSUPPORTED;      // the stage calls cover up to three quadtree levels
     if (!feats || !ws || !cover_level || !link || !root) return STTM_ERR_ARG;
     if (misaligned(feats, 16) || misaligned(ws, 256)) return STTM_ERR_ARG;
     if (ws_bytes < pl.total) return STTM_ERR_WORKSPACE;
@@ -654,7 +761,25 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
     int8_t* cover = (int8_t*)(ws + pl.cover);
     int32_t* link = (int32_t*)(ws + pl.link);
     int32_t* root = (int32_t*)(ws + pl.root);
-    g_last_path = pl.f.ok ? 1 : 0;
+    g_last_path = pl.generic ? 2 : (pl.f.ok ? 1 : 0);
+    if (pl.generic) {
+        // more than three quadtree levels: the plain kernels, no stage breakdown
+        for (int i = 0; i <= 4; i++) mark_stage(i, st);
+        if (p->in_dtype == STTM_BF16)
+            s = p->out_dtype == STTM_BF16
+                    ? run_generic((const __nv_bfloat16*)feats, p, pl, ws, (__nv_bfloat16*)out_feats, out_pos, merge_map,
+                                  out_count, out_offsets, device_status, st)
+                    : run_generic((const __nv_bfloat16*)feats, p, pl, ws, (float*)out_feats, out_pos, merge_map,
+                                  out_count, out_offsets, device_status, st);
+        else
+            s = p->out_dtype == STTM_BF16
+                    ? run_generic((const float*)feats, p, pl, ws, (__nv_bfloat16*)out_feats, out_pos, merge_map,
+                                  out_count, out_offsets, device_status, st)
+                    : run_generic((const float*)feats, p, pl, ws, (float*)out_feats, out_pos, merge_map, out_count,
+                                  out_offsets, device_status, st);
+        mark_stage(5, st);
+        return s;
+    }
     if (pl.f.ok) {
         // single-read path: fused kernel, roots, ordering, gather
         STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.ones_begin, 0xff, pl.ones_end - pl.ones_begin, st));

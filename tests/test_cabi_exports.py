@@ -35,6 +35,15 @@ def test_host_only_entry_points():
     assert binding.sttm_workspace_bytes(bad) == 0
     lib = binding.load_library()
     assert lib.sttm_status_string(2) == b"unsupported shape"
+    import ctypes as C
+    lib.sttm_budget_workspace_bytes.restype = C.c_size_t
+    three = binding.make_params((1, 8, 16, 16, 64), torch.bfloat16, 0.9, 0.9)
+    deep = binding.make_params((1, 8, 24, 24, 64), torch.bfloat16, 0.9, 0.9)        # 24 -> 12 -> 6 -> 3: four levels
+    too_deep = binding.make_params((1, 1, 600, 4, 64), torch.bfloat16, 0.9, 0.9)    # nine levels
+    assert binding.sttm_workspace_bytes(deep) > 8 * (576 // 3) * 64 * 4             # holds the pooled fp32 maps
+    assert lib.sttm_budget_workspace_bytes(C.byref(three.params)) > 0
+    assert lib.sttm_budget_workspace_bytes(C.byref(deep.params)) == 0               # budget mode: three levels
+    assert binding.sttm_workspace_bytes(too_deep) == 0
 
 
 def test_merged_positions_argument_checks_need_no_gpu():

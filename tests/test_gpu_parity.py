@@ -200,10 +200,16 @@ def test_bad_arguments_are_rejected_on_the_host():
     with pytest.raises(binding.SttmError) as e:
         binding.sttm_merge_ex(dev, 0.5, 0.5)
     assert e.value.code == 1
-    dev = torch.zeros((1, 2, 13, 13, 8), dtype=torch.bfloat16, device="cuda")   # 13 -> 7 -> 4 -> 2: four levels
+    dev = torch.zeros((1, 1, 600, 4, 8), dtype=torch.bfloat16, device="cuda")   # 600 -> ... -> 3: nine levels
     with pytest.raises(binding.SttmError) as e:
-        binding.sttm_merge_ex(dev, 0.5, 0.5, lv1=2)
+        binding.sttm_merge_ex(dev, 0.5, 0.5)
     assert e.value.code == 2
+    dev = torch.zeros((1, 2, 13, 13, 8), dtype=torch.bfloat16, device="cuda")   # 13 -> 7 -> 4 -> 2: four levels
+    for call in (lambda: binding.sttm_spatial(dev, 0.5, lv1=2),
+                 lambda: binding.sttm_merge_budget(dev, 0.5, [10], lv1=2)):
+        with pytest.raises(binding.SttmError) as e:                             # stage calls and budget mode
+            call()                                                              # stop at three levels
+        assert e.value.code == 2
     prob = binding.make_params((1, 2, 13, 13, 8), torch.bfloat16, 0.5, 0.5)
     ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
     lib = binding.load_library()
@@ -341,3 +347,65 @@ def test_budget_mode():
     torch.cuda.synchronize()
     assert float(tau[0].item()) == -2.0
     assert int(out.out_count[0].item()) == oracle.merge(video, tau_s, -2.0, want_feats=False).count
+
+
+# Quadtrees of four and five levels (the 2x2 coarsest map of the paper's ablation on its real grids,
+# and grids of more than 16 cells a side): the general kernels behind sttm_merge_ex.
+@pytest.mark.parametrize("shape", [(4, 13, 13, 64, 2, "f32"), (5, 14, 14, 128, 2, "bf16"), (3, 16, 16, 256, 2, "bf16"),
+                                   (3, 18, 12, 256, 4, "bf16"), (3, 20, 20, 64, 2, "f32"), (2, 24, 33, 132, 4, "bf16"),
+                                   (6, 24, 24, 3584, 4, "bf16")],
+                         ids=lambda s: "T%dH%dW%dD%dlv%d%s" % s)
+def test_deeper_quadtrees(shape):
+    T, H, W, D, lv1, dtype = shape
+    done = 0
+    for seed in range(4):
+        spec = helpers.small_spec(800 + seed, T, H, W, D, dtype=dtype, sigma=0.3 if D < 200 else 0.05, depth_max=4)
+        video = inputs.make_video(spec)
+        taus = helpers.safe_thresholds(video, 0.5, 0.5, lv1)
+        if taus is None:
+            continue
+        ref = oracle.merge(video, taus[0], taus[1], lv1=lv1, want_feats=False)
+        assert int(ref.cover_level.max()) <= 4
+        for out_dtype, wt, pos, match in [(torch.float32, binding.W_NODE, binding.POS_SURVIVED, binding.MATCH_TOPLEFT),
+                                          (torch.bfloat16, binding.W_AREA, binding.POS_REASSIGNED, binding.MATCH_TOPLEFT),
+                                          (torch.float32, binding.W_NODE, binding.POS_SURVIVED, binding.MATCH_BEST)]:
+            run_and_compare(video, taus[0], taus[1], lv1=lv1, out_dtype=out_dtype, wt=wt, pos=pos, stages=False,
+                            match=match)
+        done += 1
+        if done == 2:
+            break
+    assert done >= 1, "no seed gave thresholds with a margin"
+
+
+def test_deeper_quadtrees_batch_capacity_and_host_entry():
+    specs = [helpers.small_spec(840 + v, 5, 18, 20, 64, dtype="bf16", sigma=0.3, depth_max=4, p_static=p)
+             for v, p in enumerate((0.9, 0.4))]
+    videos = [inputs.make_video(s) for s in specs]
+    taus = [helpers.safe_thresholds(v, 0.5, 0.5, 4) for v in videos]
+    assert all(t is not None for t in taus)
+    refs = [oracle.merge(v, ts, tt) for v, (ts, tt) in zip(videos, taus)]
+    dev = helpers.to_torch(np.stack(videos))
+    out = binding.sttm_merge_ex(dev, [t[0] for t in taus], [t[1] for t in taus], out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    assert binding.load_library().sttm_last_path() == 2
+    offs = out.out_offsets.tolist()
+    for b, ref in enumerate(refs):
+        assert int(out.out_count[b]) == ref.count and offs[b + 1] - offs[b] == ref.count
+        np.testing.assert_array_equal(out.merge_map[b].cpu().numpy(), ref.merge_map)
+        np.testing.assert_array_equal(out.out_pos[offs[b]:offs[b + 1]].cpu().numpy(), ref.out_pos)
+        helpers.assert_features_close(out.out_feats[offs[b]:offs[b + 1]].cpu().numpy(), ref.out_feats, False)
+    # fewer rows than the result: the rows that fit are right, the rest is reported
+    cap = refs[0].count + refs[1].count // 2
+    out = binding.sttm_merge_ex(dev, [t[0] for t in taus], [t[1] for t in taus], out_dtype=torch.float32, capacity=cap)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) & (1 << 4)
+    assert [int(c) for c in out.out_count] == [r.count for r in refs]
+    both = np.concatenate([r.out_feats for r in refs])
+    helpers.assert_features_close(out.out_feats[:cap].cpu().numpy(), both[:cap], False)
+    # host buffers in, host buffers out
+    h = torch.from_numpy(videos[0].view(np.int16)).view(torch.bfloat16).pin_memory()
+    res = binding.sttm_merge_host(h, taus[0][0], taus[0][1], want_map=True)
+    assert int(res.out_count[0]) == refs[0].count
+    np.testing.assert_array_equal(res.merge_map[0].numpy(), refs[0].merge_map)
+    helpers.assert_features_close(res.out_feats[:refs[0].count].float().numpy(), refs[0].out_feats, True)

@@ -165,6 +165,52 @@ sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_
                        void* out_feats, int32_t* out_pos, int32_t* out_count, void* stream);
 
 /*
+ * One video cut into segments of consecutive frames, one segment per GPU (Section 3.3: a chain
+ * of temporal links may cross a cut).  The paper has no counterpart: it merges a video on one
+ * device.  Each segment is merged by sttm_merge_ex (fp32 rows, merge map, SURVIVED ids) with
+ * the last frame of the segment before it, the halo, as its frame 0; the halo alone (T = 1)
+ * is merged too, which gives its kept nodes u in order, their features F(u) and weights w_u.
+ * The first n_h rows of the segment's result are rooted in the halo (row b at node b) and
+ * belong to an earlier segment.  A row is held as (mean m, weight W); a contribution (S, V)
+ * turns it into (W m + S) / (W + V).  Segments are finished from the last to the first:
+ * sttm_segment_fold takes in what the next segment sent, sttm_segment_emit makes what goes to
+ * the previous one, sttm_segment_finish writes the owned rows.  All pointers are device
+ * pointers; nothing is allocated; every call is asynchronous on stream.
+ *
+ * sttm_row_weights: W of every row of a finished sttm_merge_ex call (same params, same ws,
+ *   which still holds that call's cover map): one per member node or, for STTM_W_AREA, the
+ *   node's cells.  weights float32 [min(cells, out_capacity_rows)].
+ * sttm_segment_fold: n = min(*n_dev, n_max) contributions keyed by anchors[i], the cell
+ *   (y*W + x) of a kept node of this segment's last frame; map_last int32 [HW] is the merge
+ *   map of that frame (local rows).  Adds s[i, :] to extra[row, :] and v[i] to extra_w[row]
+ *   with fp32 atomics (extra, extra_w: [capacity_rows, D] and [capacity_rows], zero before the
+ *   first call).  Entries with v[i] == 0 are skipped; an anchor outside the frame sets
+ *   (1 << STTM_ERR_ARG), a row outside capacity (1 << STTM_ERR_CAPACITY) in *device_status.
+ * sttm_segment_emit: for b < min(*n_h_dev, n_max): v_out[b] = W_b + extra_w[b] - w_u and
+ *   s_out[b, :] = W_b m_b + extra[b, :] - w_u F(u), the halo node itself left out because the
+ *   owner's row has it already.  feats/weights/extra/extra_w are the local rows, halo_feats
+ *   [n_h, D] and halo_w [n_h] the rows and weights of the halo's own merge.
+ * sttm_segment_finish: owned row r = local row r + n_h (n_h_dev NULL: no halo) with its
+ *   contributions, as out_dtype; out_pos[r] = local id + pos_shift for STTM_POS_SURVIVED (pass
+ *   (first owned frame - frames in front of it in the local input) * H * W), r + pos_shift for
+ *   STTM_POS_REASSIGNED (pass the rows owned by earlier segments); *owned_count = count - n_h.
+ *   feats, extra and out_feats 16-byte aligned, D a multiple of 4.
+ */
+sttm_status sttm_row_weights(const sttm_params* p, const void* ws, const int32_t* merge_map,
+                             const int64_t* out_offsets, float* weights, void* stream);
+sttm_status sttm_segment_fold(const int32_t* map_last, const int32_t* anchors, const float* v, const float* s,
+                              const int32_t* n_dev, int n_max, int HW, int D, float* extra, float* extra_w,
+                              long long capacity_rows, int32_t* device_status, void* stream);
+sttm_status sttm_segment_emit(const float* feats, const float* weights, const float* extra, const float* extra_w,
+                              const float* halo_feats, const float* halo_w, const int32_t* n_h_dev, int n_max, int D,
+                              float* v_out, float* s_out, void* stream);
+sttm_status sttm_segment_finish(const float* feats, const int32_t* pos, const float* weights, const float* extra,
+                                const float* extra_w, const int32_t* count_dev, const int32_t* n_h_dev, int D,
+                                long long capacity_rows, long long pos_shift, sttm_pos_mode pos_mode,
+                                sttm_dtype out_dtype, void* out_feats, int32_t* out_pos, int32_t* owned_count,
+                                void* stream);
+
+/*
  * Same computation with HOST buffers: copies feats to the device, runs sttm_merge_ex,
  * copies the used rows back and synchronises.  All pointers are host pointers (pinned
  * memory makes the copies asynchronous and faster).  h_merge_map and h_out_offsets may

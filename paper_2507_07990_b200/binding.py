@@ -28,7 +28,8 @@ EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame",
            "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
            "sttm_set_stage_events", "sttm_set_tuning", "sttm_set_ring_split", "sttm_last_path",
            "sttm_fused_launch_shape", "sttm_spatial_static", "sttm_merged_positions",
-           "sttm_merged_positions_workspace", "sttm_merge_budget", "sttm_budget_workspace_bytes"]
+           "sttm_merged_positions_workspace", "sttm_merge_budget", "sttm_budget_workspace_bytes",
+           "sttm_row_weights", "sttm_segment_fold", "sttm_segment_emit", "sttm_segment_finish"]
 
 
 class SttmParams(C.Structure):
@@ -99,6 +100,16 @@ def load_library(path: Optional[str] = None):
     lib.sttm_merged_positions.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_longlong, C.c_void_p, C.c_size_t,
                                           C.c_void_p, C.c_longlong, C.c_void_p, C.c_void_p]
     lib.sttm_merged_positions.restype = C.c_int
+    vp = C.c_void_p
+    lib.sttm_row_weights.argtypes = [pp, vp, vp, vp, vp, vp]
+    lib.sttm_row_weights.restype = C.c_int
+    lib.sttm_segment_fold.argtypes = [vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp, C.c_longlong, vp, vp]
+    lib.sttm_segment_fold.restype = C.c_int
+    lib.sttm_segment_emit.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.c_int, C.c_int, vp, vp, vp]
+    lib.sttm_segment_emit.restype = C.c_int
+    lib.sttm_segment_finish.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.c_int, C.c_longlong, C.c_longlong, C.c_int,
+                                        C.c_int, vp, vp, vp, vp]
+    lib.sttm_segment_finish.restype = C.c_int
     lib.sttm_set_ring_split.argtypes = [C.c_int, C.c_int]
     lib.sttm_set_ring_split.restype = None
     lib.sttm_last_path.argtypes = []
@@ -294,6 +305,38 @@ def sttm_merge_ex(feats: torch.Tensor, tau_s, tau_t, lv1: int = 4, out_dtype: to
     plan = MergePlan(tuple(feats.shape), feats.dtype, tau_s, tau_t, lv1, out_dtype, pos, wt, capacity, want_map,
                      feats.device, match)
     return plan.run(feats)
+
+
+def sttm_row_weights(plan: MergePlan) -> torch.Tensor:
+    """Weight of every row of the plan's last run (which must have kept its merge map)."""
+    p = plan.problem.params
+    rows = min(int(p.B * p.T * p.H * p.W), int(p.out_capacity_rows))
+    weights = torch.empty((rows,), dtype=torch.float32, device=plan.ws.device)
+    _check(load_library().sttm_row_weights(C.byref(p), _ptr(plan.ws), _ptr(plan.merge_map), _ptr(plan.out_offsets),
+                                           _ptr(weights), _stream()), "sttm_row_weights")
+    return weights
+
+
+def sttm_segment_fold(map_last, anchors, v, s, n_dev, extra, extra_w, status) -> None:
+    n_max, D = s.shape
+    _check(load_library().sttm_segment_fold(_ptr(map_last), _ptr(anchors), _ptr(v), _ptr(s), _ptr(n_dev), n_max,
+                                            map_last.numel(), D, _ptr(extra), _ptr(extra_w), extra_w.numel(),
+                                            _ptr(status), _stream()), "sttm_segment_fold")
+
+
+def sttm_segment_emit(feats, weights, extra, extra_w, halo_feats, halo_w, n_h_dev, v_out, s_out) -> None:
+    n_max, D = s_out.shape
+    _check(load_library().sttm_segment_emit(_ptr(feats), _ptr(weights), _ptr(extra), _ptr(extra_w), _ptr(halo_feats),
+                                            _ptr(halo_w), _ptr(n_h_dev), n_max, D, _ptr(v_out), _ptr(s_out),
+                                            _stream()), "sttm_segment_emit")
+
+
+def sttm_segment_finish(feats, pos, weights, extra, extra_w, count_dev, n_h_dev, pos_shift, pos_mode, out_feats,
+                        out_pos, owned_count) -> None:
+    _check(load_library().sttm_segment_finish(_ptr(feats), _ptr(pos), _ptr(weights), _ptr(extra), _ptr(extra_w),
+                                              _ptr(count_dev), _ptr(n_h_dev), feats.shape[1], extra_w.numel(),
+                                              pos_shift, pos_mode, _dtype_code(out_feats.dtype), _ptr(out_feats),
+                                              _ptr(out_pos), _ptr(owned_count), _stream()), "sttm_segment_finish")
 
 
 class BudgetPlan:

@@ -13,6 +13,7 @@
 #include "sttm_kernels.cuh"
 #include "sttm_fused.cuh"
 #include "sttm_generic.cuh"
+#include "sttm_segments.cuh"
 
 namespace {
 
@@ -960,6 +961,67 @@ sttm_status sttm_merged_positions(const int32_t* merge_map, const int64_t* out_o
     if (s != STTM_OK) return s;
     const long long rows_max = std::min<long long>(capacity_rows, (long long)B * N);
     k_pos_finish<<<blocks_for(rows_max, 256), 256, 0, st>>>(rows_max, out_offsets, B, sum, cnt, out_pos_mean);
+    return launched();
+}
+
+sttm_status sttm_row_weights(const sttm_params* p, const void* ws, const int32_t* merge_map,
+                             const int64_t* out_offsets, float* weights, void* stream) {
+    Plan pl;
+    sttm_status s = make_plan(p, &pl);
+    if (s != STTM_OK) return s;
+    if (!ws || !merge_map || !out_offsets || !weights || misaligned(ws, 256)) return STTM_ERR_ARG;
+    if (p->out_capacity_rows < 1) return STTM_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const long long rows = std::min<long long>(pl.cells, p->out_capacity_rows);
+    STTM_CUDA_TRY(cudaMemsetAsync(weights, 0, (size_t)rows * sizeof(float), st));
+    k_row_weights<<<blocks_for(pl.cells, 256), 256, 0, st>>>(pl.g, (const int8_t*)((const char*)ws + pl.cover),
+                                                            merge_map, out_offsets, weights, rows,
+                                                            (int)p->wt);
+    return launched();
+}
+
+sttm_status sttm_segment_fold(const int32_t* map_last, const int32_t* anchors, const float* v, const float* s,
+                              const int32_t* n_dev, int n_max, int HW, int D, float* extra, float* extra_w,
+                              long long capacity_rows, int32_t* device_status, void* stream) {
+    if (!map_last || !anchors || !v || !s || !n_dev || !extra || !extra_w) return STTM_ERR_ARG;
+    if (n_max < 1 || HW < 1 || D < 1 || capacity_rows < 1) return STTM_ERR_ARG;
+    k_segment_fold<<<blocks_for((long long)n_max * 32, 256), 256, 0, (cudaStream_t)stream>>>(
+        map_last, anchors, v, s, n_dev, n_max, HW, D, extra, extra_w, capacity_rows, device_status);
+    return launched();
+}
+
+sttm_status sttm_segment_emit(const float* feats, const float* weights, const float* extra, const float* extra_w,
+                              const float* halo_feats, const float* halo_w, const int32_t* n_h_dev, int n_max, int D,
+                              float* v_out, float* s_out, void* stream) {
+    if (!feats || !weights || !extra || !extra_w || !halo_feats || !halo_w || !n_h_dev || !v_out || !s_out)
+        return STTM_ERR_ARG;
+    if (n_max < 1 || D < 1) return STTM_ERR_ARG;
+    k_segment_emit<<<blocks_for((long long)n_max * 32, 256), 256, 0, (cudaStream_t)stream>>>(
+        feats, weights, extra, extra_w, halo_feats, halo_w, n_h_dev, n_max, D, v_out, s_out);
+    return launched();
+}
+
+sttm_status sttm_segment_finish(const float* feats, const int32_t* pos, const float* weights, const float* extra,
+                                const float* extra_w, const int32_t* count_dev, const int32_t* n_h_dev, int D,
+                                long long capacity_rows, long long pos_shift, sttm_pos_mode pos_mode,
+                                sttm_dtype out_dtype, void* out_feats, int32_t* out_pos, int32_t* owned_count,
+                                void* stream) {
+    if (!feats || !pos || !weights || !extra || !extra_w || !count_dev || !out_feats || !out_pos || !owned_count)
+        return STTM_ERR_ARG;
+    if (D < 1 || D % 4 != 0 || capacity_rows < 1) return STTM_ERR_ARG;
+    if (misaligned(feats, 16) || misaligned(extra, 16) || misaligned(out_feats, 16)) return STTM_ERR_ARG;
+    if (out_dtype != STTM_BF16 && out_dtype != STTM_F32) return STTM_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const unsigned blocks = blocks_for(capacity_rows * (D / VEC), 256);
+    const int re = pos_mode == STTM_POS_REASSIGNED ? 1 : 0;
+    if (out_dtype == STTM_BF16)
+        k_segment_finish<__nv_bfloat16><<<blocks, 256, 0, st>>>(feats, pos, weights, extra, extra_w, count_dev,
+                                                                n_h_dev, D, capacity_rows, pos_shift, re,
+                                                                (__nv_bfloat16*)out_feats, out_pos, owned_count);
+    else
+        k_segment_finish<float><<<blocks, 256, 0, st>>>(feats, pos, weights, extra, extra_w, count_dev, n_h_dev, D,
+                                                        capacity_rows, pos_shift, re, (float*)out_feats, out_pos,
+                                                        owned_count);
     return launched();
 }
 

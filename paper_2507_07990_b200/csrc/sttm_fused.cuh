@@ -449,11 +449,18 @@ struct SlotTable {
 // ---------------------------------------------------------------------------------
 // The kernel.  Warps: [0, NM) Gram, then 4 combine, NA sum, similarity, chain, two producers.
 // ---------------------------------------------------------------------------------
+// kLean: the common set-up (top-left destination, bf16 rows, one ring, thresholds from the host)
+// with the options compiled out -- the budget mode's additions (best candidate cosine per kept
+// node written to p.tmax with the sums left out; tau_t read from p.tau_t_dev), the second ring,
+// fp32 rows, the most-similar destination.  The kernel is a chain of dependent instructions in
+// seven code streams per SM: the unused branches cost 3 % of its time when they are present.
+template <bool kLean>
 __global__ void __launch_bounds__(kFusedMaxThreads, 1)
 k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus) {
     extern __shared__ __align__(128) unsigned char smem[];
+    const int RB2 = kLean ? 0 : p.RB;          // slots of the second ring
     unsigned char* ring = smem;
-    size_t off = (size_t)(p.R + p.RB) * p.slot_bytes;
+    size_t off = (size_t)(p.R + RB2) * p.slot_bytes;
     float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)p.NM * kGramVals * 4;
     float* redsum = reinterpret_cast<float*>(smem + off);    off += kGramVals * 4;
     float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * p.C * kSumVals * 4;
@@ -481,9 +488,9 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     if (tid == 0) {
         for (int s = 0; s < p.R; s++) {
             mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, p.NM + (p.RB == 0 ? p.NA : 0));
+            mbar_init(empty_bar + 8 * s, p.NM + (RB2 == 0 ? p.NA : 0));
         }
-        for (int s = 0; s < p.RB; s++) {
+        for (int s = 0; s < RB2; s++) {
             mbar_init(fullb_bar + 8 * s, 1);
             mbar_init(emptyb_bar + 8 * s, p.NA);
         }
@@ -502,7 +509,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int k = tid * 16; k < (p.R + p.RB) * p.slot_bytes; k += blockDim.x * 16)
+    for (int k = tid * 16; k < (p.R + RB2) * p.slot_bytes; k += blockDim.x * 16)
         *reinterpret_cast<uint4*>(ring + k) = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     cluster_arrive();
@@ -659,10 +666,10 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
             if (!skip) total += it.n;
         // the frames come from a ring of their own, or (RB == 0) from the Gram warps' ring
-        const bool own = p.RB > 0;
+        const bool own = RB2 > 0;
         const uint32_t sfull_bar = own ? fullb_bar : full_bar, sempty_bar = own ? emptyb_bar : empty_bar;
         const uint32_t sbase = own ? ringb_base : ring_base;
-        const int SR = own ? p.RB : p.R;
+        const int SR = own ? RB2 : p.R;
         // one record per frame, and a last one that only writes out what the last item left
         int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before
         for (; q <= total; q++) {
@@ -672,7 +679,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             __syncwarp();
             const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
             // (first pass of the budget mode: only the decisions are wanted, nothing is summed or written)
-            const bool dry = p.tmax != nullptr;
+            const bool dry = !kLean && p.tmax != nullptr;
             const uint32_t flush_mask = dry ? 0u : lds_u32x4(rec).x;
             // Slots g and g + 8 live in the four lanes of group g: all slots of one half of the
             // fragment are written in the same pass, every group following its own command.  One
@@ -696,7 +703,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     if (fc.y != 0) {                                                                                          \
         float* dst = p.pieces + row;                                                                          \
         STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x, y))                 \
-    } else if (p.out_f32) {                                                                                   \
+    } else if ((!kLean && p.out_f32)) {                                                                                   \
         float* dst = reinterpret_cast<float*>(p.staging) + row;                                               \
         STTM_FLUSH_LOOP(I0, I1, *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x, y))                 \
     } else {                                                                                                  \
@@ -750,7 +757,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const uint32_t xchg_a = smem_u32(xchg);
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
-            const float tau_s = taus.s[it.b], tau_t = p.tau_t_dev != nullptr ? p.tau_t_dev[it.b] : taus.t[it.b];
+            const float tau_s = taus.s[it.b], tau_t = (!kLean && p.tau_t_dev != nullptr) ? p.tau_t_dev[it.b] : taus.t[it.b];
             const LaneGeo lg = lane_geo(p.tiles[it.tile], c, L, p.W);
             const float w1 = lg.w1, w2 = lg.w2;
             const bool valid = lg.valid;
@@ -825,7 +832,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     const uint32_t passm = (__ballot_sync(full, pass) >> (16 * half)) & 0xffffu;
                     const uint32_t cand = passm & lane_region(lg, c, lv);
                     int cstar = cand ? __ffs(cand) - 1 : 0;           // first in row-major order: the top-left one
-                    if (p.match_best) {
+                    if (!kLean && p.match_best) {
                         // the most similar of them instead (equal ones: the first); the cosine itself is
                         // needed here, every lane looks at the 16 lanes of its half
                         const float cosv = pass ? dot / (sqrtf(nk) * sqrtf(pnk)) : -2.f;
@@ -836,7 +843,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                             if (((cand >> i) & 1u) && si > best) { best = si; cstar = i; }
                         }
                     }
-                    if (p.tmax != nullptr) {
+                    if (!kLean && p.tmax != nullptr) {
                         // budget mode: the number of rows as a function of tau_t only needs, per kept node,
                         // the largest cosine to its candidates (the node is linked iff that exceeds tau_t)
                         const float cosv = rep ? ((nk == 0.f || pnk == 0.f) ? 0.f : dot / (sqrtf(nk) * sqrtf(pnk))) : -2.f;
@@ -1003,12 +1010,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             __syncwarp();
             if (lane == 0) mbar_arrive(rfull_bar + 8 * hb);
         }
-    } else if (warp == w_prod || (warp == w_prod + 1 && p.RB == 0)) {
+    } else if (warp == w_prod || (warp == w_prod + 1 && RB2 == 0)) {
         // ---------------------------------- producer warps ----------------------------------
         // Issuing one bulk copy costs a warp some 80 cycles, and a frame is 16 of them, so two
         // warps share the rows (with a second ring the second warp has that ring to fill, and
         // this one issues all 16).
-        const int nprod = p.RB == 0 ? 2 : 1, which = warp - w_prod;
+        const int nprod = RB2 == 0 ? 2 : 1, which = warp - w_prod;
         const int row = lane * nprod + which;              // the tile row this lane copies
         int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
@@ -1041,7 +1048,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
             mbar_wait(full_bar + 8 * (qq % p.R), qq / p.R, late);
             timed_out |= late;
         }
-    } else if (warp == w_prod + 1 && p.RB > 0) {
+    } else if (warp == w_prod + 1 && RB2 > 0) {
         // ---------------------------------- second producer ----------------------------------
         // The sum warps need a frame only once its record exists, long after the Gram warps are
         // done with it.  Holding the frame in shared memory all that time would let too few frames
@@ -1065,12 +1072,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     bulk_g2s(ringb_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
                              (uint32_t)(p.S * 2), bar);
                 }
-                if (++s == p.RB) { s = 0; use++; }
+                if (++s == RB2) { s = 0; use++; }
             }
         }
-        for (int qq = max(0, q - p.RB); qq < q; qq++) {
+        const int rb = kLean ? 1 : RB2;       // (this role does not exist in the lean kernel)
+        for (int qq = max(0, q - RB2); qq < q; qq++) {
             bool late = false;
-            mbar_wait(fullb_bar + 8 * (qq % p.RB), qq / p.RB, late);
+            mbar_wait(fullb_bar + 8 * (qq % rb), qq / rb, late);
             timed_out |= late;
         }
     }

@@ -427,8 +427,8 @@ int fused_resident_clusters(const FusedPlan& f) {
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    cudaFuncSetAttribute(k_fused<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
-    if (cudaOccupancyMaxActiveClusters(&n, k_fused<true>, &cfg) != cudaSuccess || n < 1) {
+    cudaFuncSetAttribute(k_fused<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+    if (cudaOccupancyMaxActiveClusters(&n, k_fused<true, false>, &cfg) != cudaSuccess || n < 1) {
         cudaGetLastError();
         n = kSmCount / f.C;
     }
@@ -443,8 +443,9 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     const FusedPlan& f = pl.f;
     static bool configured = false;
     if (!configured) {
-        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         configured = true;
     }
     FusedParams fp = {};
@@ -483,8 +484,10 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
     const bool lean = fp.tmax == nullptr && fp.tau_t_dev == nullptr && fp.RB == 0 && !fp.out_f32 && !fp.match_best;
-    if (lean) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<true>, fp, taus));
-    else STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<false>, fp, taus));
+    const bool flagship = lean && fp.C == kFlagshipC && fp.S == kFlagshipS && fp.NM == kFlagshipNM && fp.NA == kFlagshipNA && fp.L == 3;
+    if (flagship) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<true, true>, fp, taus));
+    else if (lean) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<true, false>, fp, taus));
+    else STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<false, false>, fp, taus));
     g_launches++;
     return STTM_OK;
 }

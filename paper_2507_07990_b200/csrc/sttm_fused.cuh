@@ -58,6 +58,8 @@ constexpr int kFusedMaxThreads = (kMaxGramWarps + kCombineWarps + kMaxSumWarps +
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after two seconds
 
 enum : int { kStatusWaitTimeout = 1 << 6 };
+// launch shape of the instantiation with constant shape (D = 3584 bf16)
+constexpr int kFlagshipC = 4, kFlagshipS = 896, kFlagshipNM = 4, kFlagshipNA = 7;
 
 struct FlushCmd { int slot, kind, dst; float weight; };     // kind 0: finished row, 1: piece
 // Commands of one frame for the sum warps: first write out and clear the chain sums of the
@@ -454,16 +456,21 @@ struct SlotTable {
 // node written to p.tmax with the sums left out; tau_t read from p.tau_t_dev), the second ring,
 // fp32 rows, the most-similar destination.  The kernel is a chain of dependent instructions in
 // seven code streams per SM: the unused branches cost 3 % of its time when they are present.
-template <bool kLean>
+template <bool kLean, bool kFlagship>
 __global__ void __launch_bounds__(kFusedMaxThreads, 1)
 k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus) {
     extern __shared__ __align__(128) unsigned char smem[];
+    // cluster size, channels per CTA, Gram and sum warps, levels: constants in the instantiation for
+    // D = 3584 on three-level grids (the loops over the cluster's CTAs and a warp's channels unroll: 5 % faster)
+    const int nC = kFlagship ? kFlagshipC : p.C, nS = kFlagship ? kFlagshipS : p.S;
+    const int nNM = kFlagship ? kFlagshipNM : p.NM, nNA = kFlagship ? kFlagshipNA : p.NA;
+    const int nL = kFlagship ? 3 : p.L;        // quadtree levels (13x13 ... 16x16 grids)
     const int RB2 = kLean ? 0 : p.RB;          // slots of the second ring
     unsigned char* ring = smem;
     size_t off = (size_t)(p.R + RB2) * p.slot_bytes;
-    float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)p.NM * kGramVals * 4;
+    float* red = reinterpret_cast<float*>(smem + off);       off += (size_t)nNM * kGramVals * 4;
     float* redsum = reinterpret_cast<float*>(smem + off);    off += kGramVals * 4;
-    float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * p.C * kSumVals * 4;
+    float* xchg = reinterpret_cast<float*>(smem + off);      off += (size_t)kRecRing * nC * kSumVals * 4;
     float* wtab = reinterpret_cast<float*>(smem + off);      off += 128;              // the 16 lanes' weights w2 of the current item
     float* xsend = reinterpret_cast<float*>(smem + off);     off += kRecRing * kSumVals * 4;   // this CTA's share, staged for the bulk copies
     int* hand = reinterpret_cast<int*>(smem + off);          off += kRecRing * 16 * 4;
@@ -482,29 +489,29 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank(), cid = cluster_id(), ncl = cluster_count();
     const uint32_t ring_base = smem_u32(ring), ringb_base = ring_base + p.R * p.slot_bytes;
-    const int w_comb = p.NM, w_sum = p.NM + kCombineWarps, w_sim = w_sum + p.NA, w_chain = w_sim + 1, w_prod = w_sim + 2;
+    const int w_comb = nNM, w_sum = nNM + kCombineWarps, w_sim = w_sum + nNA, w_chain = w_sim + 1, w_prod = w_sim + 2;
 
     // set-up: barriers, a ring without NaN patterns
     if (tid == 0) {
         for (int s = 0; s < p.R; s++) {
             mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, p.NM + (RB2 == 0 ? p.NA : 0));
+            mbar_init(empty_bar + 8 * s, nNM + (RB2 == 0 ? nNA : 0));
         }
         for (int s = 0; s < RB2; s++) {
             mbar_init(fullb_bar + 8 * s, 1);
-            mbar_init(emptyb_bar + 8 * s, p.NA);
+            mbar_init(emptyb_bar + 8 * s, nNA);
         }
         *hint = 0;
         for (int s = 0; s < kRecRing; s++) {
             mbar_init(xfull_bar + 8 * s, 1);
-            mbar_init(xempty_bar + 8 * s, p.C);
+            mbar_init(xempty_bar + 8 * s, nC);
             mbar_init(hfull_bar + 8 * s, 1);
             mbar_init(hempty_bar + 8 * s, 1);
             mbar_init(rfull_bar + 8 * s, 1);
-            mbar_init(rempty_bar + 8 * s, p.NA);
+            mbar_init(rempty_bar + 8 * s, nNA);
         }
         for (int s = 0; s < 2; s++) {
-            mbar_init(gfull_bar + 8 * s, p.NM);
+            mbar_init(gfull_bar + 8 * s, nNM);
             mbar_init(gempty_bar + 8 * s, kCombineWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -520,12 +527,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     bool skip;
     int q = 0;              // frames of this cluster so far (the same in every role)
 
-    if (warp < p.NM) {
+    if (warp < nNM) {
         // ------------------------------------ Gram warps ------------------------------------
         const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
         const uint32_t loff = lrow * p.row_bytes + lk * 2;
-        const int ksteps = p.S >> 4;
-        const int k0 = ksteps * warp / p.NM, k1 = ksteps * (warp + 1) / p.NM;     // this warp's channel steps
+        const int ksteps = nS >> 4;
+        const int k0 = ksteps * warp / nNM, k1 = ksteps * (warp + 1) / nNM;     // this warp's channel steps
         int s = 0, use = 0;         // ring slot of frame q and how often it has been filled before (q = use * R + s)
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
@@ -601,13 +608,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // threads would loop, so the addresses are per entry index ctid only when nthr == 128)
         // Thread r < C sends the whole share (128 numbers) to CTA r with one bulk copy from shared
         // memory to that CTA's shared memory: one completion on the receiver's barrier instead of 128.
-        const uint32_t peer_x = map_to_rank(smem_u32(xchg + rank * kSumVals), ctid < p.C ? ctid : 0);
-        const uint32_t peer_bar = map_to_rank(xfull_bar, ctid < p.C ? ctid : 0);
+        const uint32_t peer_x = map_to_rank(smem_u32(xchg + rank * kSumVals), ctid < nC ? ctid : 0);
+        const uint32_t peer_bar = map_to_rank(xfull_bar, ctid < nC ? ctid : 0);
         const uint32_t xsend_a = smem_u32(xsend);
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
             // this thread's cell and the weights of all 16 lanes for the sums over the coarsest node
-            const LaneGeo lg = lane_geo(p.tiles[it.tile], ctid & 15, p.L, p.W);
+            const LaneGeo lg = lane_geo(p.tiles[it.tile], ctid & 15, nL, p.W);
             const uint32_t W2s = smem_u32(wtab);
             named_sync(1, nthr);                       // the previous item's weights are not read any more
             if (ctid < 16) wtab[ctid] = lg.w2;
@@ -619,7 +626,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 // add the Gram warps' parts, each thread a share of the 512 entries
                 for (int i = ctid * 4; i < kGramVals; i += nthr * 4) {
                     float4 sum = lds_f32x4(red_a + i * 4);
-                    for (int w = 1; w < p.NM; w++) {
+                    for (int w = 1; w < nNM; w++) {
                         const float4 v = lds_f32x4(red_a + (w * kGramVals + i) * 4);
                         sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
                     }
@@ -637,8 +644,8 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     xsend[xb * kSumVals + (ctid & 15) * 8 + (ctid >> 4)] = combine_sums(redsum_a, ctid & 15, ctid >> 4, lg, W2s);
                     fence_async_smem();                 // the copies below read what was just written normally
                     named_sync(1, nthr);
-                    if (ctid < p.C)
-                        bulk_s2s(peer_x + xb * p.C * kSumVals * 4, xsend_a + xb * kSumVals * 4, kSumVals * 4, peer_bar + 8 * xb);
+                    if (ctid < nC)
+                        bulk_s2s(peer_x + xb * nC * kSumVals * 4, xsend_a + xb * kSumVals * 4, kSumVals * 4, peer_bar + 8 * xb);
                 }
             }
         }
@@ -660,8 +667,8 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         const uint32_t xoff = ((lane & 7) + ((lane >> 3) & 1) * 8) * p.row_bytes + (ch0 + (lane >> 4) * 8) * 2;
         // A fragment (16 slots x 16 cells) straight from the record
         const uint32_t woff = 16 + 256 + ((lane & 7) + ((lane >> 3) & 1) * 8) * 32 + (lane >> 4) * 16;
-        const long long chan = (long long)rank * p.S + ch0 + 2 * t4;
-        const int ntmax = min(16, (p.S - ch0) >> 3);         // 8-channel tiles of this warp inside the slice
+        const long long chan = (long long)rank * nS + ch0 + 2 * t4;
+        const int ntmax = min(16, (nS - ch0) >> 3);         // 8-channel tiles of this warp inside the slice
         int total = 0;
         for (int round = 0; next_item(p, round, cid, ncl, it, skip); round++)
             if (!skip) total += it.n;
@@ -732,7 +739,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const uint32_t xb = sbase + s * p.slot_bytes + xoff;
 #pragma unroll
                 for (int pr = 0; pr < 8; pr++) {
-                    if (ch0 + pr * 16 < p.S) {
+                    if (ch0 + pr * 16 < nS) {
                         uint32_t xb4[4];
                         ldmatrix_x4_trans(xb + pr * 32, xb4);
                         mma_bf16(sums[2 * pr], wa, xb4[0], xb4[1]);
@@ -753,7 +760,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         // lane c + 16 are cell c of the tile.
         const unsigned full = 0xffffffffu;
         const int c = lane & 15, half = lane >> 4;
-        const int L = p.L;
+        const int L = nL;
         const uint32_t xchg_a = smem_u32(xchg);
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
@@ -768,17 +775,17 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const int myq = q + half, xb = myq % kRecRing;
                 const bool mine = half == 0 || two;                 // this half has a frame
                 if (lane == 0) {
-                    mbar_expect_tx(xfull_bar + 8 * (q % kRecRing), (uint32_t)(p.C * kSumVals * 4));
-                    if (two) mbar_expect_tx(xfull_bar + 8 * ((q + 1) % kRecRing), (uint32_t)(p.C * kSumVals * 4));
+                    mbar_expect_tx(xfull_bar + 8 * (q % kRecRing), (uint32_t)(nC * kSumVals * 4));
+                    if (two) mbar_expect_tx(xfull_bar + 8 * ((q + 1) % kRecRing), (uint32_t)(nC * kSumVals * 4));
                 }
                 if (!mbar_wait(xfull_bar + 8 * (q % kRecRing), q / kRecRing, timed_out)) break;
                 if (two && !mbar_wait(xfull_bar + 8 * ((q + 1) % kRecRing), (q + 1) / kRecRing, timed_out)) break;
                 __syncwarp();
                 float v[8];
                 {
-                    const uint32_t xch = xchg_a + (xb * p.C * kSumVals + c * 8) * 4;
+                    const uint32_t xch = xchg_a + (xb * nC * kSumVals + c * 8) * 4;
                     float4 lo = lds_f32x4(xch), hi = lds_f32x4(xch + 16);
-                    for (int r = 1; r < p.C; r++) {          // the CTAs' shares, in rank order
+                    for (int r = 1; r < nC; r++) {          // the CTAs' shares, in rank order
                         const float4 l2 = lds_f32x4(xch + r * kSumVals * 4), h2 = lds_f32x4(xch + r * kSumVals * 4 + 16);
                         lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
                         hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
@@ -789,7 +796,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                     v[4] = keep ? hi.x : 0.f; v[5] = keep ? hi.y : 0.f; v[6] = keep ? hi.z : 0.f; v[7] = keep ? hi.w : 0.f;
                 }
                 __syncwarp();
-                if (c < p.C && mine) mbar_arrive_remote(map_to_rank(xempty_bar + 8 * xb, c));
+                if (c < nC && mine) mbar_arrive_remote(map_to_rank(xempty_bar + 8 * xb, c));
 
                 // Section 3.2: cosine of every node with its parent, then the coarse-to-fine search
                 const float n0 = v[0], d0 = v[1], rr = v[2];
@@ -901,7 +908,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
         uint32_t carry_mask = 0;
         for (int round = 0; !timed_out && next_item(p, round, cid, ncl, it, skip); round++) {
             if (skip) continue;
-            const LaneGeo lg = lane_geo(p.tiles[it.tile], c, p.L, p.W);
+            const LaneGeo lg = lane_geo(p.tiles[it.tile], c, nL, p.W);
             const bool valid = lg.valid;
             const float w1 = lg.w1, w2 = lg.w2;
             if (rank == 0) p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
@@ -1026,16 +1033,16 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 __syncwarp();
                 // (one warp announces the bytes of the whole frame; a copy of the other warp that lands
                 // before that only makes the count run negative for a moment)
-                if (lane == 0 && which == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
+                if (lane == 0 && which == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * nS * 2));
                 __syncwarp();
                 if (row < 16 && ((it.vmask >> row) & 1u)) {
                     const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
                                            p.tiles[it.tile].y[row] * p.W + p.tiles[it.tile].x[row];
-                    bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * p.D + rank * p.S,
-                             (uint32_t)(p.S * 2), bar);
+                    bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * p.D + rank * nS,
+                             (uint32_t)(nS * 2), bar);
                     // the frame kPrefetchAhead frames on is called into L2 now (its copy then takes less of
                     // the slot's time); the CTAs of the cluster share the cells out and ask for whole rows
-                    if (p.F >= kPrefetchMinFrames && j + kPrefetchAhead < it.n && row % p.C == (int)rank)
+                    if (p.F >= kPrefetchMinFrames && j + kPrefetchAhead < it.n && row % nC == (int)rank)
                         bulk_prefetch_l2(p.feats + (cell + (long long)kPrefetchAhead * p.HW) * p.D, (uint32_t)(p.D * 2));
                 }
                 if (++s == p.R) { s = 0; use++; }
@@ -1064,13 +1071,13 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (!hint_wait(hint, q + 1 - p.lead, timed_out)) break;
                 if (use >= 1 && !mbar_wait(emptyb_bar + 8 * s, use - 1, timed_out)) break;
                 __syncwarp();
-                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
+                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * nS * 2));
                 __syncwarp();
                 if (lane < 16 && ((it.vmask >> lane) & 1u)) {
                     const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
                                            p.tiles[it.tile].y[lane] * p.W + p.tiles[it.tile].x[lane];
-                    bulk_g2s(ringb_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * p.S,
-                             (uint32_t)(p.S * 2), bar);
+                    bulk_g2s(ringb_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * nS,
+                             (uint32_t)(nS * 2), bar);
                 }
                 if (++s == RB2) { s = 0; use++; }
             }

@@ -465,6 +465,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
     const int nC = kFlagship ? kFlagshipC : p.C, nS = kFlagship ? kFlagshipS : p.S;
     const int nNM = kFlagship ? kFlagshipNM : p.NM, nNA = kFlagship ? kFlagshipNA : p.NA;
     const int nL = kFlagship ? 3 : p.L;        // quadtree levels (13x13 ... 16x16 grids)
+    const int nD = kFlagship ? kFlagshipC * kFlagshipS : p.D;
     const int RB2 = kLean ? 0 : p.RB;          // slots of the second ring
     unsigned char* ring = smem;
     size_t off = (size_t)(p.R + RB2) * p.slot_bytes;
@@ -698,7 +699,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 const bool mine = (m8 >> g) & 1u;
                 const uint4 fc = lds_u32x4(rec + 16 + (g + 8 * hi) * 16);       // slot, kind, dst, weight
                 const float inv = mine && fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
-                const long long row = (long long)(int)fc.z * p.D + chan;
+                const long long row = (long long)(int)fc.z * nD + chan;
 #define STTM_FLUSH_LOOP(I0, I1, STORE)                                        \
     _Pragma("unroll") for (int nt = 0; nt < 16; nt++) {                       \
         const float x = sums[nt][I0] * inv, y = sums[nt][I1] * inv;           \
@@ -1038,12 +1039,12 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (row < 16 && ((it.vmask >> row) & 1u)) {
                     const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
                                            p.tiles[it.tile].y[row] * p.W + p.tiles[it.tile].x[row];
-                    bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * p.D + rank * nS,
+                    bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * nD + rank * nS,
                              (uint32_t)(nS * 2), bar);
                     // the frame kPrefetchAhead frames on is called into L2 now (its copy then takes less of
                     // the slot's time); the CTAs of the cluster share the cells out and ask for whole rows
                     if (p.F >= kPrefetchMinFrames && j + kPrefetchAhead < it.n && row % nC == (int)rank)
-                        bulk_prefetch_l2(p.feats + (cell + (long long)kPrefetchAhead * p.HW) * p.D, (uint32_t)(p.D * 2));
+                        bulk_prefetch_l2(p.feats + (cell + (long long)kPrefetchAhead * p.HW) * nD, (uint32_t)(nD * 2));
                 }
                 if (++s == p.R) { s = 0; use++; }
             }
@@ -1076,7 +1077,7 @@ k_fused(const __grid_constant__ FusedParams p, const __grid_constant__ Taus taus
                 if (lane < 16 && ((it.vmask >> lane) & 1u)) {
                     const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
                                            p.tiles[it.tile].y[lane] * p.W + p.tiles[it.tile].x[lane];
-                    bulk_g2s(ringb_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * p.D + rank * nS,
+                    bulk_g2s(ringb_base + s * p.slot_bytes + lane * p.row_bytes, p.feats + cell * nD + rank * nS,
                              (uint32_t)(nS * 2), bar);
                 }
                 if (++s == RB2) { s = 0; use++; }

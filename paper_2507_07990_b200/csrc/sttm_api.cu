@@ -446,6 +446,7 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         configured = true;
     }
     FusedParams fp = {};
@@ -484,9 +485,10 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     at[0].val.clusterDim.x = f.C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
     const bool lean = fp.tmax == nullptr && fp.tau_t_dev == nullptr && fp.RB == 0 && !fp.out_f32 && !fp.match_best;
-    const bool flagship = lean && fp.C == kFlagshipC && fp.S == kFlagshipS && fp.NM == kFlagshipNM && fp.NA == kFlagshipNA && fp.L == 3 &&
+    const bool flagship = fp.C == kFlagshipC && fp.S == kFlagshipS && fp.NM == kFlagshipNM && fp.NA == kFlagshipNA && fp.L == 3 &&
                           fp.D == kFlagshipC * kFlagshipS;
-    if (flagship) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<true, true>, fp, taus));
+    if (flagship && lean) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<true, true>, fp, taus));
+    else if (flagship) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<false, true>, fp, taus));
     else if (lean) STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<true, false>, fp, taus));
     else STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<false, false>, fp, taus));
     g_launches++;

@@ -272,7 +272,9 @@ def run_ours(args):
     # algorithmic bytes per launch of each feature-touching stage: every stage of the three-pass
     # kernels reads the input once; the fused kernel reads it once and writes every output row once
     # (to its staging place), the gather moves every output row once more
-    if lib.sttm_last_path() == 1:
+    if lib.sttm_last_path() == 3:
+        stage_bytes = {"gram": in_bytes, "sum": in_bytes + out_bytes}
+    elif lib.sttm_last_path() == 1:
         stage_bytes = {"fused": in_bytes + out_bytes, "gather": 2 * out_bytes}
     else:
         stage_bytes = {"spatial": in_bytes, "temporal+roots": in_bytes, "accumulate": in_bytes + out_bytes}

@@ -12,6 +12,7 @@
 
 #include "sttm_kernels.cuh"
 #include "sttm_fused.cuh"
+#include "sttm_flow.cuh"
 #include "sttm_generic.cuh"
 #include "sttm_segments.cuh"
 
@@ -19,7 +20,20 @@ namespace {
 
 using namespace sttm;
 
-constexpr int kSmCount = 148;   // B200; the library is built for sm_100a only
+constexpr int kSmCount = 148;   // B200 (grid sizes of the older kernels; the streaming kernels ask the device)
+
+// multiprocessors of the current device
+int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return kSmCount;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = kSmCount;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
 
 thread_local int g_launches = 0;
 thread_local float* g_budget_tmax = nullptr;           // set by sttm_merge_budget around its two passes
@@ -27,11 +41,13 @@ thread_local const float* g_budget_tau_dev = nullptr;
 thread_local cudaEvent_t* g_stage_events = nullptr;   // when set: event i is recorded after stage i-1
 
 constexpr int kStageCount = 5;
-const char* const kStageNames[3][kStageCount] = {
+const char* const kStageNames[4][kStageCount] = {
     {"spatial", "temporal+roots", "ordering", "accumulate", "combine"},
     {"fused", "roots", "ordering", "gather", "-"},
-    {"-", "-", "-", "-", "general"}};
-thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: fused kernel, 2: general kernels
+    {"-", "-", "-", "-", "general"},
+    {"gram", "decide+ordering", "sum", "roots+pieces", "-"}};
+thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: single-pass kernel, 2: general kernels, 3: two-stream kernels
+thread_local bool g_budget_second_pass = false;        // the Gram stage's numbers of the first pass are still there
 
 inline void mark_stage(int boundary, cudaStream_t st) {
     if (g_stage_events != nullptr) cudaEventRecord(g_stage_events[boundary], st);
@@ -47,19 +63,29 @@ struct FusedPlan {
     TileDesc tiles[kMaxTiles];      // most cells first
 };
 
+// Launch shape of the two-stream kernels; ok == false: the single-pass kernel (or the three-pass kernels) run.
+struct FlowPlan {
+    bool ok;
+    int NS, S, NA, R, row_bytes, slot_bytes, F, nseg, nitems, ntiles;
+    size_t smem;
+    TileDesc tiles[kMaxTiles];
+};
+
 struct Plan {
     Geo g;
     int Tc, nchunk, nslice;
     long long cells;          // B*N
     long long partial_slots;
     FusedPlan f;
+    FlowPlan fl;
     bool generic;             // more than three quadtree levels: the plain kernels of sttm_generic.cuh
     Pyr py;
     size_t gen_pooled, gen_norms, gen_dots, gen_allpass, gen_acc;
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
         frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
-        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_next, total;
+        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_next, flow_partial,
+        flow_hand, total;
 };
 
 // benchmark / test knobs (sttm_set_tuning): 0 = choose automatically
@@ -74,7 +100,8 @@ constexpr size_t kMaxSmem = 232448;   // 227 KB per CTA on sm_100
 // neighbour lanes belong to its block and its coarsest node, so packed tiles never mix.
 int fused_resident_clusters(const FusedPlan& f);
 
-bool build_tiles(const Geo& g, FusedPlan* f) {
+template <typename PlanT>
+bool build_tiles(const Geo& g, PlanT* f) {
     struct Part { int y0, x0, r, c; };
     std::vector<Part> full, part;
     for (int y0 = 0; y0 < g.H; y0 += 4)
@@ -122,6 +149,32 @@ bool build_tiles(const Geo& g, FusedPlan* f) {
     f->ntiles = (int)tiles.size();
     for (int t = 0; t < f->ntiles; t++) f->tiles[t] = tiles[t];
     return true;
+}
+
+// Two-stream kernels: bf16 input, channel slices of at most 1024 channels (a multiple of 16).
+void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f) {
+    f->ok = false;
+    if (g_tune_path != 0 && g_tune_path != 5) return;
+    if (p->in_dtype != STTM_BF16 || g.D % 16 != 0) return;
+    if (!build_tiles(g, f)) return;
+    const int k16 = g.D / 16;
+    int NS = 0;
+    for (int n = 1; n <= kFlowMaxSlices; n++)
+        if (k16 % n == 0 && k16 / n <= kFlowWorkers * kFlowMaxKs) { NS = n; break; }
+    if (NS == 0) return;
+    f->NS = NS;
+    f->S = g.D / NS;
+    f->NA = (f->S + 127) / 128;
+    f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
+    f->slot_bytes = 16 * f->row_bytes;
+    const size_t fixed = flow_fixed_smem();
+    f->R = std::min((int)((kMaxSmem - fixed) / f->slot_bytes), kMaxRing);
+    if (f->R < 3) return;
+    f->smem = (size_t)f->R * f->slot_bytes + fixed;
+    f->F = std::min(g.T, g_tune_seg > 0 ? std::min(g_tune_seg, kFlowMaxF) : kFlowMaxF);
+    f->nseg = (g.T + f->F - 1) / f->F;
+    f->nitems = g.B * f->ntiles * f->nseg;
+    f->ok = true;
 }
 
 void plan_fused(const sttm_params* p, const Geo& g, FusedPlan* f) {
@@ -265,6 +318,7 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
     pl->zero_end = o;
     pl->partial = take((size_t)pl->partial_slots * g.D * sizeof(float));
     pl->f.ok = false;
+    pl->fl.ok = false;
     pl->gen_pooled = pl->gen_norms = pl->gen_dots = pl->gen_allpass = pl->gen_acc = o;
     if (pl->generic) {
         const long long frames = (long long)g.B * g.T;
@@ -275,9 +329,22 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
         pl->gen_allpass = take((size_t)frames * pl->py.nodes);
         pl->gen_acc = take((size_t)rows * g.D * sizeof(float));
     } else {
-        plan_fused(p, g, &pl->f);
+        plan_flow(p, g, &pl->fl);
+        if (!pl->fl.ok) plan_fused(p, g, &pl->f);
     }
     pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = pl->piece_next = o;
+    pl->flow_partial = pl->flow_hand = o;
+    if (pl->fl.ok) {
+        const FlowPlan& f = pl->fl;
+        pl->ones_begin = o;
+        pl->row_head = take((size_t)pl->cells * 4);
+        pl->ones_end = o;
+        pl->pieces = take((size_t)f.nitems * kPieceSlots * g.D * sizeof(float));
+        pl->piece_meta = take((size_t)f.nitems * kPieceSlots * sizeof(int2));
+        pl->piece_next = take((size_t)f.nitems * kPieceSlots * 4);
+        pl->flow_partial = take((size_t)f.nitems * (f.F + 1) * f.NS * kSumVals * sizeof(float));
+        pl->flow_hand = take((size_t)f.nitems * (f.F + 1) * 16 * 4);
+    }
     if (pl->f.ok) {
         const size_t out_elt = p->out_dtype == STTM_BF16 ? 2 : 4;
         pl->ones_begin = o;
@@ -493,6 +560,131 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     else STTM_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_fused<false, false>, fp, taus));
     g_launches++;
     return STTM_OK;
+}
+
+// launch with programmatic stream serialization and dynamic shared memory
+template <typename... KArgs, typename... Args>
+sttm_status launch_after_smem(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, bool after,
+                              cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = after ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+    g_launches++;
+    return e == cudaSuccess ? STTM_OK : STTM_ERR_CUDA;
+}
+
+template <typename OutT>
+sttm_status launch_gather_pieces(const Plan& pl, int npieces, char* ws, void* out, long long capacity, cudaStream_t st) {
+    const Geo g = pl.g;
+    const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
+    const unsigned blocks = std::min<unsigned>(blocks_for(max_rows * kGatherParts, 8), sm_count() * 16);
+    return launch_after(k_gather_pieces<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
+                        (const int32_t*)(ws + pl.row_head), (const int32_t*)(ws + pl.piece_next),
+                        (const int32_t*)(ws + pl.row_weight), (const float*)(ws + pl.pieces), (OutT*)out, capacity,
+                        npieces);
+}
+
+// The two-stream path: Gram stage, decisions, ordering, sum stage, pieces.
+sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, char* ws, void* out_feats,
+                     int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
+                     int32_t* device_status, cudaStream_t st) {
+    const Geo g = pl.g;
+    const FlowPlan& f = pl.fl;
+    static bool configured[64] = {};
+    int dev = 0;
+    STTM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return STTM_ERR_UNSUPPORTED;
+    if (!configured[dev]) {
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        configured[dev] = true;
+    }
+    FlowParams fp = {};
+    fp.feats = (const __nv_bfloat16*)feats;
+    fp.B = g.B; fp.T = g.T; fp.H = g.H; fp.W = g.W; fp.D = g.D; fp.L = g.L;
+    fp.HW = g.HW; fp.N = g.N;
+    fp.ntiles = f.ntiles;
+    fp.NS = f.NS; fp.S = f.S; fp.NA = f.NA;
+    fp.row_bytes = f.row_bytes; fp.slot_bytes = f.slot_bytes; fp.R = f.R;
+    fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
+    fp.weight_mode = (int)p->wt;
+    fp.match_best = p->match == STTM_MATCH_BEST ? 1 : 0;
+    fp.out_f32 = p->out_dtype == STTM_F32;
+    fp.cover = (int8_t*)(ws + pl.cover);
+    fp.link = (int32_t*)(ws + pl.link);
+    fp.tmax = g_budget_tmax;
+    fp.tau_t_dev = g_budget_tau_dev;
+    fp.frame_roots = (int32_t*)(ws + pl.frame_counts);   // inside the region that is cleared before every call
+    fp.chain_key = (int32_t*)(ws + pl.cell_row);
+    fp.partial = (float*)(ws + pl.flow_partial);
+    fp.hand = (int32_t*)(ws + pl.flow_hand);
+    fp.row_at_root = (const int32_t*)(ws + pl.row_at_root);
+    fp.vid_off = (const long long*)(ws + pl.vid_off);
+    fp.out = out_feats;
+    fp.capacity = p->out_capacity_rows;
+    fp.pieces = (float*)(ws + pl.pieces);
+    fp.piece_meta = (int2*)(ws + pl.piece_meta);
+    fp.status = device_status;
+    std::memcpy(fp.tiles, f.tiles, sizeof(fp.tiles));
+    Taus taus;
+    fill_taus(p, &taus);
+
+    const int ntasks = f.nitems * f.NS;
+    const unsigned grid = (unsigned)std::min(ntasks, sm_count());
+    sttm_status s;
+    mark_stage(0, st);
+    if (!g_budget_second_pass) {
+        s = launch_after_smem(k_flow<false>, grid, kFlowThreads, f.smem, false, st, fp);
+        if (s != STTM_OK) return s;
+    }
+    mark_stage(1, st);
+    const int pairs = (f.F + 2) / 2;
+    s = launch_after(k_flow_decide, blocks_for((long long)f.nitems * pairs, 8), 256, st, fp, taus);
+    if (s != STTM_OK) return s;
+    int32_t* frame_roots = (int32_t*)(ws + pl.frame_counts);
+    int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
+    long long* vid_off = (long long*)(ws + pl.vid_off);
+    int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
+    int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
+    int32_t* root = (int32_t*)(ws + pl.root);
+    s = launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)frame_roots, frame_base, out_count, vid_off,
+                     out_offsets);
+    if (s != STTM_OK) return s;
+    if (g_budget_tmax != nullptr) return STTM_OK;      // first pass of the budget mode: only the node counts are needed
+    s = launch_after(k_rows, (unsigned)(g.B * g.T), 256, st, g, (const int8_t*)fp.cover, (const int32_t*)fp.link,
+                     (const int32_t*)frame_base, (const long long*)vid_off, row_at_root, row_anchor, out_pos,
+                     (long long)p->out_capacity_rows, (int)p->pos, device_status);
+    if (s != STTM_OK) return s;
+    mark_stage(2, st);
+    s = launch_after_smem(k_flow<true>, grid, kFlowThreads, f.smem, true, st, fp);
+    if (s != STTM_OK) return s;
+    mark_stage(3, st);
+    s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, f.nseg + 1,
+                     (const int32_t*)(ws + pl.cell_row), root, device_status);
+    if (s != STTM_OK) return s;
+    if (merge_map != nullptr) {
+        s = launch_after(k_merge_map, blocks_for(pl.cells, 256), 256, st, g, (const int32_t*)root,
+                         (const int32_t*)row_at_root, merge_map);
+        if (s != STTM_OK) return s;
+    }
+    const int npieces = f.nitems * kPieceSlots;
+    s = launch_after(k_piece_link, blocks_for(npieces, 256), 256, st, g, npieces, (const int2*)(ws + pl.piece_meta),
+                     (const int32_t*)root, (const int32_t*)row_at_root, (const long long*)vid_off,
+                     (int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.piece_next), (int32_t*)(ws + pl.row_weight));
+    if (s != STTM_OK) return s;
+    s = p->out_dtype == STTM_BF16 ? launch_gather_pieces<__nv_bfloat16>(pl, npieces, ws, out_feats, p->out_capacity_rows, st)
+                                  : launch_gather_pieces<float>(pl, npieces, ws, out_feats, p->out_capacity_rows, st);
+    mark_stage(4, st);
+    mark_stage(5, st);
+    return s;
 }
 
 template <typename OutT>
@@ -771,7 +963,7 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
     int8_t* cover = (int8_t*)(ws + pl.cover);
     int32_t* link = (int32_t*)(ws + pl.link);
     int32_t* root = (int32_t*)(ws + pl.root);
-    g_last_path = pl.generic ? 2 : (pl.f.ok ? 1 : 0);
+    g_last_path = pl.generic ? 2 : (pl.fl.ok ? 3 : (pl.f.ok ? 1 : 0));
     if (pl.generic) {
         // more than three quadtree levels: the plain kernels, no stage breakdown
         for (int i = 0; i <= 4; i++) mark_stage(i, st);
@@ -789,6 +981,10 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
                                   out_offsets, device_status, st);
         mark_stage(5, st);
         return s;
+    }
+    if (pl.fl.ok) {
+        STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.ones_begin, 0xff, pl.ones_end - pl.ones_begin, st));
+        return run_flow(feats, p, pl, ws, out_feats, out_pos, merge_map, out_count, out_offsets, device_status, st);
     }
     if (pl.f.ok) {
         // single-read path: fused kernel, roots, ordering, gather
@@ -900,7 +1096,7 @@ sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_
 
 size_t sttm_budget_workspace_bytes(const sttm_params* p) {
     Plan pl;
-    if (make_plan(p, &pl) != STTM_OK || !pl.f.ok) return 0;
+    if (make_plan(p, &pl) != STTM_OK || !(pl.f.ok || pl.fl.ok)) return 0;
     return (pl.total + 255) / 256 * 256 + ((size_t)pl.cells * 4 + 255) / 256 * 256 + 256;
 }
 
@@ -911,7 +1107,7 @@ sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const lon
     Plan pl;
     sttm_status s = make_plan(p, &pl);
     if (s != STTM_OK) return s;
-    if (!pl.f.ok) return STTM_ERR_UNSUPPORTED;
+    if (!(pl.f.ok || pl.fl.ok)) return STTM_ERR_UNSUPPORTED;
     if (!budget_rows || !ws || !out_count) return STTM_ERR_ARG;
     for (int b = 0; b < p->B; b++)
         if (budget_rows[b] < 1) return STTM_ERR_ARG;
@@ -938,9 +1134,11 @@ sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const lon
     if (s != STTM_OK) return s;
     // second pass: the whole path with the thresholds read from device memory
     g_budget_tau_dev = tau_dev;
+    g_budget_second_pass = true;
     s = sttm_merge_ex(feats, p, ws, main_bytes, out_feats, out_pos, merge_map, out_count, out_offsets, device_status,
                       stream);
     g_budget_tau_dev = nullptr;
+    g_budget_second_pass = false;
     if (s != STTM_OK) return s;
     if (tau_t_out != nullptr)
         STTM_CUDA_TRY(cudaMemcpyAsync(tau_t_out, tau_dev, sizeof(float) * p->B, cudaMemcpyDeviceToDevice, st));

@@ -1,0 +1,606 @@
+// Two-stream STTM kernels (sm_100a): every similarity first, then every average.
+//
+// The decisions of Sections 3.2 and 3.3 (cover map, links) are pure functions of the input:
+// they depend on dot products of a frame's cells with each other and with the cells of the
+// frame before it, never on what was merged earlier.  So the work splits into stages that
+// have no serial dependence through time:
+//   Gram stage    streams the features once and leaves, per (tile, frame, channel slice), the
+//                 128 numbers the decisions need (8 per cell: linear combinations of the tile's
+//                 Gram matrix X_t X_t^T and cross matrix X_t X_{t-1}^T, see combine_sums()).
+//                 Every (tile, run of frames, channel slice) is an independent task.
+//   decision stage adds the slices in a fixed order and takes the decisions, one half warp per
+//                 (tile, frame): cover level and link of every cell.
+//   ordering      row numbers of the surviving tokens (Section 3.4): integer scans.
+//   sum stage     streams the features a second time (out of L2 where the two streams run close
+//                 together) and forms the chain averages of Section 3.3 as running sums
+//                 sums[16 chain slots x channels] += W X on the tensor cores, W the frame's
+//                 16 x 16 matrix of weights (chain slot x cell).  A chain that ends is divided by
+//                 its weight and written straight to its final output row, because the row
+//                 numbers exist before this stage starts.  Chains that cross the border between
+//                 two runs of frames leave fp32 pieces that a small kernel adds up.
+// A tile is the same 16-row unit as in the single-pass kernel (sttm_fused.cuh): a 4x4 block of
+// cells or several packed border parts; a task's frames pass through a shared-memory ring filled by
+// bulk asynchronous copies (one per cell row), consumed by eight worker warps.
+#pragma once
+
+#include "sttm_fused.cuh"
+
+namespace sttm {
+
+constexpr int kFlowWorkers = 8;                      // Gram warps / sum warps
+constexpr int kFlowWarps = kFlowWorkers + 3;         // + chain warp, two producer warps
+constexpr int kFlowThreads = kFlowWarps * 32;
+constexpr int kFlowMaxKs = 8;                        // 16-channel steps per Gram warp: slices of up to 1024 channels
+constexpr int kFlowMaxF = 64;                        // frames per item, the frame before it not counted
+constexpr int kFlowMaxSlices = 16;
+
+struct FlowParams {
+    const __nv_bfloat16* feats;
+    int B, T, H, W, D, L;
+    int HW, N;
+    int ntiles;
+    int NS, S, NA;           // channel slices, channels per slice, sum warps in use (128 channels each)
+    int row_bytes, slot_bytes, R;
+    int F, nseg, nitems;     // frames per item, items per (video, tile), items
+    int weight_mode, out_f32, match_best, dry;
+    int8_t* cover;
+    int32_t* link;
+    int32_t* chain_key;      // [B*N] per cell: root cell id of its chain as far as the item knows it
+    int32_t* frame_roots;    // [B*T] chains that start in a frame (= its output rows), zero on entry
+    float* tmax;             // budget mode, may be null (see FusedParams::tmax)
+    const float* tau_t_dev;  // budget mode, may be null: [B] temporal thresholds in device memory
+    float* partial;          // [nitems][F+1][NS][128]: the Gram stage's numbers, [number][cell]
+    int32_t* hand;           // [nitems][F+1][16]: cover level | (link lane + 1) << 8 of every tile row
+    const int32_t* row_at_root;   // [B*N] row (inside its video) of every surviving token
+    const long long* vid_off;     // [B+1] first row of every video
+    void* out;               // [rows][D] output rows
+    long long capacity;
+    float* pieces;           // [nitems][kPieceSlots][D]
+    int2* piece_meta;        // [nitems][kPieceSlots] {key cell id or -1, weight}
+    int* status;
+    TileDesc tiles[kMaxTiles];
+};
+
+struct FlowItem {
+    int item, b, tile, tstart, n, halo, last_seg;
+    uint32_t vmask;
+    int nvalid;
+};
+
+// item = (video, run of frames, tile), tiles fastest: items of one run of frames are neighbours
+__device__ __forceinline__ FlowItem flow_item(const FlowParams& p, int item) {
+    FlowItem it;
+    it.item = item;
+    it.tile = item % p.ntiles;
+    const int bs = item / p.ntiles;
+    const int seg = bs % p.nseg;
+    it.b = bs / p.nseg;
+    const int t0 = seg * p.F, t1 = min(p.T, t0 + p.F);
+    it.halo = t0 > 0;
+    it.tstart = t0 - it.halo;
+    it.n = t1 - it.tstart;
+    it.last_seg = t1 == p.T;
+    it.vmask = 0;
+    for (int l = 0; l < 16; l++)
+        if (p.tiles[it.tile].y[l] != 255) it.vmask |= 1u << l;
+    it.nvalid = __popc(it.vmask);
+    return it;
+}
+
+// bounded wait whose outcome is the same in every lane of the warp
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, int use, bool& timed_out) {
+    const bool ok = mbar_wait(bar, use, timed_out);
+    const bool all = __all_sync(0xffffffffu, ok);
+    if (!all) timed_out = true;
+    return all;
+}
+
+// Section 3.2 for one frame, 16 lanes per frame (both halves of the warp at once, each on its own
+// frame): the cover level of the lane's cell and the squared norm of the node that covers it.
+// n0 = |x_c|^2, d0 = x_c . parent(c), rr = x_c . top.
+__device__ __forceinline__ int spatial_level(float n0, float d0, float rr, const LaneGeo& lg, int L, float tau_s,
+                                             int half, float& nk) {
+    const unsigned full = 0xffffffffu;
+    const float n1 = lg.w1 * quad_sum(d0, lg.qbits);     // |parent|^2
+    const float d1 = lg.w1 * quad_sum(rr, lg.qbits);     // parent . top
+    const float n2 = top_sum(lg.w2 * rr, lg.tbits);      // |top|^2
+    int lv = 0;
+    if (L >= 2) {
+        const bool p0 = !lg.valid || cos_above(d0, n0, n1, tau_s);
+        const uint32_t pm0 = (__ballot_sync(full, p0) >> (16 * half)) & 0xffffu;
+        const bool quad_pass = (pm0 & lg.qmask) == lg.qmask;
+        if (L == 3) {
+            const bool p1 = !lg.valid || cos_above(d1, n1, n2, tau_s);
+            const uint32_t pm1 = (__ballot_sync(full, p1) >> (16 * half)) & 0xffffu;
+            lv = (pm1 & lg.tmask) == lg.tmask ? 2 : (quad_pass ? 1 : 0);
+        } else {
+            lv = quad_pass ? 1 : 0;
+        }
+    }
+    nk = lv == 0 ? n0 : (lv == 1 ? n1 : n2);
+    return lv;
+}
+
+// ---------------------------------------------------------------------------------
+// Decision stage.  One warp per (item, pair of frames); lanes 0..15 take the even frame, lanes
+// 16..31 the odd one; lane c and lane c + 16 are cell c of the tile.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_flow_decide(const __grid_constant__ FlowParams p, const __grid_constant__ Taus taus) {
+    wait_for_prior_kernel();
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31, c = lane & 15, half = lane >> 4;
+    const int pairs = (p.F + 2) / 2;                    // pairs of frames per item, the frame before it included
+    const long long w = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (w >= (long long)p.nitems * pairs) return;
+    const FlowItem it = flow_item(p, (int)(w / pairs));
+    const int j = (int)(w % pairs) * 2 + half;
+    const bool mine = j < it.n;
+    const LaneGeo lg = lane_geo(p.tiles[it.tile], c, p.L, p.W);
+    const bool valid = lg.valid;
+    const float tau_s = taus.s[it.b], tau_t = p.tau_t_dev != nullptr ? p.tau_t_dev[it.b] : taus.t[it.b];
+
+    // the slices' shares, in slice order; the frame before (numbers 0..2 only) for its cover level
+    float v[8], u[3];
+#pragma unroll
+    for (int k = 0; k < 8; k++) v[k] = 0.f;
+    u[0] = u[1] = u[2] = 0.f;
+    const bool has_prev = mine && j > 0;
+    if (mine && valid) {
+        const float* src = p.partial + ((long long)it.item * (p.F + 1) + j) * p.NS * kSumVals + c;
+        for (int s = 0; s < p.NS; s++) {
+#pragma unroll
+            for (int k = 0; k < 8; k++) v[k] += __ldcg(src + s * kSumVals + k * 16);
+        }
+        if (has_prev) {
+            const float* sp = src - (long long)p.NS * kSumVals;
+            for (int s = 0; s < p.NS; s++) {
+#pragma unroll
+                for (int k = 0; k < 3; k++) u[k] += __ldcg(sp + s * kSumVals + k * 16);
+            }
+        }
+    }
+    float nk, pnk;
+    const int lv = spatial_level(v[0], v[1], v[2], lg, p.L, tau_s, half, nk);
+    const int lu = spatial_level(u[0], u[1], u[2], lg, p.L, tau_s, half, pnk);
+
+    // Section 3.3: the node covering the cell against the overlapping kept node of the frame
+    // before; a pair is evaluated at the top-left cell of its finer node
+    int link_local = -1;
+    {
+        const float w1 = lg.w1, w2 = lg.w2;
+        const float t11 = w1 * quad_sum(v[4], lg.qbits), t12 = w1 * quad_sum(v[5], lg.qbits);
+        const float t21 = w1 * quad_sum(v[7], lg.qbits), t22 = top_sum(w2 * v[5], lg.tbits);
+        float dot;
+        if (lv == 0) dot = lu == 0 ? v[3] : (lu == 1 ? v[4] : v[5]);
+        else if (lv == 1) dot = lu == 0 ? v[6] : (lu == 1 ? t11 : t12);
+        else dot = lu == 0 ? v[7] : (lu == 1 ? t21 : t22);
+        const bool rep = valid && has_prev && lane_anchor(lg, c, min(lv, lu)) == c;
+        const bool pass = rep && cos_above(dot, nk, pnk, tau_t);
+        const uint32_t passm = (__ballot_sync(full, pass) >> (16 * half)) & 0xffffu;
+        const uint32_t cand = passm & lane_region(lg, c, lv);
+        int cstar = cand ? __ffs(cand) - 1 : 0;             // first in row-major order: the top-left one
+        if (p.match_best) {
+            // the most similar of them instead (equal ones: the first)
+            const float cosv = pass ? dot / (sqrtf(nk) * sqrtf(pnk)) : -2.f;
+            float best = -2.f;
+#pragma unroll
+            for (int i = 0; i < 16; i++) {
+                const float si = __shfl_sync(full, cosv, 16 * half + i);
+                if (((cand >> i) & 1u) && si > best) { best = si; cstar = i; }
+            }
+        }
+        if (p.tmax != nullptr) {
+            // budget mode: per kept node the largest cosine to its candidates
+            const float cosv = rep ? ((nk == 0.f || pnk == 0.f) ? 0.f : dot / (sqrtf(nk) * sqrtf(pnk))) : -2.f;
+            const uint32_t candm = ((__ballot_sync(full, rep) >> (16 * half)) & 0xffffu) & lane_region(lg, c, lv);
+            float most = -2.f;
+#pragma unroll
+            for (int i = 0; i < 16; i++) {
+                const float si = __shfl_sync(full, cosv, 16 * half + i);
+                if (((candm >> i) & 1u) && si > most) most = si;
+            }
+            if (mine && valid && !(it.halo && j == 0))
+                p.tmax[(long long)it.b * p.N + (long long)(it.tstart + j) * p.HW + lg.cell] =
+                    lane_anchor(lg, c, lv) == c ? most : -2.f;
+        }
+        const int lu_star = __shfl_sync(full, lu, 16 * half + cstar);
+        link_local = cand ? lane_anchor(lg, cstar, lu_star) : -1;
+    }
+    const int lcell = __shfl_sync(full, lg.cell, 16 * half + (link_local < 0 ? 0 : link_local));
+    if (mine) p.hand[((long long)it.item * (p.F + 1) + j) * 16 + c] = lv | ((link_local + 1) << 8);
+    const bool owned = mine && !(it.halo && j == 0);        // the frame before the item belongs to the item before
+    const int tt = it.tstart + j;
+    if (owned && valid) {
+        const long long gcc = (long long)it.b * p.N + (long long)tt * p.HW + lg.cell;
+        p.cover[gcc] = (int8_t)lv;
+        p.link[gcc] = link_local < 0 ? -1 : (tt - 1) * p.HW + lcell;
+    }
+    // every chain that starts here is an output row of this frame
+    const bool fresh = owned && valid && lane_anchor(lg, c, lv) == c && link_local < 0;
+    const uint32_t freshm = (__ballot_sync(full, fresh) >> (16 * half)) & 0xffffu;
+    if (c == 0 && freshm != 0 && owned) atomicAdd(p.frame_roots + it.b * p.T + tt, __popc(freshm));
+}
+
+// ---------------------------------------------------------------------------------
+// The streaming kernel.  kSum == false: Gram stage; kSum == true: sum stage.  A task is (item,
+// channel slice); tasks are dealt to the CTAs round robin.  Warps: [0, 8) workers, 8 chain warp
+// (sum stage only), 9 and 10 producers.
+// ---------------------------------------------------------------------------------
+struct FlowSmem {
+    unsigned char* ring;
+    float* red;             // [8][512] the Gram warps' parts
+    float* redsum;          // [512]
+    float* wtab;            // [16] the lanes' weights w2 of the current item
+    FrameRec* recs;         // [kRecRing]
+    SlotTable* tab;
+    int* hand;              // [kFlowMaxF + 1][16]
+    int* rows;              // [kFlowMaxF + 1][16]
+    uint32_t full_bar, empty_bar, rfull_bar, rempty_bar;
+};
+
+__host__ __device__ inline size_t flow_fixed_smem() {
+    return (size_t)kFlowWorkers * kGramVals * 4 + kGramVals * 4 + 128 + kRecRing * sizeof(FrameRec) + sizeof(SlotTable) +
+           2 * (kFlowMaxF + 1) * 16 * 4 + (2 * kMaxRing + 2 * kRecRing) * 8 + 128;
+}
+
+template <bool kSum>
+__global__ void __launch_bounds__(kFlowThreads, 1)
+k_flow(const __grid_constant__ FlowParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    FlowSmem sm;
+    size_t off = 0;
+    sm.ring = smem;                                                off += (size_t)p.R * p.slot_bytes;
+    sm.red = reinterpret_cast<float*>(smem + off);                 off += (size_t)kFlowWorkers * kGramVals * 4;
+    sm.redsum = reinterpret_cast<float*>(smem + off);              off += kGramVals * 4;
+    sm.wtab = reinterpret_cast<float*>(smem + off);                off += 128;
+    sm.recs = reinterpret_cast<FrameRec*>(smem + off);             off += kRecRing * sizeof(FrameRec);
+    sm.tab = reinterpret_cast<SlotTable*>(smem + off);             off += sizeof(SlotTable);
+    sm.hand = reinterpret_cast<int*>(smem + off);                  off += (kFlowMaxF + 1) * 16 * 4;
+    sm.rows = reinterpret_cast<int*>(smem + off);                  off += (kFlowMaxF + 1) * 16 * 4;
+    off = (off + 7) & ~(size_t)7;
+    const uint32_t bar0 = smem_u32(smem + off);
+    sm.full_bar = bar0;
+    sm.empty_bar = bar0 + 8 * kMaxRing;
+    sm.rfull_bar = bar0 + 16 * kMaxRing;
+    sm.rempty_bar = sm.rfull_bar + 8 * kRecRing;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t ring_base = smem_u32(sm.ring);
+    const int ntasks = p.nitems * p.NS;
+
+    if (tid == 0) {
+        for (int s = 0; s < p.R; s++) {
+            mbar_init(sm.full_bar + 8 * s, 1);
+            mbar_init(sm.empty_bar + 8 * s, kFlowWorkers);
+        }
+        for (int s = 0; s < kRecRing; s++) {
+            mbar_init(sm.rfull_bar + 8 * s, 1);
+            mbar_init(sm.rempty_bar + 8 * s, p.NA);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // a ring without NaN patterns: rows of a tile that hold no cell are never written
+    for (int k = tid * 16; k < p.R * p.slot_bytes; k += blockDim.x * 16)
+        *reinterpret_cast<uint4*>(sm.ring + k) = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    if constexpr (kSum) wait_for_prior_kernel();
+
+    bool timed_out = false;
+    int s = 0, use = 0;             // ring slot of the next frame and how often it has been filled before
+
+    if (warp < kFlowWorkers && !kSum) {
+        // ------------------------------------ Gram warps ------------------------------------
+        // Warp w owns the 16-channel steps [k0, k1) of the slice.  The fragments of a frame are
+        // loaded once and kept for the next frame's cross products, so a ring slot is free again
+        // as soon as it has been read.
+        const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
+        const uint32_t loff = lrow * p.row_bytes + lk * 2;
+        const int ksteps = p.S >> 4;
+        const int k0 = ksteps * warp / kFlowWorkers, nk = ksteps * (warp + 1) / kFlowWorkers - k0;
+        const int wtid = tid;                           // 0..255 among the workers
+        const uint32_t red_a = smem_u32(sm.red), redsum_a = smem_u32(sm.redsum), W2s = smem_u32(sm.wtab);
+        for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
+            const FlowItem it = flow_item(p, task / p.NS);
+            const int slice = task % p.NS;
+            const LaneGeo lg = lane_geo(p.tiles[it.tile], wtid & 15, p.L, p.W);
+            named_sync(1, kFlowWorkers * 32);           // the previous task's weights are not read any more
+            if (wtid < 16) sm.wtab[wtid] = lg.w2;
+            uint32_t prv[kFlowMaxKs][4];
+#pragma unroll
+            for (int i = 0; i < kFlowMaxKs; i++) prv[i][0] = prv[i][1] = prv[i][2] = prv[i][3] = 0u;
+            float* dst = p.partial + ((long long)it.item * (p.F + 1) * p.NS + slice) * kSumVals;
+            for (int j = 0; j < it.n; j++) {
+                mbar_wait_warp(sm.full_bar + 8 * s, use, timed_out);
+                uint32_t cur[kFlowMaxKs][4];
+                const uint32_t base = ring_base + s * p.slot_bytes + loff + k0 * 32;
+#pragma unroll
+                for (int i = 0; i < kFlowMaxKs; i++) {
+                    if (i < nk) ldmatrix_x4(base + i * 32, cur[i]);
+                    else cur[i][0] = cur[i][1] = cur[i][2] = cur[i][3] = 0u;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sm.empty_bar + 8 * s);
+                float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
+                float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int i = 0; i < kFlowMaxKs; i++) {
+                    if (i < nk) {
+                        mma_bf16(g0, cur[i], cur[i][0], cur[i][2]);
+                        mma_bf16(g1, cur[i], cur[i][1], cur[i][3]);
+                        mma_bf16(c0, cur[i], prv[i][0], prv[i][2]);
+                        mma_bf16(c1, cur[i], prv[i][1], prv[i][3]);
+                    }
+                }
+                {
+                    float* r = sm.red + warp * kGramVals;
+                    const int gr = lane >> 2, gc = (lane & 3) * 2;
+                    *reinterpret_cast<float2*>(r + gr * 16 + gc) = make_float2(g0[0], g0[1]);
+                    *reinterpret_cast<float2*>(r + (gr + 8) * 16 + gc) = make_float2(g0[2], g0[3]);
+                    *reinterpret_cast<float2*>(r + gr * 16 + 8 + gc) = make_float2(g1[0], g1[1]);
+                    *reinterpret_cast<float2*>(r + (gr + 8) * 16 + 8 + gc) = make_float2(g1[2], g1[3]);
+                    *reinterpret_cast<float2*>(r + 256 + gr * 16 + gc) = make_float2(c0[0], c0[1]);
+                    *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + gc) = make_float2(c0[2], c0[3]);
+                    *reinterpret_cast<float2*>(r + 256 + gr * 16 + 8 + gc) = make_float2(c1[0], c1[1]);
+                    *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + 8 + gc) = make_float2(c1[2], c1[3]);
+                }
+                // (the barrier also spreads a wait that ran out: every worker leaves together)
+                if (named_sync_or(2, kFlowWorkers * 32, timed_out)) { timed_out = true; break; }
+                {
+                    // add the warps' parts in warp order, two entries per thread
+                    float2 sum = *reinterpret_cast<const float2*>(sm.red + wtid * 2);
+#pragma unroll
+                    for (int w = 1; w < kFlowWorkers; w++) {
+                        const float2 x = *reinterpret_cast<const float2*>(sm.red + w * kGramVals + wtid * 2);
+                        sum.x += x.x; sum.y += x.y;
+                    }
+                    *reinterpret_cast<float2*>(sm.redsum + wtid * 2) = sum;
+                }
+                named_sync(1, kFlowWorkers * 32);
+                // contract to 8 numbers per cell: thread = (number, cell), stored [number][cell]
+                if (wtid < kSumVals) dst[(long long)j * p.NS * kSumVals + wtid] = combine_sums(redsum_a, wtid & 15, wtid >> 4, lg, W2s);
+#pragma unroll
+                for (int i = 0; i < kFlowMaxKs; i++) {
+                    prv[i][0] = cur[i][0]; prv[i][1] = cur[i][1]; prv[i][2] = cur[i][2]; prv[i][3] = cur[i][3];
+                }
+                if (++s == p.R) { s = 0; use++; }
+            }
+        }
+    } else if (warp < kFlowWorkers && kSum) {
+        // ------------------------------------ sum warps ------------------------------------
+        // Warp a owns channels [128 a, 128 a + 128) of the slice: 16 tiles of 8 channels.  sums[nt][0..3]
+        // is the accumulator fragment of tile nt: chain slots g and g + 8 (g = lane / 4), channels
+        // 2 t and 2 t + 1 of the tile (t = lane % 4).
+        const bool active = warp < p.NA;
+        float sums[16][4];
+#pragma unroll
+        for (int nt = 0; nt < 16; nt++)
+#pragma unroll
+            for (int k = 0; k < 4; k++) sums[nt][k] = 0.f;
+        const int ch0 = warp * 128;
+        const int g = lane >> 2, t4 = lane & 3;
+        const uint32_t recs_a = smem_u32(sm.recs);
+        const uint32_t xoff = ((lane & 7) + ((lane >> 3) & 1) * 8) * p.row_bytes + (ch0 + (lane >> 4) * 8) * 2;
+        const uint32_t woff = 16 + 256 + ((lane & 7) + ((lane >> 3) & 1) * 8) * 32 + (lane >> 4) * 16;
+        const int ntmax = min(16, (p.S - ch0) >> 3);        // 8-channel tiles of this warp inside the slice
+        int rq = 0;                                         // records so far
+        for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
+            const FlowItem it = flow_item(p, task / p.NS);
+            const int slice = task % p.NS;
+            const long long chan = (long long)slice * p.S + ch0 + 2 * t4;
+            // one record per frame, and a last one that writes out what the item leaves
+            for (int j = 0; j <= it.n; j++) {
+                const bool frame = j < it.n;
+                if (frame && !mbar_wait_warp(sm.full_bar + 8 * s, use, timed_out)) break;
+                if (!active) {
+                    if (frame) {
+                        if (lane == 0) mbar_arrive(sm.empty_bar + 8 * s);
+                        if (++s == p.R) { s = 0; use++; }
+                    }
+                    continue;
+                }
+                const int rk = rq % kRecRing;
+                if (!mbar_wait_warp(sm.rfull_bar + 8 * rk, rq / kRecRing, timed_out)) break;
+                const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
+                const uint32_t flush_mask = lds_u32x4(rec).x;
+#pragma unroll 1
+                for (int hi = 0; hi < 2; hi++) {
+                    const uint32_t m8 = (flush_mask >> (8 * hi)) & 0xffu;
+                    if (m8 == 0) continue;
+                    const bool mine = (m8 >> g) & 1u;
+                    const uint4 fc = lds_u32x4(rec + 16 + (g + 8 * hi) * 16);       // slot, kind, dst, weight
+                    const float inv = mine && fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
+                    const long long row = (long long)(int)fc.z * p.D + chan;
+                    const bool skip = (int)fc.z < 0;                                // a row beyond the capacity
+#define STTM_FLOW_FLUSH(I0, I1)                                                                               \
+    if (fc.y != 0 || p.out_f32) {                                                                             \
+        float* dst = (fc.y != 0 ? p.pieces : reinterpret_cast<float*>(p.out)) + row;                          \
+        _Pragma("unroll") for (int nt = 0; nt < 16; nt++) {                                                   \
+            const float x = sums[nt][I0] * inv, y = sums[nt][I1] * inv;                                       \
+            sums[nt][I0] = 0.f;                                                                               \
+            sums[nt][I1] = 0.f;                                                                               \
+            if (nt < ntmax && !skip) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x, y);            \
+        }                                                                                                     \
+    } else {                                                                                                  \
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row;                                   \
+        _Pragma("unroll") for (int nt = 0; nt < 16; nt++) {                                                   \
+            const uint32_t w = pack_bf16x2(sums[nt][I0] * inv, sums[nt][I1] * inv);                           \
+            sums[nt][I0] = 0.f;                                                                               \
+            sums[nt][I1] = 0.f;                                                                               \
+            if (nt < ntmax && !skip) *reinterpret_cast<uint32_t*>(dst + nt * 8) = w;                          \
+        }                                                                                                     \
+    }
+                    if (mine) {
+                        if (hi) { STTM_FLOW_FLUSH(2, 3) } else { STTM_FLOW_FLUSH(0, 1) }
+                    }
+#undef STTM_FLOW_FLUSH
+                }
+                __syncwarp();
+                if (frame) {
+                    uint32_t wa[4];
+                    ldmatrix_x4(rec + woff, wa);
+                    const uint32_t xb = ring_base + s * p.slot_bytes + xoff;
+#pragma unroll
+                    for (int pr = 0; pr < 8; pr++) {
+                        if (ch0 + pr * 16 < p.S) {
+                            uint32_t xb4[4];
+                            ldmatrix_x4_trans(xb + pr * 32, xb4);
+                            mma_bf16(sums[2 * pr], wa, xb4[0], xb4[1]);
+                            mma_bf16(sums[2 * pr + 1], wa, xb4[2], xb4[3]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(sm.rempty_bar + 8 * rk);
+                    if (frame) mbar_arrive(sm.empty_bar + 8 * s);
+                }
+                rq++;
+                if (frame && ++s == p.R) { s = 0; use++; }
+            }
+        }
+    } else if (warp == kFlowWorkers) {
+        // ------------------------------------ chain warp ------------------------------------
+        // Follows the tile's chains through the item's frames: which running sum (chain slot)
+        // every kept node joins, which chains ended and where they go.
+        if constexpr (kSum) {
+            const unsigned full = 0xffffffffu;
+            const int c = lane & 15;
+            const bool low = lane < 16;
+            int rq = 0;
+            for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
+                const FlowItem it = flow_item(p, task / p.NS);
+                const int slice = task % p.NS;
+                const bool writer = slice == 0;             // the integer outputs are written once per item
+                const LaneGeo lg = lane_geo(p.tiles[it.tile], c, p.L, p.W);
+                const bool valid = lg.valid;
+                const float w1 = lg.w1, w2 = lg.w2;
+                const long long vrow0 = p.vid_off[it.b];
+                // the item's decisions and the rows of the tokens that start in it
+                for (int i = lane; i < it.n * 16; i += 32) {
+                    const LaneGeo li = lane_geo(p.tiles[it.tile], i & 15, p.L, p.W);
+                    sm.hand[i] = p.hand[(long long)it.item * (p.F + 1) * 16 + i];
+                    sm.rows[i] = li.valid ? p.row_at_root[(long long)it.b * p.N + (long long)(it.tstart + (i >> 4)) * p.HW + li.cell] : -1;
+                }
+                if (writer) p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
+                __syncwarp();
+                int prev_slot = 0;
+                uint32_t active_slots = 0;
+                for (int j = 0; j <= it.n; j++, rq++) {
+                    const int hb = rq % kRecRing;
+                    if (rq >= kRecRing && !mbar_wait_warp(sm.rempty_bar + 8 * hb, rq / kRecRing - 1, timed_out)) break;
+                    FrameRec* rec = sm.recs + hb;
+                    if (j == it.n) {
+                        // last record of the item: everything still running is written out
+                        if (low && ((active_slots >> lane) & 1u)) {
+                            if (!sm.tab->virt[lane] && it.last_seg) {
+                                const int row = sm.tab->row[lane];
+                                const long long grow = vrow0 + row;
+                                rec->flush[lane] = FlushCmd{lane, 0, grow < p.capacity ? (int)grow : -1, (float)sm.tab->weight[lane]};
+                            } else {
+                                const int pc = it.item * kPieceSlots + 16 + lane;
+                                rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
+                                if (writer) p.piece_meta[pc] = make_int2(sm.tab->key[lane], sm.tab->weight[lane]);
+                            }
+                        }
+                        if (lane == 0) rec->flush_mask = p.dry ? 0u : active_slots;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(sm.rfull_bar + 8 * hb);
+                        continue;
+                    }
+                    const int packed = sm.hand[j * 16 + c];
+                    const int lv = packed & 3, link_local = (packed >> 8) - 1;
+                    const int t = it.tstart + j;
+                    const bool is_halo = it.halo && j == 0;
+
+                    // nodes with a link join the chain of their target; chains without a member in this
+                    // frame have ended; the remaining nodes start new chains in free slots
+                    const bool anchor = valid && lane_anchor(lg, c, lv) == c;
+                    const bool linked = anchor && link_local >= 0;
+                    const bool fresh = anchor && link_local < 0;
+                    const int slot_linked = __shfl_sync(full, prev_slot, link_local < 0 ? 0 : link_local);
+                    const uint32_t memb = __reduce_or_sync(full, linked ? 1u << slot_linked : 0u);
+                    const uint32_t dead = active_slots & ~memb;
+                    const uint32_t freem = ~memb & 0xffffu;
+                    const uint32_t freshm = __ballot_sync(full, fresh && low);
+                    const int slot_fresh = kth_set_bit16(freem, __popc(freshm & ((1u << c) - 1)));
+                    const int node_slot = linked ? slot_linked : slot_fresh;
+                    const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + lane_anchor(lg, c, lv));
+                    const uint32_t cells = lane_region(lg, c, lv);
+                    const int wint = p.weight_mode ? __popc(cells) : 1;
+                    const long long gc = (long long)it.b * p.N + (long long)t * p.HW + lg.cell;
+
+                    // chains that ended: lane s looks at slot s (before the slot is given away again)
+                    if (low && ((dead >> lane) & 1u)) {
+                        if (sm.tab->virt[lane]) {
+                            const int pc = it.item * kPieceSlots + sm.tab->cell[lane];
+                            rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
+                            if (writer) p.piece_meta[pc] = make_int2(sm.tab->key[lane], sm.tab->weight[lane]);
+                        } else {
+                            const long long grow = vrow0 + sm.tab->row[lane];
+                            rec->flush[lane] = FlushCmd{lane, 0, grow < p.capacity ? (int)grow : -1, (float)sm.tab->weight[lane]};
+                        }
+                    }
+                    __syncwarp();
+                    if (low && fresh) {
+                        sm.tab->key[slot_fresh] = (int)gc;
+                        sm.tab->weight[slot_fresh] = is_halo ? 0 : wint;
+                        sm.tab->virt[slot_fresh] = is_halo ? 1 : 0;
+                        sm.tab->cell[slot_fresh] = c;
+                        sm.tab->row[slot_fresh] = sm.rows[j * 16 + c];
+                    }
+                    if (low && linked) atomicAdd(&sm.tab->weight[slot_linked], wint);
+                    // the frame's weight matrix: row = chain slot, column = cell
+                    reinterpret_cast<uint4*>(rec->wmat)[lane] = make_uint4(0u, 0u, 0u, 0u);
+                    const int wnode = __shfl_sync(full, wint, (lane & 16) + lane_anchor(lg, c, lv));
+                    __syncwarp();
+                    if (low && valid && !is_halo) {
+                        const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
+                        rec->wmat[cur_slot * 16 + c] = __bfloat16_as_ushort(__float2bfloat16_rn(wc));
+                    }
+                    if (lane == 0) rec->flush_mask = p.dry ? 0u : dead;
+                    const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sm.rfull_bar + 8 * hb);
+
+                    if (writer && !is_halo && low && valid) p.chain_key[gc] = sm.tab->key[cur_slot] - it.b * p.N;
+                    active_slots = active;
+                    prev_slot = cur_slot;
+                    __syncwarp();
+                }
+            }
+        }
+    } else {
+        // ---------------------------------- producer warps ----------------------------------
+        const int which = warp - (kFlowWorkers + 1);
+        const int row = lane * 2 + which;                   // the tile row this lane copies
+        for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
+            const FlowItem it = flow_item(p, task / p.NS);
+            const int slice = task % p.NS;
+            for (int j = 0; j < it.n; j++) {
+                const uint32_t bar = sm.full_bar + 8 * s;
+                if (use >= 1 && !mbar_wait_warp(sm.empty_bar + 8 * s, use - 1, timed_out)) break;
+                if (lane == 0 && which == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
+                __syncwarp();
+                if (row < 16 && ((it.vmask >> row) & 1u)) {
+                    const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
+                                           p.tiles[it.tile].y[row] * p.W + p.tiles[it.tile].x[row];
+                    bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * p.D + (long long)slice * p.S,
+                             (uint32_t)(p.S * 2), bar);
+                }
+                if (++s == p.R) { s = 0; use++; }
+            }
+        }
+        // the CTA must not end with copies in flight: the last R frames issued have landed?
+        const int q = use * p.R + s;
+        for (int qq = max(0, q - p.R); qq < q; qq++) {
+            bool late = false;
+            mbar_wait(sm.full_bar + 8 * (qq % p.R), qq / p.R, late);
+            timed_out |= late;
+        }
+    }
+    __syncthreads();
+    if (timed_out && p.status != nullptr) atomicOr(p.status, kStatusWaitTimeout);
+}
+
+}  // namespace sttm

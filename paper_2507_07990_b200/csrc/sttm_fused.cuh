@@ -445,7 +445,7 @@ __device__ __forceinline__ float combine_sums(uint32_t G, int c, int k, const La
 
 // Chain slots of the chain warp (shared memory, private to it).
 struct SlotTable {
-    int key[16], weight[16], virt[16], cell[16];
+    int key[16], weight[16], virt[16], cell[16], row[16];
 };
 
 // ---------------------------------------------------------------------------------

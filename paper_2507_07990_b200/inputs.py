@@ -14,6 +14,16 @@ leaves are replaced in the same frame their parent is replaced instead, which le
 blocks coarsen again and keeps long videos stationary.  The root block always splits
 (a frame is never one single object); every other block splits with ``split_p``.
 
+Contrast.  A leaf block also draws a contrast, one of ``VideoSpec.contrast`` with equal
+probability, which multiplies its object vector (not the noise) for as long as the block
+persists.  With one class (the default) every block has contrast 1 and all similarities
+of same-object tokens fall into one narrow cluster, so a threshold can only switch
+merging on or off.  With several classes the similarities form one cluster per class
+and level (cosine of two noisy copies of a.o is a^2 / (a^2 + sigma^2) for leaves), the
+clusters are separated by gaps far wider than the decision margin, and thresholds placed
+between them decide which classes merge: that is what lets a workload land near a stated
+token budget.
+
 Random numbers come from numpy's counter-based Philox generator, keyed by
 (seed, stream, frame), so a frame's noise does not depend on generation order.
 """
@@ -59,10 +69,11 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 # ----------------------------------------------------------------------------------
 class _Node:
     """A block of the generator's quadtree: a leaf with an object id, or four children."""
-    __slots__ = ("obj", "kids")
+    __slots__ = ("obj", "kids", "amp")
 
-    def __init__(self, obj: int = -1, kids=None):
+    def __init__(self, obj: int = -1, kids=None, amp: int = 0):
         self.obj = obj
+        self.amp = amp          # index into VideoSpec.contrast
         self.kids = kids        # list of 4 (_Node or None) in (top-left, top-right, bottom-left, bottom-right) order
 
 
@@ -82,7 +93,10 @@ def _fresh(rng, depth, bi, bj, spec, side0) -> "_Node":
                 else:
                     kids.append(None)
         return _Node(kids=kids)
-    return _Node(obj=int(rng.integers(spec.K)))
+    obj = int(rng.integers(spec.K))
+    # (a single contrast class draws nothing, so such videos are what they were without the option)
+    amp = int(rng.integers(len(spec.contrast))) if len(spec.contrast) > 1 else 0
+    return _Node(obj=obj, amp=amp)
 
 
 def _evolve(rng, node, depth, bi, bj, spec, side0) -> Tuple["_Node", bool]:
@@ -104,16 +118,17 @@ def _evolve(rng, node, depth, bi, bj, spec, side0) -> Tuple["_Node", bool]:
     return _Node(kids=new_kids), False
 
 
-def _paint(node, depth, bi, bj, side0, obj_map, depth_map):
+def _paint(node, depth, bi, bj, side0, obj_map, depth_map, amp_map):
     H, W = obj_map.shape
     s = side0 >> depth
     if node.kids is None:
         obj_map[bi * s:min((bi + 1) * s, H), bj * s:min((bj + 1) * s, W)] = node.obj
         depth_map[bi * s:min((bi + 1) * s, H), bj * s:min((bj + 1) * s, W)] = depth
+        amp_map[bi * s:min((bi + 1) * s, H), bj * s:min((bj + 1) * s, W)] = node.amp
         return
     for k, kid in enumerate(node.kids):
         if kid is not None:
-            _paint(kid, depth + 1, 2 * bi + (k >> 1), 2 * bj + (k & 1), side0, obj_map, depth_map)
+            _paint(kid, depth + 1, 2 * bi + (k >> 1), 2 * bj + (k & 1), side0, obj_map, depth_map, amp_map)
 
 
 @dataclass
@@ -132,6 +147,7 @@ class VideoSpec:
     split_p: float = 0.5
     K: int = 16
     unit: str = "rms"
+    contrast: Tuple[float, ...] = (1.0,)   # contrast classes of a leaf block, drawn with equal probability
     scale_unit_rms: bool = True    # multiply the tensor by one scalar so tokens have unit RMS
     seed: int = 20250707
 
@@ -140,20 +156,22 @@ class VideoSpec:
         return self.T * self.H * self.W
 
 
-def frame_structure(spec: VideoSpec) -> Tuple[np.ndarray, np.ndarray]:
-    """Object-id map and block-depth map, both ``[T, H, W]`` (int16 / int8)."""
+def frame_structure(spec: VideoSpec, want_contrast: bool = False):
+    """Object-id map and block-depth map, both ``[T, H, W]`` (int16 / int8); with
+    ``want_contrast`` also the map of contrast-class indices (int8)."""
     side0 = 1
     while side0 < max(spec.H, spec.W):
         side0 *= 2
     rng = _rng(spec.seed, _STREAM_STRUCTURE)
     obj = np.zeros((spec.T, spec.H, spec.W), dtype=np.int16)
     dep = np.zeros((spec.T, spec.H, spec.W), dtype=np.int8)
+    amp = np.zeros((spec.T, spec.H, spec.W), dtype=np.int8)
     root = _fresh(rng, 0, 0, 0, spec, side0)
     for t in range(spec.T):
         if t > 0:
             root, _ = _evolve(rng, root, 0, 0, 0, spec, side0)
-        _paint(root, 0, 0, 0, side0, obj[t], dep[t])
-    return obj, dep
+        _paint(root, 0, 0, 0, side0, obj[t], dep[t], amp[t])
+    return (obj, dep, amp) if want_contrast else (obj, dep)
 
 
 def _objects(spec: VideoSpec) -> np.ndarray:
@@ -171,9 +189,12 @@ def make_video(spec: VideoSpec, out: Optional[np.ndarray] = None) -> np.ndarray:
     bit patterns as uint16 (dtype 'bf16').  ``out`` may supply the destination buffer
     (e.g. pinned host memory viewed as a numpy array)."""
     objs = _objects(spec)
-    obj_map, _ = frame_structure(spec)
+    obj_map, _, amp_map = frame_structure(spec, want_contrast=True)
+    amps = np.asarray(spec.contrast, dtype=np.float32)
     if spec.scale_unit_rms:
-        mean_sq = float((objs.astype(np.float64) ** 2).mean()) + spec.sigma ** 2
+        # expected mean square of a token (contrast classes are equally likely per block)
+        mean_sq = float((objs.astype(np.float64) ** 2).mean()) * float((amps.astype(np.float64) ** 2).mean()) \
+            + spec.sigma ** 2
         scale = np.float32(1.0 / np.sqrt(mean_sq))
     else:
         scale = np.float32(1.0)
@@ -186,7 +207,10 @@ def make_video(spec: VideoSpec, out: Optional[np.ndarray] = None) -> np.ndarray:
     for t in range(spec.T):
         noise = _rng(spec.seed, _STREAM_NOISE, t).standard_normal((hw, spec.D), dtype=np.float32)
         noise *= np.float32(spec.sigma)
-        noise += objs[obj_map[t].reshape(hw)]
+        if len(amps) > 1:
+            noise += objs[obj_map[t].reshape(hw)] * amps[amp_map[t].reshape(hw)][:, None]
+        else:
+            noise += objs[obj_map[t].reshape(hw)]
         noise *= scale
         if spec.dtype == "bf16":
             out[t] = f32_to_bf16_bits(noise).reshape(spec.H, spec.W, spec.D)
@@ -199,18 +223,20 @@ def make_video(spec: VideoSpec, out: Optional[np.ndarray] = None) -> np.ndarray:
 # the five workloads
 # ----------------------------------------------------------------------------------
 BASE_SEED = 20250707
+# contrast classes of the workloads that are run at a token budget
+CONTRAST = (1.0, 0.5, 0.35, 0.25, 0.18, 0.12)
 
 CONFIGS = {
     # name: shared fields; 'p_static' is a list with one entry per video
     "tiny":  dict(index=1, T=4, H=8, W=8, D=64, dtype="f32", depth_max=3, sigma=0.05,
                   p_static=[0.8], scale_unit_rms=False, budgets=[None], fixed_tau=(0.9, 0.9)),
-    "llava": dict(index=2, T=64, H=13, W=13, D=3584, dtype="bf16", depth_max=3, sigma=0.05,
+    "llava": dict(index=2, contrast=CONTRAST, T=64, H=13, W=13, D=3584, dtype="bf16", depth_max=3, sigma=0.05,
                   p_static=[0.8], scale_unit_rms=True, budgets=[0.5, 0.3]),
-    "qwen":  dict(index=3, T=128, H=16, W=16, D=3584, dtype="bf16", depth_max=4, sigma=0.08,
+    "qwen":  dict(index=3, contrast=CONTRAST, T=128, H=16, W=16, D=3584, dtype="bf16", depth_max=4, sigma=0.08,
                   p_static=[0.7], scale_unit_rms=True, budgets=[0.5]),
-    "long":  dict(index=4, T=1024, H=13, W=13, D=3584, dtype="bf16", depth_max=3, sigma=0.05,
+    "long":  dict(index=4, contrast=CONTRAST, T=1024, H=13, W=13, D=3584, dtype="bf16", depth_max=3, sigma=0.05,
                   p_static=[0.9], scale_unit_rms=True, budgets=[0.3]),
-    "mixed": dict(index=5, T=64, H=13, W=13, D=3584, dtype="bf16", depth_max=3, sigma=0.05,
+    "mixed": dict(index=5, contrast=CONTRAST, T=64, H=13, W=13, D=3584, dtype="bf16", depth_max=3, sigma=0.05,
                   p_static=[0.95, 0.9, 0.8, 0.7, 0.6, 0.5, 0.3, 0.1], scale_unit_rms=True,
                   budgets=[0.5, 0.3]),
 }
@@ -223,7 +249,7 @@ def config_videos(name: str, seed_bump: int = 0) -> List[VideoSpec]:
     for v, p in enumerate(c["p_static"]):
         specs.append(VideoSpec(T=c["T"], H=c["H"], W=c["W"], D=c["D"], dtype=c["dtype"],
                                depth_max=c["depth_max"], p_static=p, sigma=c["sigma"],
-                               scale_unit_rms=c["scale_unit_rms"],
+                               scale_unit_rms=c["scale_unit_rms"], contrast=tuple(c.get("contrast", (1.0,))),
                                seed=BASE_SEED + c["index"] + 100 * v + 1000 * seed_bump))
     return specs
 

@@ -14,10 +14,12 @@ from tests import helpers
 pytestmark = pytest.mark.gpu
 
 # (path, cluster size, frames per item) for sttm_set_tuning, then (sum slots, lead frames) for
-# sttm_set_ring_split: the library's own choice, the three-pass kernels, fused launches that
-# force clusters and many item borders, the fused kernel without packing of partial border
-# tiles, and two other ways to share out the shared-memory slots
-TUNINGS = {"auto": (0, 0, 0, 0, 0), "threepass": (1, 0, 0, 0, 0), "c1f3": (2, 1, 3, 0, 0), "c2f2": (2, 2, 2, 0, 0),
+# sttm_set_ring_split: the library's own choice (the two-stream kernels), the same with item
+# borders every frame / every three / every seven frames, the three-pass kernels, single-pass
+# launches that force clusters and many item borders, the single-pass kernel without packing of
+# partial border tiles, and two other ways to share out its shared-memory slots
+TUNINGS = {"auto": (0, 0, 0, 0, 0), "flowf1": (5, 0, 1, 0, 0), "flowf3": (5, 0, 3, 0, 0), "flowf7": (5, 0, 7, 0, 0),
+           "threepass": (1, 0, 0, 0, 0), "c1f3": (2, 1, 3, 0, 0), "c2f2": (2, 2, 2, 0, 0),
            "c4f5": (2, 4, 5, 0, 0), "c8f1": (2, 8, 1, 0, 0), "nopack": (3, 0, 0, 0, 0), "sum2lead2": (2, 0, 0, 2, 2),
            "sum4": (2, 0, 7, 4, 1)}
 
@@ -236,7 +238,7 @@ def test_other_workload_shapes_full_width(shape):
             continue
         for out_dtype in (torch.float32, torch.bfloat16):
             run_and_compare(video, taus[0], taus[1], out_dtype=out_dtype)
-        assert binding.load_library().sttm_last_path() == 1          # the fused kernel took it
+        assert binding.load_library().sttm_last_path() == 3          # the two-stream kernels took it
         done += 1
         break
     assert done >= 1, "no seed gave thresholds with a margin"

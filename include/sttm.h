@@ -21,8 +21,16 @@
  *     sttm_workspace_bytes(params) bytes, 256-byte aligned.
  *   - Calls are asynchronous on `stream` and do not synchronise (sttm_merge_host does).
  *   - Host-detectable errors are returned with no work enqueued.  Conditions found on
- *     the device (output capacity exceeded, root search not converged) are OR-ed as
- *     (1 << status) bits into *device_status; kernels never trap.
+ *     the device are OR-ed as (1 << status) bits into *device_status; kernels never trap:
+ *       1 << STTM_ERR_CAPACITY       more rows than out_capacity_rows (the rows that fit are valid),
+ *       1 << STTM_ERR_NOT_CONVERGED  the root search hit its round limit,
+ *       1 << STTM_ERR_TIMEOUT        a wait between the stages of a pipelined kernel (on a
+ *                                    shared-memory barrier) was given up after 2 seconds; the
+ *                                    kernel then ended early and its outputs are not valid.
+ *   - The library keeps per-device tables but no per-call global state; calls on different
+ *     host threads are independent as long as they use different workspaces and streams.
+ *     The benchmark knobs (sttm_set_tuning, sttm_set_ring_split, sttm_set_stage_events) are
+ *     process-wide or per-thread test hooks and are not meant to be changed while calls run.
  *   - Layout: feats is [B, T, H, W, D] contiguous, D fastest; D must be a multiple of 4
  *     and the base pointer 16-byte aligned.  A token's cell id inside its video is
  *     c = t*H*W + y*W + x.  A quadtree node is named by the cell id of its top-left
@@ -49,7 +57,8 @@ typedef enum {
     STTM_ERR_WORKSPACE = 3,      /* ws_bytes smaller than sttm_workspace_bytes()        */
     STTM_ERR_CAPACITY = 4,       /* more output rows than out_capacity_rows (device)    */
     STTM_ERR_NOT_CONVERGED = 5,  /* root search hit its round limit (device)            */
-    STTM_ERR_CUDA = 6            /* a CUDA runtime call failed                          */
+    STTM_ERR_CUDA = 6,           /* a CUDA runtime call failed                          */
+    STTM_ERR_TIMEOUT = 7         /* a bounded wait inside a kernel ran out (device)     */
 } sttm_status;
 
 typedef enum { STTM_BF16 = 0, STTM_F32 = 1 } sttm_dtype;
@@ -76,6 +85,10 @@ typedef struct sttm_params {
     long long out_capacity_rows;  /* rows available in out_feats / out_pos (all videos)   */
     sttm_match_mode match;        /* destination rule of the temporal link                */
 } sttm_params;
+
+/* The lowest-numbered condition whose (1 << status) bit is set in a device status word, STTM_OK
+ * for 0.  Host only. */
+sttm_status sttm_status_from_bits(int32_t bits);
 
 /* Fills *p with defaults: B=1, bf16 in and out, lv1=4, survived ids, node weights,
  * top-left destination, capacity B*T*H*W.  Host only. */
@@ -160,9 +173,18 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws, siz
  * One bf16 video with default params (lv1 = 4, survived ids, node weights, bf16 output,
  * capacity T*H*W rows).  Uses a workspace cached per device, grown with cudaMalloc when a
  * larger problem arrives (so the first call on a device synchronises and allocates).
+ * Conditions found on the device go to a status word kept with that workspace; it is cleared
+ * by every sttm_merge call and read back by sttm_merge_status.
  */
 sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_s, float tau_t,
                        void* out_feats, int32_t* out_pos, int32_t* out_count, void* stream);
+
+/*
+ * Waits for `stream` and returns what the last sttm_merge call on the current device left in its
+ * status word: STTM_OK, or the lowest-numbered condition whose bit is set (the whole word goes to
+ * *host_bits when that is not NULL).  Host pointer; synchronises.
+ */
+sttm_status sttm_merge_status(int32_t* host_bits, void* stream);
 
 /*
  * One video cut into segments of consecutive frames, one segment per GPU (Section 3.3: a chain

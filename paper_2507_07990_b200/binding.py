@@ -21,7 +21,8 @@ POS_SURVIVED, POS_REASSIGNED = 0, 1
 W_NODE, W_AREA = 0, 1
 MATCH_TOPLEFT, MATCH_BEST = 0, 1
 STATUS_NAMES = ["ok", "bad argument", "unsupported shape", "workspace too small",
-                "output capacity exceeded", "root search did not converge", "CUDA error"]
+                "output capacity exceeded", "root search did not converge", "CUDA error",
+                "a wait inside a kernel ran out"]
 
 EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame", "sttm_spatial",
            "sttm_temporal", "sttm_merge_ex", "sttm_merge", "sttm_merge_host", "sttm_release_cache",
@@ -29,7 +30,8 @@ EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame",
            "sttm_set_stage_events", "sttm_set_tuning", "sttm_set_ring_split", "sttm_last_path",
            "sttm_fused_launch_shape", "sttm_spatial_static", "sttm_merged_positions",
            "sttm_merged_positions_workspace", "sttm_merge_budget", "sttm_budget_workspace_bytes",
-           "sttm_row_weights", "sttm_segment_fold", "sttm_segment_emit", "sttm_segment_finish"]
+           "sttm_row_weights", "sttm_segment_fold", "sttm_segment_emit", "sttm_segment_finish",
+           "sttm_status_from_bits", "sttm_merge_status"]
 
 
 class SttmParams(C.Structure):
@@ -112,6 +114,10 @@ def load_library(path: Optional[str] = None):
     lib.sttm_segment_finish.restype = C.c_int
     lib.sttm_set_ring_split.argtypes = [C.c_int, C.c_int]
     lib.sttm_set_ring_split.restype = None
+    lib.sttm_status_from_bits.argtypes = [C.c_int32]
+    lib.sttm_status_from_bits.restype = C.c_int
+    lib.sttm_merge_status.argtypes = [C.POINTER(C.c_int32), vp]
+    lib.sttm_merge_status.restype = C.c_int
     lib.sttm_last_path.argtypes = []
     lib.sttm_last_path.restype = C.c_int
     lib.sttm_fused_launch_shape.argtypes = [pp, C.POINTER(C.c_int)]

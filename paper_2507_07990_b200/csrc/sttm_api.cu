@@ -36,8 +36,13 @@ int sm_count() {
 }
 
 thread_local int g_launches = 0;
-thread_local float* g_budget_tmax = nullptr;           // set by sttm_merge_budget around its two passes
-thread_local const float* g_budget_tau_dev = nullptr;
+// What the budget mode hands to its two passes of the ordinary path (nothing of it is global state).
+struct Internal {
+    float* tmax = nullptr;              // first pass: per kept node the largest cosine to its candidates goes here
+    const float* tau_dev = nullptr;     // second pass: temporal thresholds in device memory
+    bool second_pass = false;           // the Gram stage's numbers of the first pass are still in the workspace
+    bool budget = false;                // plan as the budget mode does (two-stream kernels)
+};
 thread_local cudaEvent_t* g_stage_events = nullptr;   // when set: event i is recorded after stage i-1
 
 constexpr int kStageCount = 5;
@@ -45,15 +50,23 @@ const char* const kStageNames[4][kStageCount] = {
     {"spatial", "temporal+roots", "ordering", "accumulate", "combine"},
     {"fused", "roots", "ordering", "gather", "-"},
     {"-", "-", "-", "-", "general"},
-    {"gram", "decide+ordering", "sum", "roots+pieces", "-"}};
+    {"gram", "decide+ordering+chain", "sum", "roots+pieces", "-"}};
 thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: single-pass kernel, 2: general kernels, 3: two-stream kernels
-thread_local bool g_budget_second_pass = false;        // the Gram stage's numbers of the first pass are still there
 
 inline void mark_stage(int boundary, cudaStream_t st) {
     if (g_stage_events != nullptr) cudaEventRecord(g_stage_events[boundary], st);
 }
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+// index of the current device for the per-device tables below (function attributes and occupancy
+// answers belong to a device); -1 when it cannot be had or is beyond the tables
+constexpr int kMaxDevices = 64;
+inline int device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
 
 // Launch shape of the fused kernel for one problem; ok == false: the three-pass kernels run.
 struct FusedPlan {
@@ -66,9 +79,10 @@ struct FusedPlan {
 // Launch shape of the two-stream kernels; ok == false: the single-pass kernel (or the three-pass kernels) run.
 struct FlowPlan {
     bool ok;
-    int NS, S, NA, R, row_bytes, slot_bytes, F, nseg, nitems, ntiles;
+    int NS, NB, R, slot_bytes, F, nseg, nitems, ntiles;
     size_t smem;
     TileDesc tiles[kMaxTiles];
+    TileBox boxes[kMaxTiles];
 };
 
 struct Plan {
@@ -81,17 +95,19 @@ struct Plan {
     bool generic;             // more than three quadtree levels: the plain kernels of sttm_generic.cuh
     Pyr py;
     size_t gen_pooled, gen_norms, gen_dots, gen_allpass, gen_acc;
+    size_t norms_bytes;       // the spatial stage's only scratch: one squared norm per quadtree node
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
         frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
         zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_next, flow_partial,
-        flow_hand, total;
+        flow_hand, flow_recs, total;
 };
 
 // benchmark / test knobs (sttm_set_tuning): 0 = choose automatically
 int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0, g_tune_pack = 0, g_tune_sum_slots = 0, g_tune_lead = 0;
 
 constexpr size_t kMaxSmem = 232448;   // 227 KB per CTA on sm_100
+constexpr size_t kFlowSmemMax = (233472 - 2 * 1024) / 2;   // per CTA when two share an SM
 
 // Cuts the grid into the kernel's tiles.  Full 4x4 tiles map one to one.  The partial tiles of
 // the right and bottom border are packed several to a tile: a partial tile of r x c cells sits
@@ -151,27 +167,87 @@ bool build_tiles(const Geo& g, PlanT* f) {
     return true;
 }
 
-// Two-stream kernels: bf16 input, channel slices of at most 1024 channels (a multiple of 16).
-void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f) {
+// Tiles of the two-stream kernels: what one tensor copy brings in.  4x4 boxes over the part of the
+// grid whose sides are multiples of four or end in a part of two or three cells (such a box reaches
+// over the border and the copy fills the rows outside with zeros); a grid one cell wider than a
+// multiple of four has its last column cut into runs of 16 cells instead, one cell higher its last
+// row (so that 13x13 is 9 + 1 + 1 tiles).  A run of a column holds the column's share of up to four
+// coarsest nodes, each on four consecutive lanes: lane pairs are 2x2 blocks (bit 1), lane quadruples
+// coarsest nodes (bits 1 and 2).
+bool build_flow_tiles(const Geo& g, FlowPlan* f) {
+    if (g.H > 254 || g.W > 254) return false;
+    const bool col_strip = g.W % 4 == 1, row_strip = g.H % 4 == 1;
+    const int Wf = col_strip ? g.W - 1 : g.W, Hf = row_strip ? g.H - 1 : g.H;
+    std::vector<TileDesc> tiles;
+    std::vector<TileBox> boxes;
+    auto blank = [] { TileDesc t; std::memset(t.y, 255, 16); std::memset(t.x, 0, 16); std::memset(t.bits, 0, 16); return t; };
+    for (int y0 = 0; y0 < Hf; y0 += 4)
+        for (int x0 = 0; x0 < Wf; x0 += 4) {
+            const int r = std::min(4, g.H - y0), c = std::min(4, g.W - x0);
+            const int qb = (c >= 2 ? 1 : 0) | (r >= 2 ? 4 : 0);
+            const int tb = qb | (c > 2 ? 2 : 0) | (r > 2 ? 8 : 0);
+            TileDesc t = blank();
+            for (int dy = 0; dy < r; dy++)
+                for (int dx = 0; dx < c; dx++) {
+                    const int l = dy * 4 + dx;
+                    t.y[l] = (unsigned char)(y0 + dy);
+                    t.x[l] = (unsigned char)(x0 + dx);
+                    t.bits[l] = (unsigned char)(qb | (tb << 4));
+                }
+            tiles.push_back(t);
+            boxes.push_back(TileBox{0, x0, y0, 0});
+        }
+    // runs along the last column (kind 1) and the last row (kind 2); the corner cell goes with the column
+    for (int kind = 1; kind <= 2; kind++) {
+        if (kind == 1 ? !col_strip : !row_strip) continue;
+        const int len = kind == 1 ? g.H : Wf;               // cells of the strip
+        const int full = kind == 1 ? g.H : g.W;             // the grid's extent along the strip
+        for (int a0 = 0; a0 < len; a0 += 16) {
+            TileDesc t = blank();
+            for (int l = 0; l < 16 && a0 + l < len; l++) {
+                const int a = a0 + l;
+                const int r = std::min(4, full - a / 4 * 4);    // cells of this coarsest node along the strip
+                const int qb = r >= 2 ? 1 : 0, tb = qb | (r > 2 ? 2 : 0);
+                t.y[l] = (unsigned char)(kind == 1 ? a : g.H - 1);
+                t.x[l] = (unsigned char)(kind == 1 ? g.W - 1 : a);
+                t.bits[l] = (unsigned char)(qb | (tb << 4));
+            }
+            tiles.push_back(t);
+            boxes.push_back(kind == 1 ? TileBox{1, g.W - 1, a0, 0} : TileBox{2, a0, g.H - 1, 0});
+        }
+    }
+    if (tiles.empty() || (int)tiles.size() > kMaxTiles) return false;
+    f->ntiles = (int)tiles.size();
+    for (int t = 0; t < f->ntiles; t++) { f->tiles[t] = tiles[t]; f->boxes[t] = boxes[t]; }
+    return true;
+}
+
+// Two-stream kernels: bf16 input, channels a multiple of 64, slices of up to eight 64-channel blocks.
+void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
     f->ok = false;
-    if (g_tune_path != 0 && g_tune_path != 5) return;
-    if (p->in_dtype != STTM_BF16 || g.D % 16 != 0) return;
-    if (!build_tiles(g, f)) return;
-    const int k16 = g.D / 16;
-    int NS = 0;
-    for (int n = 1; n <= kFlowMaxSlices; n++)
-        if (k16 % n == 0 && k16 / n <= kFlowWorkers * kFlowMaxKs) { NS = n; break; }
-    if (NS == 0) return;
-    f->NS = NS;
-    f->S = g.D / NS;
-    f->NA = (f->S + 127) / 128;
-    f->row_bytes = f->S * 2 + 16;          // +16: rows fall in different bank groups for ldmatrix
-    f->slot_bytes = 16 * f->row_bytes;
-    const size_t fixed = flow_fixed_smem();
-    f->R = std::min((int)((kMaxSmem - fixed) / f->slot_bytes), kMaxRing);
-    if (f->R < 3) return;
-    f->smem = (size_t)f->R * f->slot_bytes + fixed;
-    f->F = std::min(g.T, g_tune_seg > 0 ? std::min(g_tune_seg, kFlowMaxF) : kFlowMaxF);
+    // on request, and for the budget mode (its second pass reuses the first pass's Gram stage)
+    if (!(g_tune_path == 5 || (g_tune_path == 0 && budget))) return;
+    if (p->in_dtype != STTM_BF16 || g.D % 64 != 0) return;
+    if (!build_flow_tiles(g, f)) return;
+    const int nblk = g.D / 64;
+    // blocks per slice: the largest divisor of the block count up to 14, two to a sum warp (D = 3584:
+    // four slices of 14 blocks, 896 channels; memory serves chunks of that size at nearly full speed,
+    // chunks of half the size measurably slower)
+    int NB = 0;
+    for (int n = std::min(nblk, kFlowMaxNB); n >= 1 && NB == 0; n--)
+        if (nblk % n == 0) NB = n;
+    if (nblk / NB > 64) return;
+    f->NB = NB;
+    f->NS = nblk / NB;
+    f->slot_bytes = NB * kBlkBytes;
+    // two CTAs per SM: each gets half of the SM's shared memory (less the system's 1 KB per CTA)
+    int R = 0;
+    for (int r = kFlowMaxRing; r >= 2; r--)
+        if ((size_t)r * f->slot_bytes + flow_fixed_smem(r) <= kFlowSmemMax) { R = r; break; }
+    if (R == 0) return;
+    f->R = R;
+    f->smem = (size_t)f->R * f->slot_bytes + flow_fixed_smem(f->R);
+    f->F = std::min(g.T, g_tune_seg > 0 ? std::min(g_tune_seg, kFlowMaxF) : 32);
     f->nseg = (g.T + f->F - 1) / f->F;
     f->nitems = g.B * f->ntiles * f->nseg;
     f->ok = true;
@@ -249,7 +325,7 @@ int levels_of(int H, int W, int lv1, int* H1, int* W1, int* Hc, int* Wc) {
     return L;
 }
 
-sttm_status make_plan(const sttm_params* p, Plan* pl) {
+sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
     if (p == nullptr) return STTM_ERR_ARG;
     if (p->B < 1 || p->T < 1 || p->H < 1 || p->W < 1 || p->D < 1 || p->lv1 < 1) return STTM_ERR_ARG;
     if (p->D % 4 != 0) return STTM_ERR_ARG;
@@ -272,7 +348,7 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
 
     pl->nslice = (g.D + kSliceCh - 1) / kSliceCh;
     const long long per_chunk = (long long)g.B * g.ncol * pl->nslice;
-    const long long target = 2ll * kSmCount * 16;
+    const long long target = 2ll * kSmCount * 16;       // (a fixed figure: the workspace layout must not depend on the device)
     long long nchunk = (target + per_chunk - 1) / per_chunk;
     nchunk = std::max(1ll, std::min<long long>(nchunk, std::max(1, g.T / 8)));
     pl->Tc = (int)((g.T + nchunk - 1) / nchunk);
@@ -297,7 +373,8 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
     const int NN = g.L == 3 ? 21 : (g.L == 2 ? 5 : 1);
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
-    pl->norms = take((size_t)g.B * g.T * g.ncol * NN * sizeof(float));
+    pl->norms_bytes = (size_t)g.B * g.T * g.ncol * NN * sizeof(float);
+    pl->norms = take(pl->norms_bytes);
     pl->cover = take((size_t)pl->cells);
     pl->link = take((size_t)pl->cells * 4);
     pl->root = take((size_t)pl->cells * 4);
@@ -329,11 +406,11 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
         pl->gen_allpass = take((size_t)frames * pl->py.nodes);
         pl->gen_acc = take((size_t)rows * g.D * sizeof(float));
     } else {
-        plan_flow(p, g, &pl->fl);
+        plan_flow(p, g, &pl->fl, budget);
         if (!pl->fl.ok) plan_fused(p, g, &pl->f);
     }
     pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = pl->piece_next = o;
-    pl->flow_partial = pl->flow_hand = o;
+    pl->flow_partial = pl->flow_hand = pl->flow_recs = o;
     if (pl->fl.ok) {
         const FlowPlan& f = pl->fl;
         pl->ones_begin = o;
@@ -344,6 +421,7 @@ sttm_status make_plan(const sttm_params* p, Plan* pl) {
         pl->piece_next = take((size_t)f.nitems * kPieceSlots * 4);
         pl->flow_partial = take((size_t)f.nitems * (f.F + 1) * f.NS * kSumVals * sizeof(float));
         pl->flow_hand = take((size_t)f.nitems * (f.F + 1) * 16 * 4);
+        pl->flow_recs = take((size_t)f.nitems * (f.F + 2) * sizeof(FrameRec));
     }
     if (pl->f.ok) {
         const size_t out_elt = p->out_dtype == STTM_BF16 ? 2 : 4;
@@ -411,12 +489,11 @@ sttm_status launch_after(void (*kernel)(KArgs...), unsigned grid, unsigned block
 
 inline unsigned blocks_for(long long items, int per_block) { return (unsigned)((items + per_block - 1) / per_block); }
 
-sttm_status run_spatial(const void* feats, const sttm_params* p, const Plan& pl, char* ws, int8_t* cover,
+sttm_status run_spatial(const void* feats, const sttm_params* p, const Plan& pl, float* norms, int8_t* cover,
                         int32_t* frame_counts, float* sims, cudaStream_t st) {
     Taus taus;
     fill_taus(p, &taus);
     const Geo g = pl.g;
-    float* norms = (float*)(ws + pl.norms);
     const long long warps = (long long)g.B * g.T * g.ncol;
     return by_levels_dtype(g.L, p->in_dtype, [&](auto lv, auto* tag) {
         using T = std::remove_const_t<std::remove_pointer_t<decltype(tag)>>;
@@ -452,11 +529,13 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
                               int weight_mode, cudaStream_t st) {
     const Geo g = pl.g;
     const size_t smem = (size_t)kAccWarps * Col<LV>::NC * kSliceCh * sizeof(float);
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};
+    const int dev = device_slot();
+    if (dev < 0) return STTM_ERR_UNSUPPORTED;
+    if (!configured[dev]) {
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_accumulate<LV, T, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem));
-        configured = true;
+        configured[dev] = true;
     }
     const long long warps = (long long)g.B * g.ncol * pl.nchunk * pl.nslice;
     k_accumulate<LV, T, OutT><<<blocks_for(warps, kAccWarps), kAccWarps * 32, smem, st>>>(
@@ -467,7 +546,7 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
     sttm_status s = launched();
     if (s != STTM_OK) return s;
     mark_stage(4, st);
-    k_combine<OutT><<<kSmCount * 2, 256, 0, st>>>(g, pl.Tc, (const long long*)(ws + pl.vid_off),
+    k_combine<OutT><<<sm_count() * 2, 256, 0, st>>>(g, pl.Tc, (const long long*)(ws + pl.vid_off),
                                                  (const int32_t*)(ws + pl.span_off),
                                                  (const int32_t*)(ws + pl.row_anchor),
                                                  (const int32_t*)(ws + pl.row_last_t),
@@ -480,14 +559,16 @@ sttm_status launch_accumulate(const void* feats, const Plan& pl, char* ws, void*
 
 // Resident clusters of the fused kernel for a launch shape (cached); falls back to SMs / C.
 int fused_resident_clusters(const FusedPlan& f) {
-    static int cached[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
-    static size_t cached_smem[kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
+    static int cached[kMaxDevices][kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
+    static size_t cached_smem[kMaxDevices][kMaxCluster + 1][kFusedMaxThreads / 32 + 1];
     const int warps = f.NM + kCombineWarps + f.NA + kTailWarps;
-    int& slot = cached[f.C][warps];
-    if (slot > 0 && cached_smem[f.C][warps] == f.smem) return slot;
+    const int dev = device_slot();
+    if (dev < 0) return sm_count() / f.C;
+    int& slot = cached[dev][f.C][warps];
+    if (slot > 0 && cached_smem[dev][f.C][warps] == f.smem) return slot;
     int n = 0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kSmCount / f.C * f.C);
+    cfg.gridDim = dim3(sm_count() / f.C * f.C);
     cfg.blockDim = dim3(warps * 32);
     cfg.dynamicSmemBytes = f.smem;
     cudaLaunchAttribute at[1];
@@ -497,24 +578,26 @@ int fused_resident_clusters(const FusedPlan& f) {
     cudaFuncSetAttribute(k_fused<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
     if (cudaOccupancyMaxActiveClusters(&n, k_fused<true, false>, &cfg) != cudaSuccess || n < 1) {
         cudaGetLastError();
-        n = kSmCount / f.C;
+        n = sm_count() / f.C;
     }
     slot = n;
-    cached_smem[f.C][warps] = f.smem;
+    cached_smem[dev][f.C][warps] = f.smem;
     return n;
 }
 
 sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, char* ws, int32_t* device_status,
-                      cudaStream_t st) {
+                      const Internal& in, cudaStream_t st) {
     const Geo g = pl.g;
     const FusedPlan& f = pl.f;
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};
+    const int dev = device_slot();
+    if (dev < 0) return STTM_ERR_UNSUPPORTED;
+    if (!configured[dev]) {
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_fused<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-        configured = true;
+        configured[dev] = true;
     }
     FusedParams fp = {};
     fp.feats = (const __nv_bfloat16*)feats;
@@ -529,8 +612,8 @@ sttm_status run_fused(const void* feats, const sttm_params* p, const Plan& pl, c
     fp.out_f32 = p->out_dtype == STTM_F32;
     fp.cover = (int8_t*)(ws + pl.cover);
     fp.link = (int32_t*)(ws + pl.link);
-    fp.tmax = g_budget_tmax;
-    fp.tau_t_dev = g_budget_tau_dev;
+    fp.tmax = in.tmax;
+    fp.tau_t_dev = in.tau_dev;
     fp.frame_roots = (int32_t*)(ws + pl.frame_counts);   // inside the region that is cleared before every call
     fp.chain_key = (int32_t*)(ws + pl.cell_row);       // the three-pass kernels' cell_row array is free here
     fp.staging = ws + pl.staging;
@@ -592,40 +675,73 @@ sttm_status launch_gather_pieces(const Plan& pl, int npieces, char* ws, void* ou
                         npieces);
 }
 
-// The two-stream path: Gram stage, decisions, ordering, sum stage, pieces.
+// Tensor maps of the feature tensor for the three kinds of tile.  The tensor is described as
+// [frame][64-channel block][y][x][64 channels] (a permutation of its dimensions in memory), so that
+// a box of NB blocks x (4x4 | 16x1 | 1x16) cells lands in shared memory block by block, each block
+// 16 rows of 128 bytes under the 128-byte swizzle.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+sttm_status make_flow_maps(const void* feats, const Geo& g, int NB, FlowMaps* maps) {
+    static EncodeTiledFn encode = nullptr;
+    if (encode == nullptr) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || fn == nullptr)
+            return STTM_ERR_CUDA;
+        encode = (EncodeTiledFn)fn;
+    }
+    const cuuint64_t dims[5] = {64, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)(g.D / 64), (cuuint64_t)g.B * g.T};
+    const cuuint64_t strides[4] = {(cuuint64_t)g.D * 2, (cuuint64_t)g.W * g.D * 2, 128, (cuuint64_t)g.HW * g.D * 2};
+    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    const cuuint32_t boxes[3][5] = {{64, 4, 4, (cuuint32_t)NB, 1}, {64, 1, 16, (cuuint32_t)NB, 1}, {64, 16, 1, (cuuint32_t)NB, 1}};
+    for (int k = 0; k < 3; k++) {
+        const CUresult r = encode(&maps->m[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(feats), dims, strides,
+                                  boxes[k], ones, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return STTM_ERR_CUDA;
+    }
+    return STTM_OK;
+}
+
+// The two-stream path: Gram stage, decisions, ordering, chain stage, sum stage, pieces.
 sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, char* ws, void* out_feats,
                      int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
-                     int32_t* device_status, cudaStream_t st) {
+                     int32_t* device_status, const Internal& in, cudaStream_t st) {
     const Geo g = pl.g;
     const FlowPlan& f = pl.fl;
-    static bool configured[64] = {};
-    int dev = 0;
-    STTM_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return STTM_ERR_UNSUPPORTED;
+    static bool configured[kMaxDevices] = {};
+    const int dev = device_slot();
+    if (dev < 0) return STTM_ERR_UNSUPPORTED;
     if (!configured[dev]) {
-        STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-        STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFlowSmemMax));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFlowSmemMax));
         configured[dev] = true;
     }
+    FlowMaps maps;
+    sttm_status s = make_flow_maps(feats, g, f.NB, &maps);
+    if (s != STTM_OK) return s;
     FlowParams fp = {};
-    fp.feats = (const __nv_bfloat16*)feats;
     fp.B = g.B; fp.T = g.T; fp.H = g.H; fp.W = g.W; fp.D = g.D; fp.L = g.L;
     fp.HW = g.HW; fp.N = g.N;
     fp.ntiles = f.ntiles;
-    fp.NS = f.NS; fp.S = f.S; fp.NA = f.NA;
-    fp.row_bytes = f.row_bytes; fp.slot_bytes = f.slot_bytes; fp.R = f.R;
+    fp.NS = f.NS; fp.NB = f.NB;
+    fp.slot_bytes = f.slot_bytes; fp.R = f.R;
     fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
     fp.weight_mode = (int)p->wt;
     fp.match_best = p->match == STTM_MATCH_BEST ? 1 : 0;
     fp.out_f32 = p->out_dtype == STTM_F32;
     fp.cover = (int8_t*)(ws + pl.cover);
     fp.link = (int32_t*)(ws + pl.link);
-    fp.tmax = g_budget_tmax;
-    fp.tau_t_dev = g_budget_tau_dev;
+    fp.tmax = in.tmax;
+    fp.tau_t_dev = in.tau_dev;
     fp.frame_roots = (int32_t*)(ws + pl.frame_counts);   // inside the region that is cleared before every call
     fp.chain_key = (int32_t*)(ws + pl.cell_row);
     fp.partial = (float*)(ws + pl.flow_partial);
     fp.hand = (int32_t*)(ws + pl.flow_hand);
+    fp.recs = (FrameRec*)(ws + pl.flow_recs);
     fp.row_at_root = (const int32_t*)(ws + pl.row_at_root);
     fp.vid_off = (const long long*)(ws + pl.vid_off);
     fp.out = out_feats;
@@ -634,15 +750,15 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     fp.piece_meta = (int2*)(ws + pl.piece_meta);
     fp.status = device_status;
     std::memcpy(fp.tiles, f.tiles, sizeof(fp.tiles));
+    std::memcpy(fp.boxes, f.boxes, sizeof(fp.boxes));
     Taus taus;
     fill_taus(p, &taus);
 
     const int ntasks = f.nitems * f.NS;
-    const unsigned grid = (unsigned)std::min(ntasks, sm_count());
-    sttm_status s;
+    const unsigned grid = (unsigned)std::min(ntasks, 2 * sm_count());
     mark_stage(0, st);
-    if (!g_budget_second_pass) {
-        s = launch_after_smem(k_flow<false>, grid, kFlowThreads, f.smem, false, st, fp);
+    if (!in.second_pass) {
+        s = launch_after_smem(k_flow<false>, grid, kFlowThreads, f.smem, false, st, fp, maps);
         if (s != STTM_OK) return s;
     }
     mark_stage(1, st);
@@ -658,13 +774,15 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     s = launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)frame_roots, frame_base, out_count, vid_off,
                      out_offsets);
     if (s != STTM_OK) return s;
-    if (g_budget_tmax != nullptr) return STTM_OK;      // first pass of the budget mode: only the node counts are needed
+    if (in.tmax != nullptr) return STTM_OK;            // first pass of the budget mode: only the node counts are needed
     s = launch_after(k_rows, (unsigned)(g.B * g.T), 256, st, g, (const int8_t*)fp.cover, (const int32_t*)fp.link,
                      (const int32_t*)frame_base, (const long long*)vid_off, row_at_root, row_anchor, out_pos,
                      (long long)p->out_capacity_rows, (int)p->pos, device_status);
     if (s != STTM_OK) return s;
+    s = launch_after(k_flow_chain, blocks_for(f.nitems, kChainWarps), kChainWarps * 32, st, fp);
+    if (s != STTM_OK) return s;
     mark_stage(2, st);
-    s = launch_after_smem(k_flow<true>, grid, kFlowThreads, f.smem, true, st, fp);
+    s = launch_after_smem(k_flow<true>, grid, kFlowThreads, f.smem, true, st, fp, maps);
     if (s != STTM_OK) return s;
     mark_stage(3, st);
     s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, f.nseg + 1,
@@ -694,7 +812,7 @@ sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacit
     // covers the most rows there can be, up to a few waves of blocks (most tokens merge: few rows,
     // and blocks without a row would only cost their launch)
     const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
-    const unsigned blocks = std::min<unsigned>(blocks_for(max_rows * kGatherParts, 8), kSmCount * 16);
+    const unsigned blocks = std::min<unsigned>(blocks_for(max_rows * kGatherParts, 8), sm_count() * 16);
     sttm_status s = launch_after(k_gather_rows<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
                                  (const int32_t*)(ws + pl.row_anchor), (const int32_t*)(ws + pl.row_head),
                                  (const OutT*)(ws + pl.staging), (OutT*)out, capacity);
@@ -785,7 +903,7 @@ bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
 // cudaGetSymbolAddress, asked once per device while that device is current.
 constexpr size_t kStaticScratchBytes = STTM_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-void* g_static_scratch_addr[64] = {};
+void* g_static_scratch_addr[kMaxDevices] = {};
 
 sttm_status static_scratch_address(void** out) {
     int dev = 0;
@@ -807,8 +925,9 @@ struct Cache {
     void* feats = nullptr; size_t feats_bytes = 0;
     void* out = nullptr; size_t out_bytes = 0;
     void* ints = nullptr; size_t ints_bytes = 0;   // pos, map, count, offsets, status
+    int32_t* merge_status = nullptr;               // status word of sttm_merge
 };
-Cache g_cache[64];
+Cache g_cache[kMaxDevices];
 
 sttm_status grow(void** ptr, size_t* have, size_t need) {
     if (*have >= need) return STTM_OK;
@@ -817,6 +936,10 @@ sttm_status grow(void** ptr, size_t* have, size_t need) {
     *have = need;
     return STTM_OK;
 }
+
+sttm_status merge_impl(const void* feats, const sttm_params* p, void* ws_, size_t ws_bytes, void* out_feats,
+                       int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
+                       int32_t* device_status, const Internal& in, void* stream);
 
 }  // namespace
 
@@ -831,8 +954,15 @@ const char* sttm_status_string(sttm_status s) {
         case STTM_ERR_CAPACITY: return "output capacity exceeded";
         case STTM_ERR_NOT_CONVERGED: return "root search did not converge";
         case STTM_ERR_CUDA: return "CUDA error";
+        case STTM_ERR_TIMEOUT: return "a wait inside a kernel ran out";
     }
     return "unknown";
+}
+
+sttm_status sttm_status_from_bits(int32_t bits) {
+    for (int code = STTM_ERR_ARG; code <= STTM_ERR_TIMEOUT; code++)
+        if (bits & (1 << code)) return (sttm_status)code;
+    return STTM_OK;
 }
 
 void sttm_default_params(sttm_params* p, int T, int H, int W, int D, float tau_s, float tau_t) {
@@ -904,7 +1034,7 @@ sttm_status sttm_spatial(const void* feats, const sttm_params* p, void* ws, size
     cudaStream_t st = (cudaStream_t)stream;
     g_launches = 0;
     STTM_CUDA_TRY(cudaMemsetAsync(frame_counts, 0, (size_t)pl.g.B * pl.g.T * 4, st));
-    return run_spatial(feats, p, pl, (char*)ws, cover_level, frame_counts, spatial_sims, st);
+    return run_spatial(feats, p, pl, (float*)((char*)ws + pl.norms), cover_level, frame_counts, spatial_sims, st);
 }
 
 sttm_status sttm_spatial_static(const void* feats, const sttm_params* p, int8_t* cover_level, int32_t* frame_counts,
@@ -916,9 +1046,7 @@ sttm_status sttm_spatial_static(const void* feats, const sttm_params* p, int8_t*
     if (!feats || !cover_level || !frame_counts) return STTM_ERR_ARG;
     if (misaligned(feats, 16)) return STTM_ERR_ARG;
     // the only scratch of the spatial stage: one squared norm per quadtree node
-    const int nodes_per_column = pl.g.L == 3 ? 21 : (pl.g.L == 2 ? 5 : 1);
-    const size_t need = (size_t)pl.g.B * pl.g.T * pl.g.ncol * nodes_per_column * sizeof(float);
-    if (need > kStaticScratchBytes) return STTM_ERR_WORKSPACE;
+    if (pl.norms_bytes > kStaticScratchBytes) return STTM_ERR_WORKSPACE;
     void* scratch = nullptr;
     if ((s = static_scratch_address(&scratch)) != STTM_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
@@ -926,7 +1054,7 @@ sttm_status sttm_spatial_static(const void* feats, const sttm_params* p, int8_t*
     // the counts are added to, so they start at zero; the norms are overwritten, nothing of an
     // earlier call is read
     STTM_CUDA_TRY(cudaMemsetAsync(frame_counts, 0, (size_t)pl.g.B * pl.g.T * 4, st));
-    return run_spatial(feats, p, pl, (char*)scratch - pl.norms, cover_level, frame_counts, spatial_sims, st);
+    return run_spatial(feats, p, pl, (float*)scratch, cover_level, frame_counts, spatial_sims, st);
 }
 
 sttm_status sttm_temporal(const void* feats, const sttm_params* p, void* ws, size_t ws_bytes,
@@ -947,8 +1075,20 @@ sttm_status sttm_temporal(const void* feats, const sttm_params* p, void* ws, siz
 sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, size_t ws_bytes, void* out_feats,
                           int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
                           int32_t* device_status, void* stream) {
+    return merge_impl(feats, p, ws_, ws_bytes, out_feats, out_pos, merge_map, out_count, out_offsets, device_status,
+                      Internal(), stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+// The whole path; `in` carries what the budget mode adds to its two passes.
+sttm_status merge_impl(const void* feats, const sttm_params* p, void* ws_, size_t ws_bytes, void* out_feats,
+                       int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
+                       int32_t* device_status, const Internal& in, void* stream) {
     Plan pl;
-    sttm_status s = make_plan(p, &pl);
+    sttm_status s = make_plan(p, &pl, in.budget);
     if (s != STTM_OK) return s;
     if (!feats || !ws_ || !out_feats || !out_pos || !out_count) return STTM_ERR_ARG;
     if (p->out_capacity_rows < 0) return STTM_ERR_ARG;
@@ -984,16 +1124,16 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
     }
     if (pl.fl.ok) {
         STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.ones_begin, 0xff, pl.ones_end - pl.ones_begin, st));
-        return run_flow(feats, p, pl, ws, out_feats, out_pos, merge_map, out_count, out_offsets, device_status, st);
+        return run_flow(feats, p, pl, ws, out_feats, out_pos, merge_map, out_count, out_offsets, device_status, in, st);
     }
     if (pl.f.ok) {
         // single-read path: fused kernel, roots, ordering, gather
         STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.ones_begin, 0xff, pl.ones_end - pl.ones_begin, st));
         mark_stage(0, st);
-        s = run_fused(feats, p, pl, ws, device_status, st);
+        s = run_fused(feats, p, pl, ws, device_status, in, st);
         if (s != STTM_OK) return s;
         mark_stage(1, st);
-        if (g_budget_tmax != nullptr) {
+        if (in.tmax != nullptr) {
             // first pass of the budget mode: only the node counts per video are needed
             return launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)(ws + pl.frame_counts),
                                 (int32_t*)(ws + pl.frame_base), out_count, (long long*)(ws + pl.vid_off), out_offsets);
@@ -1033,7 +1173,7 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
         return s;
     }
     mark_stage(0, st);
-    s = run_spatial(feats, p, pl, ws, cover, (int32_t*)(ws + pl.frame_counts), nullptr, st);
+    s = run_spatial(feats, p, pl, (float*)(ws + pl.norms), cover, (int32_t*)(ws + pl.frame_counts), nullptr, st);
     if (s != STTM_OK) return s;
     mark_stage(1, st);
     s = run_temporal(feats, p, pl, ws, cover, link, root, nullptr, device_status, st);
@@ -1073,6 +1213,10 @@ sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, si
     });
 }
 
+}  // namespace
+
+extern "C" {
+
 sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_s, float tau_t, void* out_feats,
                        int32_t* out_pos, int32_t* out_count, void* stream) {
     sttm_params p;
@@ -1082,21 +1226,36 @@ sttm_status sttm_merge(const void* feats, int T, int H, int W, int D, float tau_
         Plan pl;
         return make_plan(&p, &pl);
     }
-    int dev = 0;
-    STTM_CUDA_TRY(cudaGetDevice(&dev));
-    Cache& c = g_cache[dev % 64];
-    if (c.ws_bytes < need) {
+    const int dev = device_slot();
+    if (dev < 0) return STTM_ERR_UNSUPPORTED;
+    Cache& c = g_cache[dev];
+    if (c.ws_bytes < need || c.merge_status == nullptr) {
         STTM_CUDA_TRY(cudaDeviceSynchronize());
         sttm_status s = grow(&c.ws, &c.ws_bytes, need);
         if (s != STTM_OK) return s;
+        if (c.merge_status == nullptr) STTM_CUDA_TRY(cudaMalloc((void**)&c.merge_status, 256));
     }
-    return sttm_merge_ex(feats, &p, c.ws, c.ws_bytes, out_feats, out_pos, nullptr, out_count, nullptr, nullptr,
+    STTM_CUDA_TRY(cudaMemsetAsync(c.merge_status, 0, 4, (cudaStream_t)stream));
+    return sttm_merge_ex(feats, &p, c.ws, c.ws_bytes, out_feats, out_pos, nullptr, out_count, nullptr, c.merge_status,
                          stream);
+}
+
+sttm_status sttm_merge_status(int32_t* host_bits, void* stream) {
+    const int dev = device_slot();
+    if (dev < 0) return STTM_ERR_UNSUPPORTED;
+    Cache& c = g_cache[dev];
+    int32_t bits = 0;
+    if (c.merge_status != nullptr) {
+        STTM_CUDA_TRY(cudaMemcpyAsync(&bits, c.merge_status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+        STTM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    }
+    if (host_bits != nullptr) *host_bits = bits;
+    return sttm_status_from_bits(bits);
 }
 
 size_t sttm_budget_workspace_bytes(const sttm_params* p) {
     Plan pl;
-    if (make_plan(p, &pl) != STTM_OK || !(pl.f.ok || pl.fl.ok)) return 0;
+    if (make_plan(p, &pl, true) != STTM_OK || !(pl.f.ok || pl.fl.ok)) return 0;
     return (pl.total + 255) / 256 * 256 + ((size_t)pl.cells * 4 + 255) / 256 * 256 + 256;
 }
 
@@ -1105,7 +1264,7 @@ sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const lon
                               int32_t* out_count, int64_t* out_offsets, float* tau_t_out, int32_t* device_status,
                               void* stream) {
     Plan pl;
-    sttm_status s = make_plan(p, &pl);
+    sttm_status s = make_plan(p, &pl, true);
     if (s != STTM_OK) return s;
     if (!(pl.f.ok || pl.fl.ok)) return STTM_ERR_UNSUPPORTED;
     if (!budget_rows || !ws || !out_count) return STTM_ERR_ARG;
@@ -1121,11 +1280,11 @@ sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const lon
     sttm_params q = *p;
     q.tau_t = 2.f;
     q.tau_t_per_video = nullptr;
-    g_budget_tmax = tmax;
-    g_budget_tau_dev = nullptr;
-    s = sttm_merge_ex(feats, &q, ws, main_bytes, out_feats, out_pos, nullptr, out_count, out_offsets, device_status,
-                      stream);
-    g_budget_tmax = nullptr;
+    Internal first;
+    first.budget = true;
+    first.tmax = tmax;
+    s = merge_impl(feats, &q, ws, main_bytes, out_feats, out_pos, nullptr, out_count, out_offsets, device_status, first,
+                   stream);
     if (s != STTM_OK) return s;
     Budgets bd = {};
     for (int b = 0; b < p->B; b++) bd.rows[b] = budget_rows[b];
@@ -1133,12 +1292,12 @@ sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const lon
                      (const int32_t*)out_count, bd, tau_dev);
     if (s != STTM_OK) return s;
     // second pass: the whole path with the thresholds read from device memory
-    g_budget_tau_dev = tau_dev;
-    g_budget_second_pass = true;
-    s = sttm_merge_ex(feats, p, ws, main_bytes, out_feats, out_pos, merge_map, out_count, out_offsets, device_status,
-                      stream);
-    g_budget_tau_dev = nullptr;
-    g_budget_second_pass = false;
+    Internal second;
+    second.budget = true;
+    second.tau_dev = tau_dev;
+    second.second_pass = pl.fl.ok;      // the two-stream kernels keep the first pass's Gram stage
+    s = merge_impl(feats, p, ws, main_bytes, out_feats, out_pos, merge_map, out_count, out_offsets, device_status, second,
+                   stream);
     if (s != STTM_OK) return s;
     if (tau_t_out != nullptr)
         STTM_CUDA_TRY(cudaMemcpyAsync(tau_t_out, tau_dev, sizeof(float) * p->B, cudaMemcpyDeviceToDevice, st));
@@ -1291,6 +1450,7 @@ void sttm_release_cache(void) {
     cudaDeviceSynchronize();
     if (c.ws) cudaFree(c.ws);
     if (c.feats) cudaFree(c.feats);
+    if (c.merge_status) cudaFree(c.merge_status);
     if (c.out) cudaFree(c.out);
     if (c.ints) cudaFree(c.ints);
     c = Cache();

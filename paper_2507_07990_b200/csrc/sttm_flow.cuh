@@ -11,38 +11,48 @@
 //   decision stage adds the slices in a fixed order and takes the decisions, one half warp per
 //                 (tile, frame): cover level and link of every cell.
 //   ordering      row numbers of the surviving tokens (Section 3.4): integer scans.
+//   chain stage   one warp per (tile, run of frames) follows the chains through the run and
+//                 leaves one command record per frame: a 16 x 16 matrix W (chain slot x cell)
+//                 and the list of chains that ended, each with its final output row.
 //   sum stage     streams the features a second time (out of L2 where the two streams run close
 //                 together) and forms the chain averages of Section 3.3 as running sums
-//                 sums[16 chain slots x channels] += W X on the tensor cores, W the frame's
-//                 16 x 16 matrix of weights (chain slot x cell).  A chain that ends is divided by
-//                 its weight and written straight to its final output row, because the row
-//                 numbers exist before this stage starts.  Chains that cross the border between
-//                 two runs of frames leave fp32 pieces that a small kernel adds up.
-// A tile is the same 16-row unit as in the single-pass kernel (sttm_fused.cuh): a 4x4 block of
-// cells or several packed border parts; a task's frames pass through a shared-memory ring filled by
-// bulk asynchronous copies (one per cell row), consumed by eight worker warps.
+//                 sums[16 chain slots x channels] += W X on the tensor cores.  A chain that ends
+//                 is divided by its weight and written straight to its output row.  Chains that
+//                 cross the border between two runs of frames leave fp32 pieces that a small
+//                 kernel adds up.
+// A tile is 16 cells: a 4x4 block of the grid (clipped at the border), or, when the grid is one
+// cell wider (higher) than a multiple of four, 16 cells of its last column (row).  One tensor
+// copy (cp.async.bulk.tensor, 128-byte swizzle) brings a tile's frame and channel slice into a
+// shared-memory ring as [64-channel block][cell][64 channels]; rows outside the grid arrive as zeros.
 #pragma once
+
+#include <cuda.h>
 
 #include "sttm_fused.cuh"
 
 namespace sttm {
 
-constexpr int kFlowWorkers = 8;                      // Gram warps / sum warps
-constexpr int kFlowWarps = kFlowWorkers + 3;         // + chain warp, two producer warps
+constexpr int kFlowWorkers = 7;                      // Gram warps / sum warps (with the producer: 256 threads,
+                                                     // so that two CTAs on an SM leave 128 registers a thread)
+constexpr int kFlowWarps = kFlowWorkers + 1;         // + producer warp
 constexpr int kFlowThreads = kFlowWarps * 32;
-constexpr int kFlowMaxKs = 8;                        // 16-channel steps per Gram warp: slices of up to 1024 channels
+constexpr int kFlowMaxRing = 16;
+constexpr int kFlowMaxNB = 14;                       // 64-channel blocks per slice: two per sum warp
+constexpr int kFlowMaxKs = 8;                        // 16-channel steps per Gram warp
+constexpr int kBlkBytes = 2048;                      // 16 cells x 128 bytes
 constexpr int kFlowMaxF = 64;                        // frames per item, the frame before it not counted
-constexpr int kFlowMaxSlices = 16;
+constexpr int kRecBytes = (int)sizeof(FrameRec);
+
+struct TileBox { int kind, x0, y0, pad; };           // 0: 4x4 box at (x0, y0); 1: 16 cells down column x0; 2: 16 cells along row y0
 
 struct FlowParams {
-    const __nv_bfloat16* feats;
     int B, T, H, W, D, L;
     int HW, N;
     int ntiles;
-    int NS, S, NA;           // channel slices, channels per slice, sum warps in use (128 channels each)
-    int row_bytes, slot_bytes, R;
+    int NS, NB;              // channel slices, 64-channel blocks per slice
+    int slot_bytes, R;
     int F, nseg, nitems;     // frames per item, items per (video, tile), items
-    int weight_mode, out_f32, match_best, dry;
+    int weight_mode, out_f32, match_best;
     int8_t* cover;
     int32_t* link;
     int32_t* chain_key;      // [B*N] per cell: root cell id of its chain as far as the item knows it
@@ -51,6 +61,7 @@ struct FlowParams {
     const float* tau_t_dev;  // budget mode, may be null: [B] temporal thresholds in device memory
     float* partial;          // [nitems][F+1][NS][128]: the Gram stage's numbers, [number][cell]
     int32_t* hand;           // [nitems][F+1][16]: cover level | (link lane + 1) << 8 of every tile row
+    FrameRec* recs;          // [nitems][F+2]: the chain stage's records, one per frame and a closing one
     const int32_t* row_at_root;   // [B*N] row (inside its video) of every surviving token
     const long long* vid_off;     // [B+1] first row of every video
     void* out;               // [rows][D] output rows
@@ -59,12 +70,13 @@ struct FlowParams {
     int2* piece_meta;        // [nitems][kPieceSlots] {key cell id or -1, weight}
     int* status;
     TileDesc tiles[kMaxTiles];
+    TileBox boxes[kMaxTiles];
 };
+
+struct FlowMaps { CUtensorMap m[3]; };               // one per kind of TileBox
 
 struct FlowItem {
     int item, b, tile, tstart, n, halo, last_seg;
-    uint32_t vmask;
-    int nvalid;
 };
 
 // item = (video, run of frames, tile), tiles fastest: items of one run of frames are neighbours
@@ -80,19 +92,53 @@ __device__ __forceinline__ FlowItem flow_item(const FlowParams& p, int item) {
     it.tstart = t0 - it.halo;
     it.n = t1 - it.tstart;
     it.last_seg = t1 == p.T;
-    it.vmask = 0;
-    for (int l = 0; l < 16; l++)
-        if (p.tiles[it.tile].y[l] != 255) it.vmask |= 1u << l;
-    it.nvalid = __popc(it.vmask);
     return it;
 }
 
+// has the phase with this parity completed?  Suspends the thread for a while (the hardware's own
+// limit) instead of returning at once: a waiting warp of these kernels must not take issue slots
+// from the warps that have work.
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait (see mbar_wait) on the suspending form
+__device__ __forceinline__ bool mbar_wait_sleep(uint32_t bar, int use, bool& timed_out) {
+    if (timed_out) return false;
+    const uint32_t parity = (uint32_t)(use & 1);
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    while (!mbar_try(bar, parity)) {
+        if (global_timer_ns() - t0 > kWaitLimitNs) {
+            timed_out = true;
+            return false;
+        }
+    }
+    return true;
+}
 // bounded wait whose outcome is the same in every lane of the warp
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, int use, bool& timed_out) {
-    const bool ok = mbar_wait(bar, use, timed_out);
+    const bool ok = mbar_wait_sleep(bar, use, timed_out);
     const bool all = __all_sync(0xffffffffu, ok);
     if (!all) timed_out = true;
     return all;
+}
+
+// one tile of one frame, NB 64-channel blocks from block `blk0` on: global -> shared memory,
+// completion counted in bytes on an mbarrier
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int x, int y, int blk0, int frame,
+                                              uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(x), "r"(y), "r"(blk0), "r"(frame), "r"(bar)
+        : "memory");
 }
 
 // Section 3.2 for one frame, 16 lanes per frame (both halves of the warp at once, each on its own
@@ -223,104 +269,204 @@ k_flow_decide(const __grid_constant__ FlowParams p, const __grid_constant__ Taus
 }
 
 // ---------------------------------------------------------------------------------
-// The streaming kernel.  kSum == false: Gram stage; kSum == true: sum stage.  A task is (item,
-// channel slice); tasks are dealt to the CTAs round robin.  Warps: [0, 8) workers, 8 chain warp
-// (sum stage only), 9 and 10 producers.
+// Chain stage.  One warp per item follows the tile's chains through the item's frames: which
+// running sum (chain slot) every kept node joins, which chains ended and where they go.  Leaves
+// one record per frame and a closing record that writes out what still runs at the item's end.
 // ---------------------------------------------------------------------------------
-struct FlowSmem {
-    unsigned char* ring;
-    float* red;             // [8][512] the Gram warps' parts
-    float* redsum;          // [512]
-    float* wtab;            // [16] the lanes' weights w2 of the current item
-    FrameRec* recs;         // [kRecRing]
-    SlotTable* tab;
-    int* hand;              // [kFlowMaxF + 1][16]
-    int* rows;              // [kFlowMaxF + 1][16]
-    uint32_t full_bar, empty_bar, rfull_bar, rempty_bar;
-};
+constexpr int kChainWarps = 4;
 
-__host__ __device__ inline size_t flow_fixed_smem() {
-    return (size_t)kFlowWorkers * kGramVals * 4 + kGramVals * 4 + 128 + kRecRing * sizeof(FrameRec) + sizeof(SlotTable) +
-           2 * (kFlowMaxF + 1) * 16 * 4 + (2 * kMaxRing + 2 * kRecRing) * 8 + 128;
+__global__ void __launch_bounds__(kChainWarps * 32)
+k_flow_chain(const __grid_constant__ FlowParams p) {
+    wait_for_prior_kernel();
+    __shared__ __align__(16) FrameRec s_rec[kChainWarps];
+    __shared__ SlotTable s_tab[kChainWarps];
+    const unsigned full = 0xffffffffu;
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31, c = lane & 15;
+    const bool low = lane < 16;
+    const int item = blockIdx.x * kChainWarps + wib;
+    if (item >= p.nitems) return;
+    const FlowItem it = flow_item(p, item);
+    FrameRec* rec = &s_rec[wib];
+    SlotTable* tab = &s_tab[wib];
+    const LaneGeo lg = lane_geo(p.tiles[it.tile], c, p.L, p.W);
+    const bool valid = lg.valid;
+    const float w1 = lg.w1, w2 = lg.w2;
+    const long long vrow0 = p.vid_off[it.b];
+    p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
+    FrameRec* dst = p.recs + (long long)it.item * (p.F + 2);
+    const int32_t* hand = p.hand + (long long)it.item * (p.F + 1) * 16;
+    int prev_slot = 0;
+    uint32_t active_slots = 0;
+    // (the next frame's decisions and row numbers are fetched while this frame is worked on)
+    int packed_next = hand[c];
+    int row_next = valid ? p.row_at_root[(long long)it.b * p.N + (long long)it.tstart * p.HW + lg.cell] : -1;
+    for (int j = 0; j <= it.n; j++) {
+        const int packed = packed_next, my_row = row_next;
+        if (j + 1 < it.n) {
+            packed_next = hand[(j + 1) * 16 + c];
+            row_next = valid ? p.row_at_root[(long long)it.b * p.N + (long long)(it.tstart + j + 1) * p.HW + lg.cell] : -1;
+        }
+        if (j == it.n) {
+            // closing record: everything still running is written out
+            if (low && ((active_slots >> lane) & 1u)) {
+                if (!tab->virt[lane] && it.last_seg) {
+                    const long long grow = vrow0 + tab->row[lane];
+                    rec->flush[lane] = FlushCmd{lane, 0, grow < p.capacity ? (int)grow : -1, (float)tab->weight[lane]};
+                } else {
+                    const int pc = it.item * kPieceSlots + 16 + lane;
+                    rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
+                    p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
+                }
+            }
+            if (lane == 0) rec->flush_mask = active_slots;
+        } else {
+            const int lv = packed & 3, link_local = (packed >> 8) - 1;
+            const int t = it.tstart + j;
+            const bool is_halo = it.halo && j == 0;
+            // nodes with a link join the chain of their target; chains without a member in this
+            // frame have ended; the remaining nodes start new chains in free slots
+            const bool anchor = valid && lane_anchor(lg, c, lv) == c;
+            const bool linked = anchor && link_local >= 0;
+            const bool fresh = anchor && link_local < 0;
+            const int slot_linked = __shfl_sync(full, prev_slot, link_local < 0 ? 0 : link_local);
+            const uint32_t memb = __reduce_or_sync(full, linked ? 1u << slot_linked : 0u);
+            const uint32_t dead = active_slots & ~memb;
+            const uint32_t freem = ~memb & 0xffffu;
+            const uint32_t freshm = __ballot_sync(full, fresh && low);
+            const int slot_fresh = kth_set_bit16(freem, __popc(freshm & ((1u << c) - 1)));
+            const int node_slot = linked ? slot_linked : slot_fresh;
+            const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + lane_anchor(lg, c, lv));
+            const uint32_t cells = lane_region(lg, c, lv);
+            const int wint = p.weight_mode ? __popc(cells) : 1;
+            const long long gc = (long long)it.b * p.N + (long long)t * p.HW + lg.cell;
+            // chains that ended: lane s looks at slot s (before the slot is given away again)
+            if (low && ((dead >> lane) & 1u)) {
+                if (tab->virt[lane]) {
+                    const int pc = it.item * kPieceSlots + tab->cell[lane];
+                    rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
+                    p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
+                } else {
+                    const long long grow = vrow0 + tab->row[lane];
+                    rec->flush[lane] = FlushCmd{lane, 0, grow < p.capacity ? (int)grow : -1, (float)tab->weight[lane]};
+                }
+            }
+            __syncwarp();
+            if (low && fresh) {
+                tab->key[slot_fresh] = (int)gc;
+                tab->weight[slot_fresh] = is_halo ? 0 : wint;
+                tab->virt[slot_fresh] = is_halo ? 1 : 0;
+                tab->cell[slot_fresh] = c;
+                tab->row[slot_fresh] = my_row;
+            }
+            __syncwarp();
+            if (low && linked) atomicAdd(&tab->weight[slot_linked], wint);
+            // the frame's weight matrix: row = chain slot, column = cell
+            reinterpret_cast<uint4*>(rec->wmat)[lane] = make_uint4(0u, 0u, 0u, 0u);
+            const int wnode = __shfl_sync(full, wint, (lane & 16) + lane_anchor(lg, c, lv));
+            __syncwarp();
+            if (low && valid && !is_halo) {
+                const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
+                rec->wmat[cur_slot * 16 + c] = __bfloat16_as_ushort(__float2bfloat16_rn(wc));
+            }
+            if (lane == 0) rec->flush_mask = dead;
+            if (!is_halo && low && valid) p.chain_key[gc] = tab->key[cur_slot] - it.b * p.N;
+            active_slots = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
+            prev_slot = cur_slot;
+        }
+        __syncwarp();
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(rec);
+            uint4* d4 = reinterpret_cast<uint4*>(dst + j);
+            for (int i = lane; i < kRecBytes / 16; i += 32) d4[i] = src[i];
+        }
+        __syncwarp();
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// The streaming kernel.  kSum == false: Gram stage; kSum == true: sum stage.  A task is (item,
+// channel slice); tasks are dealt to the CTAs round robin.  Warps: [0, 7) workers, 7 producer.
+// Two CTAs share an SM: each runs its frames through its phases in step, and the two fill each
+// other's gaps.
+//   Gram stage: the seven workers share the slice's 16-channel steps and keep a frame's fragments
+//   in registers for the next frame's cross products (a ring slot is free again as soon as it has
+//   been read); their parts of G and C meet in shared memory between two named barriers, are added
+//   in warp order and contracted to the 128 numbers.
+//   Sum stage: warp a owns the slice's 64-channel blocks 2a and 2a + 1.
+// Shared memory: ring of R slots (1024-byte aligned), R records, the Gram warps' parts, barriers.
+// ---------------------------------------------------------------------------------
+__host__ __device__ inline size_t flow_fixed_smem(int R) {
+    return (size_t)R * kRecBytes + (size_t)kFlowWorkers * kGramVals * 4 + kGramVals * 4 + 128 + 2 * kFlowMaxRing * 8 + 1024;
 }
 
 template <bool kSum>
-__global__ void __launch_bounds__(kFlowThreads, 1)
-k_flow(const __grid_constant__ FlowParams p) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    FlowSmem sm;
-    size_t off = 0;
-    sm.ring = smem;                                                off += (size_t)p.R * p.slot_bytes;
-    sm.red = reinterpret_cast<float*>(smem + off);                 off += (size_t)kFlowWorkers * kGramVals * 4;
-    sm.redsum = reinterpret_cast<float*>(smem + off);              off += kGramVals * 4;
-    sm.wtab = reinterpret_cast<float*>(smem + off);                off += 128;
-    sm.recs = reinterpret_cast<FrameRec*>(smem + off);             off += kRecRing * sizeof(FrameRec);
-    sm.tab = reinterpret_cast<SlotTable*>(smem + off);             off += sizeof(SlotTable);
-    sm.hand = reinterpret_cast<int*>(smem + off);                  off += (kFlowMaxF + 1) * 16 * 4;
-    sm.rows = reinterpret_cast<int*>(smem + off);                  off += (kFlowMaxF + 1) * 16 * 4;
-    off = (off + 7) & ~(size_t)7;
+__global__ void __launch_bounds__(kFlowThreads, 2)
+k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps maps) {
+    extern __shared__ unsigned char smem_raw[];
+    // the swizzle pattern of the tensor copies is a function of the shared-memory address
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    unsigned char* ring = smem;
+    size_t off = (size_t)p.R * p.slot_bytes;
+    unsigned char* recs = smem + off;                              off += (size_t)p.R * kRecBytes;
+    float* red = reinterpret_cast<float*>(smem + off);             off += (size_t)kFlowWorkers * kGramVals * 4;
+    float* redsum = reinterpret_cast<float*>(smem + off);          off += kGramVals * 4;
+    float* wtab = reinterpret_cast<float*>(smem + off);            off += 128;
     const uint32_t bar0 = smem_u32(smem + off);
-    sm.full_bar = bar0;
-    sm.empty_bar = bar0 + 8 * kMaxRing;
-    sm.rfull_bar = bar0 + 16 * kMaxRing;
-    sm.rempty_bar = sm.rfull_bar + 8 * kRecRing;
+    const uint32_t full_bar = bar0, empty_bar = bar0 + 8 * kFlowMaxRing;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t ring_base = smem_u32(sm.ring);
+    const uint32_t ring_base = smem_u32(ring), recs_base = smem_u32(recs);
     const int ntasks = p.nitems * p.NS;
+    const int nsum = (p.NB + 1) / 2;                    // sum warps at work
 
     if (tid == 0) {
         for (int s = 0; s < p.R; s++) {
-            mbar_init(sm.full_bar + 8 * s, 1);
-            mbar_init(sm.empty_bar + 8 * s, kFlowWorkers);
-        }
-        for (int s = 0; s < kRecRing; s++) {
-            mbar_init(sm.rfull_bar + 8 * s, 1);
-            mbar_init(sm.rempty_bar + 8 * s, p.NA);
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, kSum ? nsum : kFlowWorkers);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // a ring without NaN patterns: rows of a tile that hold no cell are never written
-    for (int k = tid * 16; k < p.R * p.slot_bytes; k += blockDim.x * 16)
-        *reinterpret_cast<uint4*>(sm.ring + k) = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     if constexpr (kSum) wait_for_prior_kernel();
 
     bool timed_out = false;
-    int s = 0, use = 0;             // ring slot of the next frame and how often it has been filled before
+    int q = 0;                      // slots used so far by this CTA's tasks: slot q % R, filled q / R times before
 
     if (warp < kFlowWorkers && !kSum) {
         // ------------------------------------ Gram warps ------------------------------------
-        // Warp w owns the 16-channel steps [k0, k1) of the slice.  The fragments of a frame are
-        // loaded once and kept for the next frame's cross products, so a ring slot is free again
-        // as soon as it has been read.
-        const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lk = (lane >> 4) * 8;
-        const uint32_t loff = lrow * p.row_bytes + lk * 2;
-        const int ksteps = p.S >> 4;
+        const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int ksteps = p.NB * 4;
         const int k0 = ksteps * warp / kFlowWorkers, nk = ksteps * (warp + 1) / kFlowWorkers - k0;
-        const int wtid = tid;                           // 0..255 among the workers
-        const uint32_t red_a = smem_u32(sm.red), redsum_a = smem_u32(sm.redsum), W2s = smem_u32(sm.wtab);
+        uint32_t koff[kFlowMaxKs];          // where this lane's rows of the warp's 16-channel steps sit in a slot
+#pragma unroll
+        for (int i = 0; i < kFlowMaxKs; i++) {
+            const uint32_t kk = (uint32_t)(k0 + i);
+            koff[i] = (kk >> 2) * kBlkBytes + lrow * 128 + ((((kk & 3) * 2 + (lane >> 4)) ^ (lrow & 7)) << 4);
+        }
+        const int nthr = kFlowWorkers * 32;
+        const uint32_t redsum_a = smem_u32(redsum), W2s = smem_u32(wtab);
         for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
             const FlowItem it = flow_item(p, task / p.NS);
             const int slice = task % p.NS;
-            const LaneGeo lg = lane_geo(p.tiles[it.tile], wtid & 15, p.L, p.W);
-            named_sync(1, kFlowWorkers * 32);           // the previous task's weights are not read any more
-            if (wtid < 16) sm.wtab[wtid] = lg.w2;
+            const LaneGeo lg = lane_geo(p.tiles[it.tile], tid & 15, p.L, p.W);
+            named_sync(1, nthr);                       // the previous task's weights are not read any more
+            if (tid < 16) wtab[tid] = lg.w2;
+            float* dst = p.partial + ((long long)it.item * (p.F + 1) * p.NS + slice) * kSumVals;
             uint32_t prv[kFlowMaxKs][4];
 #pragma unroll
             for (int i = 0; i < kFlowMaxKs; i++) prv[i][0] = prv[i][1] = prv[i][2] = prv[i][3] = 0u;
-            float* dst = p.partial + ((long long)it.item * (p.F + 1) * p.NS + slice) * kSumVals;
-            for (int j = 0; j < it.n; j++) {
-                mbar_wait_warp(sm.full_bar + 8 * s, use, timed_out);
+            for (int j = 0; j < it.n; j++, q++) {
+                const int s = q % p.R;
+                mbar_wait_warp(full_bar + 8 * s, q / p.R, timed_out);
                 uint32_t cur[kFlowMaxKs][4];
-                const uint32_t base = ring_base + s * p.slot_bytes + loff + k0 * 32;
+                const uint32_t base = ring_base + s * p.slot_bytes;
 #pragma unroll
                 for (int i = 0; i < kFlowMaxKs; i++) {
-                    if (i < nk) ldmatrix_x4(base + i * 32, cur[i]);
+                    if (i < nk) ldmatrix_x4(base + koff[i], cur[i]);
                     else cur[i][0] = cur[i][1] = cur[i][2] = cur[i][3] = 0u;
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(sm.empty_bar + 8 * s);
+                if (lane == 0) mbar_arrive(empty_bar + 8 * s);
                 float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
                 float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -333,7 +479,7 @@ k_flow(const __grid_constant__ FlowParams p) {
                     }
                 }
                 {
-                    float* r = sm.red + warp * kGramVals;
+                    float* r = red + warp * kGramVals;
                     const int gr = lane >> 2, gc = (lane & 3) * 2;
                     *reinterpret_cast<float2*>(r + gr * 16 + gc) = make_float2(g0[0], g0[1]);
                     *reinterpret_cast<float2*>(r + (gr + 8) * 16 + gc) = make_float2(g0[2], g0[3]);
@@ -345,73 +491,67 @@ k_flow(const __grid_constant__ FlowParams p) {
                     *reinterpret_cast<float2*>(r + 256 + (gr + 8) * 16 + 8 + gc) = make_float2(c1[2], c1[3]);
                 }
                 // (the barrier also spreads a wait that ran out: every worker leaves together)
-                if (named_sync_or(2, kFlowWorkers * 32, timed_out)) { timed_out = true; break; }
-                {
-                    // add the warps' parts in warp order, two entries per thread
-                    float2 sum = *reinterpret_cast<const float2*>(sm.red + wtid * 2);
+                if (named_sync_or(2, nthr, timed_out)) { timed_out = true; break; }
+                for (int e = tid * 2; e < kGramVals; e += nthr * 2) {
+                    // add the warps' parts in warp order, two entries at a time
+                    float2 sum = *reinterpret_cast<const float2*>(red + e);
 #pragma unroll
                     for (int w = 1; w < kFlowWorkers; w++) {
-                        const float2 x = *reinterpret_cast<const float2*>(sm.red + w * kGramVals + wtid * 2);
+                        const float2 x = *reinterpret_cast<const float2*>(red + w * kGramVals + e);
                         sum.x += x.x; sum.y += x.y;
                     }
-                    *reinterpret_cast<float2*>(sm.redsum + wtid * 2) = sum;
+                    *reinterpret_cast<float2*>(redsum + e) = sum;
                 }
-                named_sync(1, kFlowWorkers * 32);
+                named_sync(1, nthr);
                 // contract to 8 numbers per cell: thread = (number, cell), stored [number][cell]
-                if (wtid < kSumVals) dst[(long long)j * p.NS * kSumVals + wtid] = combine_sums(redsum_a, wtid & 15, wtid >> 4, lg, W2s);
+                if (tid < kSumVals) dst[(long long)j * p.NS * kSumVals + tid] = combine_sums(redsum_a, tid & 15, tid >> 4, lg, W2s);
 #pragma unroll
                 for (int i = 0; i < kFlowMaxKs; i++) {
                     prv[i][0] = cur[i][0]; prv[i][1] = cur[i][1]; prv[i][2] = cur[i][2]; prv[i][3] = cur[i][3];
                 }
-                if (++s == p.R) { s = 0; use++; }
             }
         }
     } else if (warp < kFlowWorkers && kSum) {
         // ------------------------------------ sum warps ------------------------------------
-        // Warp a owns channels [128 a, 128 a + 128) of the slice: 16 tiles of 8 channels.  sums[nt][0..3]
-        // is the accumulator fragment of tile nt: chain slots g and g + 8 (g = lane / 4), channels
-        // 2 t and 2 t + 1 of the tile (t = lane % 4).
-        const bool active = warp < p.NA;
-        float sums[16][4];
+        // Warp a owns the slice's 64-channel blocks 2a and 2a + 1: 16 tiles of 8 channels.  sums[nt][0..3]
+        // is the accumulator fragment of tile nt: chain slots g and g + 8 (g = lane / 4), channels 2 t
+        // and 2 t + 1 of the tile (t = lane % 4).
+        if (warp < nsum) {
+            float sums[16][4];
 #pragma unroll
-        for (int nt = 0; nt < 16; nt++)
+            for (int nt = 0; nt < 16; nt++)
 #pragma unroll
-            for (int k = 0; k < 4; k++) sums[nt][k] = 0.f;
-        const int ch0 = warp * 128;
-        const int g = lane >> 2, t4 = lane & 3;
-        const uint32_t recs_a = smem_u32(sm.recs);
-        const uint32_t xoff = ((lane & 7) + ((lane >> 3) & 1) * 8) * p.row_bytes + (ch0 + (lane >> 4) * 8) * 2;
-        const uint32_t woff = 16 + 256 + ((lane & 7) + ((lane >> 3) & 1) * 8) * 32 + (lane >> 4) * 16;
-        const int ntmax = min(16, (p.S - ch0) >> 3);        // 8-channel tiles of this warp inside the slice
-        int rq = 0;                                         // records so far
-        for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
-            const FlowItem it = flow_item(p, task / p.NS);
-            const int slice = task % p.NS;
-            const long long chan = (long long)slice * p.S + ch0 + 2 * t4;
-            // one record per frame, and a last one that writes out what the item leaves
-            for (int j = 0; j <= it.n; j++) {
-                const bool frame = j < it.n;
-                if (frame && !mbar_wait_warp(sm.full_bar + 8 * s, use, timed_out)) break;
-                if (!active) {
-                    if (frame) {
-                        if (lane == 0) mbar_arrive(sm.empty_bar + 8 * s);
-                        if (++s == p.R) { s = 0; use++; }
-                    }
-                    continue;
-                }
-                const int rk = rq % kRecRing;
-                if (!mbar_wait_warp(sm.rfull_bar + 8 * rk, rq / kRecRing, timed_out)) break;
-                const uint32_t rec = recs_a + rk * (uint32_t)sizeof(FrameRec);
-                const uint32_t flush_mask = lds_u32x4(rec).x;
+                for (int k = 0; k < 4; k++) sums[nt][k] = 0.f;
+            const int g = lane >> 2, t4 = lane & 3;
+            const uint32_t lrow = (lane & 7) + ((lane >> 3) & 1) * 8;
+            uint32_t xoff[4];
+#pragma unroll
+            for (int pr = 0; pr < 4; pr++)
+                xoff[pr] = 2 * warp * kBlkBytes + lrow * 128 + ((((uint32_t)pr * 2 + (lane >> 4)) ^ (lrow & 7)) << 4);
+            const uint32_t woff = 16 + 256 + lrow * 32 + (lane >> 4) * 16;
+            const int ntmax = 2 * warp + 1 < p.NB ? 16 : 8;     // an odd block count leaves the last warp one block
+            for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
+                const FlowItem it = flow_item(p, task / p.NS);
+                const int slice = task % p.NS;
+                const long long chan0 = ((long long)slice * p.NB + 2 * warp) * 64;
+                // one record per frame, and a closing one that writes out what the item leaves
+                for (int j = 0; j <= it.n; j++, q++) {
+                    const bool frame = j < it.n;
+                    const int s = q % p.R;
+                    if (!mbar_wait_warp(full_bar + 8 * s, q / p.R, timed_out)) break;
+                    const uint32_t rec = recs_base + s * kRecBytes;
+                    const uint32_t flush_mask = lds_u32x4(rec).x;
 #pragma unroll 1
-                for (int hi = 0; hi < 2; hi++) {
-                    const uint32_t m8 = (flush_mask >> (8 * hi)) & 0xffu;
-                    if (m8 == 0) continue;
-                    const bool mine = (m8 >> g) & 1u;
-                    const uint4 fc = lds_u32x4(rec + 16 + (g + 8 * hi) * 16);       // slot, kind, dst, weight
-                    const float inv = mine && fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
-                    const long long row = (long long)(int)fc.z * p.D + chan;
-                    const bool skip = (int)fc.z < 0;                                // a row beyond the capacity
+                    for (int hi = 0; hi < 2; hi++) {
+                        const uint32_t m8 = (flush_mask >> (8 * hi)) & 0xffu;
+                        if (m8 == 0) continue;
+                        // chains that ended: slot g + 8 hi is held by the four lanes of group g, which
+                        // scale its 128 channels and write them to the chain's row (or piece)
+                        const bool mine = (m8 >> g) & 1u;
+                        const uint4 fc = lds_u32x4(rec + 16 + (g + 8 * hi) * 16);       // slot, kind, dst, weight
+                        const float inv = mine && fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
+                        const long long row = (long long)(int)fc.z * p.D + chan0 + 2 * t4;
+                        const bool skip = (int)fc.z < 0;                                // a row beyond the capacity
 #define STTM_FLOW_FLUSH(I0, I1)                                                                               \
     if (fc.y != 0 || p.out_f32) {                                                                             \
         float* dst = (fc.y != 0 ? p.pieces : reinterpret_cast<float*>(p.out)) + row;                          \
@@ -430,172 +570,60 @@ k_flow(const __grid_constant__ FlowParams p) {
             if (nt < ntmax && !skip) *reinterpret_cast<uint32_t*>(dst + nt * 8) = w;                          \
         }                                                                                                     \
     }
-                    if (mine) {
-                        if (hi) { STTM_FLOW_FLUSH(2, 3) } else { STTM_FLOW_FLUSH(0, 1) }
-                    }
+                        if (mine) {
+                            if (hi) { STTM_FLOW_FLUSH(2, 3) } else { STTM_FLOW_FLUSH(0, 1) }
+                        }
 #undef STTM_FLOW_FLUSH
-                }
-                __syncwarp();
-                if (frame) {
-                    uint32_t wa[4];
-                    ldmatrix_x4(rec + woff, wa);
-                    const uint32_t xb = ring_base + s * p.slot_bytes + xoff;
+                    }
+                    __syncwarp();
+                    if (frame) {
+                        uint32_t wa[4];
+                        ldmatrix_x4(rec + woff, wa);
+                        const uint32_t xb = ring_base + s * p.slot_bytes;
 #pragma unroll
-                    for (int pr = 0; pr < 8; pr++) {
-                        if (ch0 + pr * 16 < p.S) {
-                            uint32_t xb4[4];
-                            ldmatrix_x4_trans(xb + pr * 32, xb4);
-                            mma_bf16(sums[2 * pr], wa, xb4[0], xb4[1]);
-                            mma_bf16(sums[2 * pr + 1], wa, xb4[2], xb4[3]);
+                        for (int pr = 0; pr < 8; pr++) {
+                            if (pr * 2 < ntmax) {
+                                uint32_t xb4[4];
+                                ldmatrix_x4_trans(xb + xoff[pr & 3] + (pr >> 2) * kBlkBytes, xb4);
+                                mma_bf16(sums[2 * pr], wa, xb4[0], xb4[1]);
+                                mma_bf16(sums[2 * pr + 1], wa, xb4[2], xb4[3]);
+                            }
                         }
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_bar + 8 * s);
                 }
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(sm.rempty_bar + 8 * rk);
-                    if (frame) mbar_arrive(sm.empty_bar + 8 * s);
-                }
-                rq++;
-                if (frame && ++s == p.R) { s = 0; use++; }
             }
         }
     } else if (warp == kFlowWorkers) {
-        // ------------------------------------ chain warp ------------------------------------
-        // Follows the tile's chains through the item's frames: which running sum (chain slot)
-        // every kept node joins, which chains ended and where they go.
-        if constexpr (kSum) {
-            const unsigned full = 0xffffffffu;
-            const int c = lane & 15;
-            const bool low = lane < 16;
-            int rq = 0;
-            for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
-                const FlowItem it = flow_item(p, task / p.NS);
-                const int slice = task % p.NS;
-                const bool writer = slice == 0;             // the integer outputs are written once per item
-                const LaneGeo lg = lane_geo(p.tiles[it.tile], c, p.L, p.W);
-                const bool valid = lg.valid;
-                const float w1 = lg.w1, w2 = lg.w2;
-                const long long vrow0 = p.vid_off[it.b];
-                // the item's decisions and the rows of the tokens that start in it
-                for (int i = lane; i < it.n * 16; i += 32) {
-                    const LaneGeo li = lane_geo(p.tiles[it.tile], i & 15, p.L, p.W);
-                    sm.hand[i] = p.hand[(long long)it.item * (p.F + 1) * 16 + i];
-                    sm.rows[i] = li.valid ? p.row_at_root[(long long)it.b * p.N + (long long)(it.tstart + (i >> 4)) * p.HW + li.cell] : -1;
-                }
-                if (writer) p.piece_meta[(long long)it.item * kPieceSlots + lane] = make_int2(-1, 0);
-                __syncwarp();
-                int prev_slot = 0;
-                uint32_t active_slots = 0;
-                for (int j = 0; j <= it.n; j++, rq++) {
-                    const int hb = rq % kRecRing;
-                    if (rq >= kRecRing && !mbar_wait_warp(sm.rempty_bar + 8 * hb, rq / kRecRing - 1, timed_out)) break;
-                    FrameRec* rec = sm.recs + hb;
-                    if (j == it.n) {
-                        // last record of the item: everything still running is written out
-                        if (low && ((active_slots >> lane) & 1u)) {
-                            if (!sm.tab->virt[lane] && it.last_seg) {
-                                const int row = sm.tab->row[lane];
-                                const long long grow = vrow0 + row;
-                                rec->flush[lane] = FlushCmd{lane, 0, grow < p.capacity ? (int)grow : -1, (float)sm.tab->weight[lane]};
-                            } else {
-                                const int pc = it.item * kPieceSlots + 16 + lane;
-                                rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
-                                if (writer) p.piece_meta[pc] = make_int2(sm.tab->key[lane], sm.tab->weight[lane]);
-                            }
-                        }
-                        if (lane == 0) rec->flush_mask = p.dry ? 0u : active_slots;
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(sm.rfull_bar + 8 * hb);
-                        continue;
-                    }
-                    const int packed = sm.hand[j * 16 + c];
-                    const int lv = packed & 3, link_local = (packed >> 8) - 1;
-                    const int t = it.tstart + j;
-                    const bool is_halo = it.halo && j == 0;
-
-                    // nodes with a link join the chain of their target; chains without a member in this
-                    // frame have ended; the remaining nodes start new chains in free slots
-                    const bool anchor = valid && lane_anchor(lg, c, lv) == c;
-                    const bool linked = anchor && link_local >= 0;
-                    const bool fresh = anchor && link_local < 0;
-                    const int slot_linked = __shfl_sync(full, prev_slot, link_local < 0 ? 0 : link_local);
-                    const uint32_t memb = __reduce_or_sync(full, linked ? 1u << slot_linked : 0u);
-                    const uint32_t dead = active_slots & ~memb;
-                    const uint32_t freem = ~memb & 0xffffu;
-                    const uint32_t freshm = __ballot_sync(full, fresh && low);
-                    const int slot_fresh = kth_set_bit16(freem, __popc(freshm & ((1u << c) - 1)));
-                    const int node_slot = linked ? slot_linked : slot_fresh;
-                    const int cur_slot = __shfl_sync(full, node_slot, (lane & 16) + lane_anchor(lg, c, lv));
-                    const uint32_t cells = lane_region(lg, c, lv);
-                    const int wint = p.weight_mode ? __popc(cells) : 1;
-                    const long long gc = (long long)it.b * p.N + (long long)t * p.HW + lg.cell;
-
-                    // chains that ended: lane s looks at slot s (before the slot is given away again)
-                    if (low && ((dead >> lane) & 1u)) {
-                        if (sm.tab->virt[lane]) {
-                            const int pc = it.item * kPieceSlots + sm.tab->cell[lane];
-                            rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
-                            if (writer) p.piece_meta[pc] = make_int2(sm.tab->key[lane], sm.tab->weight[lane]);
-                        } else {
-                            const long long grow = vrow0 + sm.tab->row[lane];
-                            rec->flush[lane] = FlushCmd{lane, 0, grow < p.capacity ? (int)grow : -1, (float)sm.tab->weight[lane]};
-                        }
-                    }
-                    __syncwarp();
-                    if (low && fresh) {
-                        sm.tab->key[slot_fresh] = (int)gc;
-                        sm.tab->weight[slot_fresh] = is_halo ? 0 : wint;
-                        sm.tab->virt[slot_fresh] = is_halo ? 1 : 0;
-                        sm.tab->cell[slot_fresh] = c;
-                        sm.tab->row[slot_fresh] = sm.rows[j * 16 + c];
-                    }
-                    if (low && linked) atomicAdd(&sm.tab->weight[slot_linked], wint);
-                    // the frame's weight matrix: row = chain slot, column = cell
-                    reinterpret_cast<uint4*>(rec->wmat)[lane] = make_uint4(0u, 0u, 0u, 0u);
-                    const int wnode = __shfl_sync(full, wint, (lane & 16) + lane_anchor(lg, c, lv));
-                    __syncwarp();
-                    if (low && valid && !is_halo) {
-                        const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
-                        rec->wmat[cur_slot * 16 + c] = __bfloat16_as_ushort(__float2bfloat16_rn(wc));
-                    }
-                    if (lane == 0) rec->flush_mask = p.dry ? 0u : dead;
-                    const uint32_t active = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(sm.rfull_bar + 8 * hb);
-
-                    if (writer && !is_halo && low && valid) p.chain_key[gc] = sm.tab->key[cur_slot] - it.b * p.N;
-                    active_slots = active;
-                    prev_slot = cur_slot;
-                    __syncwarp();
-                }
-            }
-        }
-    } else {
-        // ---------------------------------- producer warps ----------------------------------
-        const int which = warp - (kFlowWorkers + 1);
-        const int row = lane * 2 + which;                   // the tile row this lane copies
+        // ------------------------------------- producer -------------------------------------
+        // One tensor copy per frame (and, in the sum stage, one plain bulk copy of the frame's
+        // record), all on the slot's barrier.
         for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
             const FlowItem it = flow_item(p, task / p.NS);
             const int slice = task % p.NS;
-            for (int j = 0; j < it.n; j++) {
-                const uint32_t bar = sm.full_bar + 8 * s;
-                if (use >= 1 && !mbar_wait_warp(sm.empty_bar + 8 * s, use - 1, timed_out)) break;
-                if (lane == 0 && which == 0) mbar_expect_tx(bar, (uint32_t)(it.nvalid * p.S * 2));
-                __syncwarp();
-                if (row < 16 && ((it.vmask >> row) & 1u)) {
-                    const long long cell = ((long long)it.b * p.T + it.tstart + j) * p.HW +
-                                           p.tiles[it.tile].y[row] * p.W + p.tiles[it.tile].x[row];
-                    bulk_g2s(ring_base + s * p.slot_bytes + row * p.row_bytes, p.feats + cell * p.D + (long long)slice * p.S,
-                             (uint32_t)(p.S * 2), bar);
+            const TileBox bx = p.boxes[it.tile];
+            const int nslots = it.n + (kSum ? 1 : 0);
+            for (int j = 0; j < nslots; j++, q++) {
+                const int s = q % p.R;
+                const uint32_t bar = full_bar + 8 * s;
+                if (q >= p.R && !mbar_wait_warp(empty_bar + 8 * s, q / p.R - 1, timed_out)) break;
+                if (lane == 0) {
+                    const bool frame = j < it.n;
+                    mbar_expect_tx(bar, (uint32_t)((frame ? p.slot_bytes : 0) + (kSum ? kRecBytes : 0)));
+                    if (frame)
+                        tma_load_tile(ring_base + s * p.slot_bytes, &maps.m[bx.kind], bx.x0, bx.y0, slice * p.NB,
+                                      it.b * p.T + it.tstart + j, bar);
+                    if (kSum)
+                        bulk_g2s(recs_base + s * kRecBytes, p.recs + (long long)it.item * (p.F + 2) + j, kRecBytes, bar);
                 }
-                if (++s == p.R) { s = 0; use++; }
+                __syncwarp();
             }
         }
-        // the CTA must not end with copies in flight: the last R frames issued have landed?
-        const int q = use * p.R + s;
+        // the CTA must not end with copies in flight: the last R slots issued have landed?
         for (int qq = max(0, q - p.R); qq < q; qq++) {
             bool late = false;
-            mbar_wait(sm.full_bar + 8 * (qq % p.R), qq / p.R, late);
+            mbar_wait_sleep(full_bar + 8 * (qq % p.R), qq / p.R, late);
             timed_out |= late;
         }
     }

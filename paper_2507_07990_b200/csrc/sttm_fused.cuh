@@ -57,7 +57,7 @@ constexpr int kTailWarps = 4;           // similarity, chain, two producers
 constexpr int kFusedMaxThreads = (kMaxGramWarps + kCombineWarps + kMaxSumWarps + kTailWarps) * 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after two seconds
 
-enum : int { kStatusWaitTimeout = 1 << 6 };
+enum : int { kStatusWaitTimeout = 1 << 7 };         // 1 << STTM_ERR_TIMEOUT
 // launch shape of the instantiation with constant shape (D = 3584 bf16)
 constexpr int kFlagshipC = 4, kFlagshipS = 896, kFlagshipNM = 4, kFlagshipNA = 7;
 
@@ -147,7 +147,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // leaves its loops without touching the data it waited for; the warps that depend on it
 // run out in turn, every CTA still reaches the end of the kernel, and the host sees
 // kStatusWaitTimeout in the status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, int use, bool& timed_out) {
+__device__ __forceinline__ bool mbar_wait_lane(uint32_t bar, int use, bool& timed_out) {
     if (timed_out) return false;
     const uint32_t parity = (uint32_t)(use & 1);
     if (mbar_test(bar, parity)) return true;
@@ -161,18 +161,30 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, int use, bool& timed_out
     }
     return true;
 }
+// The same for a whole warp (every caller is one): the lanes agree on the outcome, so that a warp
+// never splits at the time limit with some lanes leaving and the others entering a warp-wide
+// primitive.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, int use, bool& timed_out) {
+    const bool ok = mbar_wait_lane(bar, use, timed_out);
+    const bool all = __all_sync(0xffffffffu, ok);
+    if (!all) timed_out = true;
+    return all;
+}
 // waits until a progress counter in shared memory (written by another warp of the CTA; only
 // a timing hint, no data hangs on it) has reached `target`; time-bounded like mbar_wait
 __device__ __forceinline__ bool hint_wait(const int* counter, int target, bool& timed_out) {
-    if (timed_out) return false;
+    bool ok = !timed_out;
     const volatile int* c = counter;
-    if (*c >= target) return true;
-    const unsigned long long t0 = global_timer_ns();
-    while (*c < target) {
-        __nanosleep(64);
-        if (global_timer_ns() - t0 > kWaitLimitNs) { timed_out = true; return false; }
+    if (ok && *c < target) {
+        const unsigned long long t0 = global_timer_ns();
+        while (*c < target) {
+            __nanosleep(64);
+            if (global_timer_ns() - t0 > kWaitLimitNs) { ok = false; break; }
+        }
     }
-    return true;
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) timed_out = true;
+    return ok;
 }
 // this CTA's shared memory -> shared memory of a CTA of the cluster, completion counted in
 // bytes on that CTA's mbarrier (both given as cluster addresses)

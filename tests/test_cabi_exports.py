@@ -59,3 +59,20 @@ def test_merged_positions_argument_checks_need_no_gpu():
     assert lib.sttm_merged_positions(addr, addr, 0, 10, addr, 2048, addr, 10, None, None) == 1
     assert lib.sttm_merged_positions(addr, addr, 1, 10, addr + 4, 2048, addr, 10, None, None) == 1   # misaligned ws
     assert lib.sttm_merged_positions(addr, addr, 1, 10, addr, 16, addr, 10, None, None) == 3        # STTM_ERR_WORKSPACE
+
+
+def test_device_status_word_decoding_needs_no_gpu():
+    """Host handling of the status word kernels OR their conditions into: every condition has a
+    bit of its own (the wait that ran out does not share one with a CUDA error), the lowest set
+    bit names the status, and every status has a message."""
+    lib = binding.load_library()
+    lib.sttm_status_string.restype = __import__("ctypes").c_char_p
+    names = {"capacity": 4, "not_converged": 5, "cuda": 6, "timeout": 7}
+    assert lib.sttm_status_from_bits(0) == 0
+    for code in names.values():
+        assert lib.sttm_status_from_bits(1 << code) == code
+    assert lib.sttm_status_from_bits((1 << names["timeout"]) | (1 << names["capacity"])) == names["capacity"]
+    assert lib.sttm_status_from_bits(1 << names["timeout"]) != lib.sttm_status_from_bits(1 << names["cuda"])
+    assert lib.sttm_status_string(names["timeout"]) == b"a wait inside a kernel ran out"
+    assert binding.STATUS_NAMES[names["timeout"]] == "a wait inside a kernel ran out"
+    assert len(binding.STATUS_NAMES) == 8

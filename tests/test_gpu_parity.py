@@ -238,7 +238,7 @@ def test_other_workload_shapes_full_width(shape):
             continue
         for out_dtype in (torch.float32, torch.bfloat16):
             run_and_compare(video, taus[0], taus[1], out_dtype=out_dtype)
-        assert binding.load_library().sttm_last_path() == 3          # the two-stream kernels took it
+        assert binding.load_library().sttm_last_path() == 1          # the single-pass kernel took it
         done += 1
         break
     assert done >= 1, "no seed gave thresholds with a margin"

@@ -45,6 +45,23 @@ def test_static_scratch_matches_workspace_variant_twice_in_a_row():
     _spatial_both_ways(first, 0.97)
 
 
+def test_static_entry_point_allocates_nothing():
+    # the array's address is known by now (first call done above or here); from then on the free
+    # device memory must not move across a call: no cudaMalloc, no growing cache behind the scenes
+    video = inputs.make_video(helpers.small_spec(44, 6, 13, 13, 256))
+    dev = helpers.to_torch(video)
+    T, H, W, D = video.shape
+    cover = torch.empty((1, T, H, W), dtype=torch.int8, device="cuda")
+    counts = torch.empty((1, T), dtype=torch.int32, device="cuda")
+    binding.sttm_spatial_static(dev, 0.9, cover, counts)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    binding.sttm_spatial_static(dev, 0.9, cover, counts)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+
+
 def test_static_scratch_fp32_and_two_level_grid():
     video = inputs.make_video(helpers.small_spec(43, 4, 8, 8, 64, dtype="f32", sigma=0.3))
     _spatial_both_ways(video, 0.9)
@@ -60,3 +77,8 @@ def test_problem_beyond_the_fixed_scratch_is_refused():
     with pytest.raises(binding.SttmError) as e:
         binding.sttm_spatial_static(feats, 0.9, cover, counts)
     assert e.value.code == 3
+    # exactly at the limit: 3120 frames are accepted
+    T = 3120
+    binding.sttm_spatial_static(feats[:, :T], 0.9, cover[:, :T], counts[:, :T])
+    torch.cuda.synchronize()
+    assert int(counts[0, :T].min()) >= 16

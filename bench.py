@@ -1,14 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the STTM token-merging path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload long]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload long|llava|qwen|mixed|tiny] [--budget 0.3|0.5]
 
 One step = one pass of the whole path (spatial quadtree search, temporal linking, root
-resolution, ordering, averaging into a packed output) over one synthetic video of the
-named workload, through the C ABI (sttm_merge_ex).  The default workload is the
-1024-frame, 13x13, D=3584 bf16 video (1.24 GB, ten times the L2) with the thresholds
-stored for it.  With N > 1 every rank merges its own copy of the video (independent
-videos, no data-path collective); the time is the maximum over ranks.
+resolution, ordering, averaging into a packed output) over the synthetic videos of the named
+workload, through the C ABI (one sttm_merge_ex call; the `mixed` workload is one call on its
+batch of eight videos with per-video thresholds).  The default workload is the 1024-frame,
+13x13, D=3584 bf16 video (1.24 GB, ten times the L2) at the thresholds stored for its 30 %
+token budget.  With N > 1 every rank merges its own copy of the workload (independent
+videos, no data-path collective); the time is the maximum over ranks.  Without a launcher
+(`WORLD_SIZE` unset) `--gpus N` starts the N ranks itself.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 """
@@ -17,8 +20,8 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import re
 import statistics
-import subprocess
 import sys
 import time
 
@@ -33,22 +36,34 @@ from paper_2507_07990_b200 import inputs  # noqa: E402
 METRIC = "input visual tokens/sec merged on 1 B200; achieved HBM GB/s vs peak"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-
-# DRAM traffic of a kernel as a multiple of its algorithmic bytes, from the ncu capture
-# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on the qwen workload;
-# a streaming kernel's traffic grows in proportion to the bytes it must move, so the ratio is
-# applied to the benchmark workload's algorithmic bytes).  Absent = no capture of the current kernel.
-NCU_TRAFFIC_RATIO = {"fused": 0.946}
+PROFILE_SUMMARY = os.path.join(ROOT, "profiles", "fused_kernel_long_and_qwen.md")
 
 
-def workload_setup(name: str):
+def ncu_traffic_ratio(kernel: str):
+    """DRAM traffic of a kernel as a multiple of its algorithmic bytes, as the ncu summary under
+    profiles/ states it (a line `dram_traffic_ratio <kernel> = <number>`); None when the summary
+    has no such line, i.e. there is no capture of the kernel as it stands."""
+    try:
+        with open(PROFILE_SUMMARY) as f:
+            m = re.search(r"dram_traffic_ratio\s+%s\s*=\s*([0-9.]+)" % re.escape(kernel), f.read())
+        return float(m.group(1)) if m else None
+    except OSError:
+        return None
+
+
+def workload_setup(name: str, budget=None):
+    """(config, specs, thresholds per video, budget key) of a named workload."""
     cfg = inputs.CONFIGS[name]
     table = inputs.load_thresholds()[name]
-    spec = inputs.config_videos(name, table.get("seed_bump", 0))[0]
-    per_budget = table["videos"][0]
-    key = "fixed" if "fixed" in per_budget else "%.2f" % cfg["budgets"][-1]
-    th = per_budget[key]
-    return cfg, spec, th, key
+    specs = inputs.config_videos(name, table.get("seed_bump", 0))
+    if "fixed" in table["videos"][0]:
+        key = "fixed"
+    else:
+        key = "%.2f" % (budget if budget is not None else cfg["budgets"][-1])
+        if key not in table["videos"][0]:
+            raise SystemExit("workload %s has no thresholds for budget %s (has %s)" % (name, key, sorted(table["videos"][0])))
+    ths = [v[key] for v in table["videos"]]
+    return cfg, specs, ths, key
 
 
 def measured_peak():
@@ -61,11 +76,11 @@ def measured_peak():
 
 
 class ClockSampler:
-    """SM clock and throttle reasons while the timed region runs, read through NVML every few
-    milliseconds from a thread (reading only: nothing on the GPU is set)."""
+    """SM clock and throttle reasons while the timed region runs, read through NVML every
+    millisecond or two from a thread (reading only: nothing on the GPU is set)."""
     REASONS = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40, "sw_power_cap": 0x4}
 
-    def __init__(self, index: int, period_s: float = 0.004):
+    def __init__(self, index: int, period_s: float = 0.001):
         import threading
         self.samples, self.max_mhz, self.bits = [], None, 0
         self._stop = threading.Event()
@@ -104,56 +119,126 @@ class ClockSampler:
                 "samples": len(self.samples), "reasons": reasons}
 
 
-def cpu_baseline(video_np, th, frames):
-    """The oracle as it stands, on the host cores, on the first `frames` frames."""
+def oracle_on_cores(video_np, th, chunk_frames, max_threads=None):
+    """The oracle as it stands on the host cores this process may use: the sample is cut into
+    runs of `chunk_frames` frames and every thread runs the whole oracle on its own run (the C
+    code releases the interpreter lock).  Chains that would cross a cut are cut, which changes
+    the row count a little and the work not at all.  Returns (tokens/s, threads, seconds, rows, frames)."""
+    import concurrent.futures as cf
     from oracle import oracle
-    sample = video_np[:frames]
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    threads = max(1, min(cores, video_np.shape[0] // chunk_frames, max_threads or cores))
+    chunks = [video_np[i * chunk_frames:(i + 1) * chunk_frames] for i in range(threads)]
+    oracle.merge(chunks[0][:2], th["tau_s"], th["tau_t"], want_feats=True)          # load the library first
+
+    def work(c):
+        return oracle.merge(c, th["tau_s"], th["tau_t"], want_feats=True).count
+
     t0 = time.perf_counter()
-    r = oracle.merge(sample, th["tau_s"], th["tau_t"], want_feats=True)
+    with cf.ThreadPoolExecutor(max_workers=threads) as ex:
+        rows = sum(ex.map(work, chunks))
     dt = time.perf_counter() - t0
-    tokens = sample.shape[0] * sample.shape[1] * sample.shape[2]
-    # want_feats runs the structure pass twice (once to size the output buffer)
-    return {"value": tokens / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": "first %d of %d frames (%d tokens), one thread, fp64, %.2f s, %d rows"
-                      % (sample.shape[0], video_np.shape[0], tokens, dt, r.count)}
+    frames = threads * chunk_frames
+    tokens = frames * video_np.shape[1] * video_np.shape[2]
+    return tokens / dt, threads, dt, rows, frames
+
+
+def cpu_baseline(video_np, th, chunk_frames):
+    value, threads, dt, rows, frames = oracle_on_cores(video_np, th, chunk_frames)
+    one, _, dt1, _, _ = oracle_on_cores(video_np, th, chunk_frames, max_threads=1)
+    return {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "cores_available": len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count(),
+            "one_thread": one,
+            "sample": "first %d of %d frames of video 0, %d threads x %d frames each, fp64, %.2f s (one thread on "
+                      "%d frames: %.2f s), %d rows" % (frames, video_np.shape[0], threads, chunk_frames, dt,
+                                                       chunk_frames, dt1, rows)}
+
+
+def workload_config(name, specs, ths, key):
+    spec = specs[0]
+    in_bytes = sum(s.tokens * s.D * (2 if s.dtype == "bf16" else 4) for s in specs)
+    tokens = sum(s.tokens for s in specs)
+    rows = sum(t["count"] for t in ths)
+    return {"workload": "%s: %d video%s/GPU, T=%d, %dx%d grid, D=%d %s, block generator p_static=%s sigma=%.2f, "
+                        "contrast classes %s"
+                        % (name, len(specs), "" if len(specs) == 1 else "s in one call", spec.T, spec.H, spec.W, spec.D,
+                           spec.dtype, "/".join("%.2f" % s.p_static for s in specs), spec.sigma, list(spec.contrast)),
+            "budget": key, "tau_s": [t["tau_s"] for t in ths], "tau_t": [t["tau_t"] for t in ths], "lv1": 4,
+            "kept_fraction": rows / tokens, "out_rows": rows, "rows_per_video": [t["count"] for t in ths],
+            "l2": "input (%.0f MB) larger than L2; no flush" % (in_bytes / 1e6) if in_bytes > 200e6
+                  else "L2 flushed between steps"}
 
 
 def run_reference(args):
+    """The reference arm: there is no reference implementation (the reference is a paper), so this
+    times the CPU oracle, as it stands, on a bounded sample of the workload per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    cfg, spec, th, key = workload_setup(args.workload)
+    cfg, specs, ths, key = workload_setup(args.workload, args.budget)
+    spec, th = specs[0], ths[0]
     frames = min(spec.T, args.reference_frames)
     import dataclasses
     video = inputs.make_video(dataclasses.replace(spec, T=frames))
-    from oracle import oracle
-    tokens = frames * spec.H * spec.W
+    chunk = max(2, min(frames, 32))
     for _ in range(args.warmup):
-        oracle.merge(video, th["tau_s"], th["tau_t"], want_feats=True)
+        oracle_on_cores(video, th, chunk)
     t0 = time.perf_counter()
+    used = 0
     for _ in range(args.steps):
-        oracle.merge(video, th["tau_s"], th["tau_t"], want_feats=True)
+        _, threads, _, _, used = oracle_on_cores(video, th, chunk)
     dt = time.perf_counter() - t0
+    tokens = used * spec.H * spec.W
     value = tokens * args.steps / dt
-    sample = "first %d of %d frames (%d tokens) per step, one thread, fp64" % (frames, spec.T, tokens)
+    sample = "first %d of %d frames of video 0 (%d tokens) per step, %d threads x %d frames, fp64" % (
+        used, spec.T, tokens, threads, chunk)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(args.workload, spec, th, key),
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "config": workload_config(args.workload, specs, ths, key),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
     return 0
 
 
-def workload_config(name, spec, th, key):
-    return {"workload": "%s: 1 video/GPU, T=%d, %dx%d grid, D=%d %s, block generator p_static=%.2f sigma=%.2f"
-                        % (name, spec.T, spec.H, spec.W, spec.D, spec.dtype, spec.p_static, spec.sigma),
-            "budget": key, "tau_s": th["tau_s"], "tau_t": th["tau_t"], "lv1": 4,
-            "kept_fraction": th["fraction"], "out_rows": th["count"],
-            "l2": "input (%.0f MB) larger than L2; no flush" % (spec.tokens * spec.D * 2 / 1e6)
-                  if spec.tokens * spec.D * 2 > 200e6 else "L2 flushed between steps"}
+def spawn_selftest(rank, world, port):
+    """CPU check of the rank start-up: gloo ranks, a max over ranks, one line from rank 0."""
+    import torch
+    import torch.distributed as dist
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    t = torch.tensor([float(rank + 1)], dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "selftest": True, "n_gpus": world, "max_over_ranks": float(t.item())}))
+    dist.destroy_process_group()
+
+
+def _spawned(rank, world, port, argv):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    sys.argv = argv
+    args = parse_args()
+    if args.selftest_spawn:
+        return spawn_selftest(rank, world, port)
+    run_ours(args)
+
+
+def spawn_ranks(args):
+    """`--gpus N` without a launcher: start the N ranks here (one process per GPU, NCCL)."""
+    import socket
+    import torch
+    import torch.multiprocessing as mp
+    if not args.selftest_spawn and torch.cuda.device_count() < args.gpus:
+        raise SystemExit("bench.py --gpus %d: only %d CUDA devices visible" % (args.gpus, torch.cuda.device_count()))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_spawned, args=(args.gpus, port, list(sys.argv)), nprocs=args.gpus, join=True)
+    return 0
 
 
 def run_ours(args):
@@ -169,29 +254,35 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    lib = binding.load_library()
     tuning = [int(v) for v in args.tuning.split(",")]
-    binding.load_library().sttm_set_tuning(*tuning[:3])
+    lib.sttm_set_tuning(*tuning[:3])
     if len(tuning) > 3:
-        binding.load_library().sttm_set_ring_split(*(tuning[3:5] + [0])[:2])
+        lib.sttm_set_ring_split(*(tuning[3:5] + [0])[:2])
 
-    cfg, spec, th, key = workload_setup(args.workload)
-    N = spec.tokens
-    in_bytes = N * spec.D * (2 if spec.dtype == "bf16" else 4)
+    cfg, specs, ths, key = workload_setup(args.workload, args.budget)
+    spec = specs[0]
+    B = len(specs)
+    N = sum(s.tokens for s in specs)
+    elt = 2 if spec.dtype == "bf16" else 4
+    in_bytes = N * spec.D * elt
     small = in_bytes <= 200e6
     tdtype = torch.bfloat16 if spec.dtype == "bf16" else torch.float32
+    tau_s = [t["tau_s"] for t in ths] if B > 1 else ths[0]["tau_s"]
+    tau_t = [t["tau_t"] for t in ths] if B > 1 else ths[0]["tau_t"]
 
-    # the video, generated once into pinned host memory and copied to the device
-    h_feats = torch.empty((1, spec.T, spec.H, spec.W, spec.D), dtype=tdtype).pin_memory()
+    # the videos, generated once into pinned host memory and copied to the device
+    shape = (B, spec.T, spec.H, spec.W, spec.D)
+    h_feats = torch.empty(shape, dtype=tdtype).pin_memory()
     view = h_feats.view(torch.int16).numpy().view(np.uint16) if spec.dtype == "bf16" else h_feats.numpy()
-    inputs.make_video(spec, out=view[0])
+    for b, s in enumerate(specs):
+        inputs.make_video(s, out=view[b])
     d_feats = h_feats.cuda()
     if args.budget_rows > 0:
-        # budget mode: tau_t chosen on the device for this many rows (two passes of the fused kernel)
-        plan = binding.BudgetPlan((1, spec.T, spec.H, spec.W, spec.D), tdtype, th["tau_s"], args.budget_rows,
-                                  out_dtype=torch.bfloat16, want_map=False)
+        # budget mode: tau_t chosen on the device for this many rows per video
+        plan = binding.BudgetPlan(shape, tdtype, tau_s, args.budget_rows, out_dtype=torch.bfloat16, want_map=False)
     else:
-        plan = binding.MergePlan((1, spec.T, spec.H, spec.W, spec.D), tdtype, th["tau_s"], th["tau_t"],
-                                 out_dtype=torch.bfloat16, want_map=False,
+        plan = binding.MergePlan(shape, tdtype, tau_s, tau_t, out_dtype=torch.bfloat16, want_map=False,
                                  match=binding.MATCH_BEST if args.match == "best" else binding.MATCH_TOPLEFT)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
 
@@ -204,15 +295,18 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         out = plan.run(d_feats)
     torch.cuda.synchronize()
-    count = int(out.out_count[0].item())
+    counts = [int(v) for v in out.out_count.tolist()]
+    count = sum(counts)
     status = int(out.device_status.item())
     if status != 0:
         raise RuntimeError("device status %d" % status)
+    if args.budget_rows == 0 and args.match == "topleft" and counts != [t["count"] for t in ths]:
+        raise RuntimeError("row counts %s differ from the calibrated %s" % (counts, [t["count"] for t in ths]))
     launches_per_step = out.launches
 
     # The step is also captured once as a CUDA graph (the same kernels, launched by one replay
-    # instead of nine calls).  Every fourth timed step goes through the library call with stage
-    # events set (they give the kernels' own durations), the others replay the graph.
+    # instead of one call per kernel).  Every fourth timed step goes through the library call with
+    # stage events set (they give the kernels' own durations), the others replay the graph.
     graph = None
     if not args.no_graph:
         try:
@@ -226,14 +320,13 @@ def run_ours(args):
                 plan.run(d_feats)
             graph.replay()
             torch.cuda.synchronize()
-            if int(plan.out_count[0].item()) != count or int(plan.status.item()) != 0:
+            if int(plan.out_count.sum().item()) != count or int(plan.status.item()) != 0:
                 raise RuntimeError("graph replay gave another result")
         except Exception as exc:          # capture not possible here: every step is a direct call
             print("bench: no CUDA graph (%s)" % exc, file=sys.stderr)
             graph = None
     sampled = [k for k in range(args.steps) if graph is None or k % 4 == 0]
     timers = {k: binding.StageTimer() for k in sampled}
-    lib = binding.load_library()
     step_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                    for _ in range(args.steps)]
     sampler = ClockSampler(local) if rank == 0 else None
@@ -260,6 +353,8 @@ def run_ours(args):
     total_ms = float(total_ms.item())
     ms_per_step = total_ms / args.steps
     value = world * N * args.steps / (total_ms / 1e3)
+    direct_ms = [step_ms[k] for k in sampled]
+    replay_ms = [step_ms[k] for k in range(args.steps) if k not in timers]
 
     # per-stage times over the sampled steps of the timed region (events on the launching stream)
     stage_ms = {}
@@ -269,89 +364,109 @@ def run_ours(args):
     out_bytes = count * spec.D * 2
     id_bytes = count * 4
     path_bytes = in_bytes + out_bytes + id_bytes
-    # algorithmic bytes per launch of each feature-touching stage: every stage of the three-pass
-    # kernels reads the input once; the fused kernel reads it once and writes every output row once
-    # (to its staging place), the gather moves every output row once more
-    if lib.sttm_last_path() == 3:
+    # algorithmic bytes per launch of each feature-touching stage: the single-pass kernel reads the
+    # input once and writes every output row once (to its staging place), its gather moves every row
+    # once more; the Gram stage of the two-stream kernels reads the input, their sum stage reads it
+    # again and writes every row; every stage of the three-pass kernels reads the input once
+    path_id = lib.sttm_last_path()
+    if path_id == 3:
         stage_bytes = {"gram": in_bytes, "sum": in_bytes + out_bytes}
-    elif lib.sttm_last_path() == 1:
+    elif path_id == 1:
         stage_bytes = {"fused": in_bytes + out_bytes, "gather": 2 * out_bytes}
     else:
         stage_bytes = {"spatial": in_bytes, "temporal+roots": in_bytes, "accumulate": in_bytes + out_bytes}
     dominant = max(stage_bytes, key=lambda n: stage_ms.get(n, 0.0))
     peak, peak_kind = measured_peak()
     achieved = stage_bytes[dominant] / (stage_ms[dominant] / 1e3) / 1e9
+    ratio = ncu_traffic_ratio(dominant)
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": "of " + peak_kind,
-                "traffic": (NCU_TRAFFIC_RATIO[dominant] * stage_bytes[dominant]
-                            if dominant in NCU_TRAFFIC_RATIO else None),
+                "traffic": ratio * stage_bytes[dominant] if ratio is not None else None,
                 "algorithmic_bytes": stage_bytes[dominant], "kernel_ms": stage_ms[dominant],
                 "stage_ms": stage_ms,
                 "path": {"algorithmic_bytes": path_bytes, "achieved": path_bytes / (ms_per_step / 1e3) / 1e9,
                          "frac": path_bytes / (ms_per_step / 1e3) / 1e9 / peak,
                          "frac_of_8000": path_bytes / (ms_per_step / 1e3) / 1e9 / 8000.0}}
 
-    # end to end through the host-buffer entry point: H2D of the video, D2H of the result
+    # end to end through the host-buffer entry point: H2D of the videos, D2H of the result
     e2e_steps = max(1, min(args.steps, 5 if not small else args.steps))
     h_out = torch.empty((N, spec.D), dtype=torch.bfloat16).pin_memory()
     h_pos = torch.empty((N,), dtype=torch.int32).pin_memory()
-    binding.sttm_merge_host(h_feats, th["tau_s"], th["tau_t"], h_out_feats=h_out, h_out_pos=h_pos)
+    e2e_tau_t = tau_t
+    if args.budget_rows > 0:
+        e2e_tau_t = [float(v) for v in plan.tau.tolist()] if B > 1 else float(plan.tau[0].item())
+    binding.sttm_merge_host(h_feats, tau_s, e2e_tau_t, h_out_feats=h_out, h_out_pos=h_pos)
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        r = binding.sttm_merge_host(h_feats, th["tau_s"], th["tau_t"], h_out_feats=h_out, h_out_pos=h_pos)
+        r = binding.sttm_merge_host(h_feats, tau_s, e2e_tau_t, h_out_feats=h_out, h_out_pos=h_pos)
     barrier()
     e2e_s = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
     e2e = {"value": world * N * e2e_steps / float(e2e_s.item()), "unit": UNIT, "h2d_bytes_per_step": in_bytes,
-           "d2h_bytes_per_step": out_bytes + id_bytes + 4 + 16, "steps": e2e_steps,
+           "d2h_bytes_per_step": out_bytes + id_bytes + 4 * B + 8 * (B + 1) + 4, "steps": e2e_steps,
            "ms_per_step": 1e3 * float(e2e_s.item()) / e2e_steps}
-    assert int(r.out_count[0]) == count
+    assert int(sum(r.out_count)) == count
 
     if rank == 0:
+        mhz = clocks["sm_mhz"] if clocks else None
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+                "ms_median": statistics.median(step_ms), "ms_best": min(step_ms),
+                "ms_direct_call": statistics.mean(direct_ms) if direct_ms else None,
+                "ms_graph_replay": statistics.mean(replay_ms) if replay_ms else None,
+                "ms_x_mhz": ms_per_step * mhz if mhz else None,
+                "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": dict(workload_config(args.workload, spec, th, key),
+                "config": dict(workload_config(args.workload, specs, ths, key),
                                match=args.match, budget_rows=args.budget_rows,
                                launch=("3 of 4 steps replay a CUDA graph of the library call, every 4th is the call "
                                        "itself with stage events") if graph is not None else "library calls"),
-                "out_rows": count,
+                "out_rows": count, "rows_per_video": counts,
                 "launch_shape": binding.sttm_fused_launch_shape(plan.problem),
                 "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "clocks": clocks}
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(view[0], th, min(spec.T, args.baseline_frames))
+            line["cpu_baseline"] = cpu_baseline(view[0], ths[0], min(spec.T, args.baseline_frames))
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
     return 0
 
 
-def main():
+def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long", choices=list(inputs.CONFIGS))
-    ap.add_argument("--baseline-frames", type=int, default=512,
-                    help="frames of the workload the CPU-baseline leg runs the oracle on")
-    ap.add_argument("--reference-frames", type=int, default=64,
-                    help="frames per step of the --impl reference arm")
+    ap.add_argument("--budget", type=float, default=None,
+                    help="token budget whose stored thresholds are used (0.5 or 0.3; default: the workload's last)")
+    ap.add_argument("--baseline-frames", type=int, default=64,
+                    help="frames every thread of the CPU-baseline leg runs the oracle on")
+    ap.add_argument("--reference-frames", type=int, default=256,
+                    help="frames of video 0 the --impl reference arm shares out over its threads per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="every timed step is a direct library call")
     ap.add_argument("--budget-rows", type=int, default=0,
-                    help="time the budget mode (sttm_merge_budget) with this row budget instead of fixed thresholds")
+                    help="time the budget mode (sttm_merge_budget) with this row budget per video instead of fixed thresholds")
     ap.add_argument("--match", default="topleft", choices=["topleft", "best"],
                     help="destination rule of the temporal link (the paper's default, or its most-similar variant)")
     ap.add_argument("--tuning", default="0,0,0",
-                    help="path,cluster_size,frames_per_item for sttm_set_tuning, optionally followed by "
-                         "sum_slots,lead_frames for sttm_set_ring_split (0 = library's choice)")
-    args = ap.parse_args()
+                    help="path,cluster_size,frames_per_item for sttm_set_tuning (path 5: the two-stream kernels), "
+                         "optionally followed by sum_slots,lead_frames for sttm_set_ring_split (0 = library's choice)")
+    ap.add_argument("--selftest-spawn", action="store_true", help=argparse.SUPPRESS)
+    return ap.parse_args()
+
+
+def main():
+    args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if "WORLD_SIZE" not in os.environ and (args.gpus > 1 or args.selftest_spawn):
+        return spawn_ranks(args)
     return run_ours(args)
 
 

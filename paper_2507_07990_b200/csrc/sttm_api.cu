@@ -99,7 +99,7 @@ struct Plan {
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
         frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
-        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_next, flow_partial,
+        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_row, lead_n, lead_ids, flow_partial,
         flow_hand, flow_recs, total;
 };
 
@@ -409,7 +409,8 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         plan_flow(p, g, &pl->fl, budget);
         if (!pl->fl.ok) plan_fused(p, g, &pl->f);
     }
-    pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = pl->piece_next = o;
+    pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = o;
+    pl->piece_row = pl->lead_n = pl->lead_ids = o;
     pl->flow_partial = pl->flow_hand = pl->flow_recs = o;
     if (pl->fl.ok) {
         const FlowPlan& f = pl->fl;
@@ -418,7 +419,9 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         pl->ones_end = o;
         pl->pieces = take((size_t)f.nitems * kPieceSlots * g.D * sizeof(float));
         pl->piece_meta = take((size_t)f.nitems * kPieceSlots * sizeof(int2));
-        pl->piece_next = take((size_t)f.nitems * kPieceSlots * 4);
+        pl->piece_row = take((size_t)f.nitems * kPieceSlots * 4);
+        pl->lead_n = take((size_t)f.nitems * kPieceSlots * 4);
+        pl->lead_ids = take((size_t)f.nitems * kPieceSlots * kRowPieces * 4);
         pl->flow_partial = take((size_t)f.nitems * (f.F + 1) * f.NS * kSumVals * sizeof(float));
         pl->flow_hand = take((size_t)f.nitems * (f.F + 1) * 16 * 4);
         pl->flow_recs = take((size_t)f.nitems * (f.F + 2) * sizeof(FrameRec));
@@ -431,7 +434,9 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         pl->staging = take((size_t)pl->cells * g.D * out_elt);
         pl->pieces = take((size_t)pl->f.nitems * kPieceSlots * g.D * sizeof(float));
         pl->piece_meta = take((size_t)pl->f.nitems * kPieceSlots * sizeof(int2));
-        pl->piece_next = take((size_t)pl->f.nitems * kPieceSlots * 4);
+        pl->piece_row = take((size_t)pl->f.nitems * kPieceSlots * 4);
+        pl->lead_n = take((size_t)pl->f.nitems * kPieceSlots * 4);
+        pl->lead_ids = take((size_t)pl->f.nitems * kPieceSlots * kRowPieces * 4);
     }
     pl->total = o;
     return STTM_OK;
@@ -664,15 +669,23 @@ sttm_status launch_after_smem(void (*kernel)(KArgs...), unsigned grid, unsigned 
     return e == cudaSuccess ? STTM_OK : STTM_ERR_CUDA;
 }
 
+// Chains cut by item borders: rows, leaders and lists of the pieces, then the rows themselves.
 template <typename OutT>
-sttm_status launch_gather_pieces(const Plan& pl, int npieces, char* ws, void* out, long long capacity, cudaStream_t st) {
+sttm_status launch_pieces(const Plan& pl, int npieces, char* ws, void* out, long long capacity, cudaStream_t st) {
     const Geo g = pl.g;
-    const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
-    const unsigned blocks = std::min<unsigned>(blocks_for(max_rows * kGatherParts, 8), sm_count() * 16);
-    return launch_after(k_gather_pieces<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
-                        (const int32_t*)(ws + pl.row_head), (const int32_t*)(ws + pl.piece_next),
-                        (const int32_t*)(ws + pl.row_weight), (const float*)(ws + pl.pieces), (OutT*)out, capacity,
-                        npieces);
+    sttm_status s = launch_after(k_piece_link, blocks_for(npieces, 256), 256, st, g, npieces,
+                                 (const int2*)(ws + pl.piece_meta), (const int32_t*)(ws + pl.root),
+                                 (const int32_t*)(ws + pl.row_at_root), (const long long*)(ws + pl.vid_off),
+                                 (int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.piece_row), (int32_t*)(ws + pl.lead_n),
+                                 (int32_t*)(ws + pl.row_weight));
+    if (s != STTM_OK) return s;
+    s = launch_after(k_piece_group, blocks_for(npieces, 256), 256, st, npieces, (const int32_t*)(ws + pl.piece_row),
+                     (const int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.lead_n), (int32_t*)(ws + pl.lead_ids));
+    if (s != STTM_OK) return s;
+    const unsigned blocks = std::min<unsigned>(blocks_for((long long)npieces * kPieceParts, 8), sm_count() * 8);
+    return launch_after(k_gather_pieces<OutT>, blocks, 256, st, g, npieces, (const int32_t*)(ws + pl.piece_row),
+                        (const int32_t*)(ws + pl.lead_n), (const int32_t*)(ws + pl.lead_ids),
+                        (const int32_t*)(ws + pl.row_weight), (const float*)(ws + pl.pieces), (OutT*)out, capacity);
 }
 
 // Tensor maps of the feature tensor for the three kinds of tile.  The tensor is described as
@@ -794,12 +807,8 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
         if (s != STTM_OK) return s;
     }
     const int npieces = f.nitems * kPieceSlots;
-    s = launch_after(k_piece_link, blocks_for(npieces, 256), 256, st, g, npieces, (const int2*)(ws + pl.piece_meta),
-                     (const int32_t*)root, (const int32_t*)row_at_root, (const long long*)vid_off,
-                     (int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.piece_next), (int32_t*)(ws + pl.row_weight));
-    if (s != STTM_OK) return s;
-    s = p->out_dtype == STTM_BF16 ? launch_gather_pieces<__nv_bfloat16>(pl, npieces, ws, out_feats, p->out_capacity_rows, st)
-                                  : launch_gather_pieces<float>(pl, npieces, ws, out_feats, p->out_capacity_rows, st);
+    s = p->out_dtype == STTM_BF16 ? launch_pieces<__nv_bfloat16>(pl, npieces, ws, out_feats, p->out_capacity_rows, st)
+                                  : launch_pieces<float>(pl, npieces, ws, out_feats, p->out_capacity_rows, st);
     mark_stage(4, st);
     mark_stage(5, st);
     return s;
@@ -813,14 +822,13 @@ sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacit
     // and blocks without a row would only cost their launch)
     const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
     const unsigned blocks = std::min<unsigned>(blocks_for(max_rows * kGatherParts, 8), sm_count() * 16);
-    sttm_status s = launch_after(k_gather_rows<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
+    // (first the rows made of pieces: the copy below leaves out the rows that have a leader piece)
+    sttm_status s = launch_pieces<OutT>(pl, pl.f.nitems * kPieceSlots, ws, out, capacity, st);
+    if (s != STTM_OK) return s;
+    s = launch_after(k_gather_rows<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
                                  (const int32_t*)(ws + pl.row_anchor), (const int32_t*)(ws + pl.row_head),
                                  (const OutT*)(ws + pl.staging), (OutT*)out, capacity);
-    if (s != STTM_OK) return s;
-    return launch_after(k_gather_pieces<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
-                        (const int32_t*)(ws + pl.row_head), (const int32_t*)(ws + pl.piece_next),
-                        (const int32_t*)(ws + pl.row_weight), (const float*)(ws + pl.pieces), (OutT*)out, capacity,
-                        pl.f.nitems * kPieceSlots);
+    return s;
 }
 
 template <typename T, typename OutT>
@@ -1159,12 +1167,6 @@ sttm_status merge_impl(const void* feats, const sttm_params* p, void* ws_, size_
                              (const int32_t*)row_at_root, merge_map);
             if (s != STTM_OK) return s;
         }
-        const int npieces = pl.f.nitems * kPieceSlots;
-        s = launch_after(k_piece_link, blocks_for(npieces, 256), 256, st, g, npieces,
-                         (const int2*)(ws + pl.piece_meta), (const int32_t*)root, (const int32_t*)row_at_root,
-                         (const long long*)vid_off, (int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.piece_next),
-                         (int32_t*)(ws + pl.row_weight));
-        if (s != STTM_OK) return s;
         mark_stage(3, st);
         s = p->out_dtype == STTM_BF16 ? launch_gather<__nv_bfloat16>(pl, ws, out_feats, p->out_capacity_rows, st)
                                       : launch_gather<float>(pl, ws, out_feats, p->out_capacity_rows, st);

@@ -307,18 +307,33 @@ k_flow_chain(const __grid_constant__ FlowParams p) {
             row_next = valid ? p.row_at_root[(long long)it.b * p.N + (long long)(it.tstart + j + 1) * p.HW + lg.cell] : -1;
         }
         if (j == it.n) {
-            // closing record: everything still running is written out
+            // Closing record: everything still running is written out.  A chain goes on into the next
+            // item iff a node of that item's first frame is linked to its node of this frame; the
+            // others end here like any chain that ends inside the item.
+            uint32_t goes_on = 0;
+            if (!it.last_seg) {
+                const int nxt = p.hand[((long long)(it.item + p.ntiles) * (p.F + 1) + 1) * 16 + c];
+                const int nlv = nxt & 3, nlink = (nxt >> 8) - 1;
+                const bool nlinked = valid && lane_anchor(lg, c, nlv) == c && nlink >= 0;
+                const int tslot = __shfl_sync(full, prev_slot, nlink < 0 ? 0 : nlink);
+                goes_on = __reduce_or_sync(full, nlinked ? 1u << tslot : 0u);
+            }
+            uint32_t empty = 0;
             if (low && ((active_slots >> lane) & 1u)) {
-                if (!tab->virt[lane] && it.last_seg) {
+                const bool on = (goes_on >> lane) & 1u;
+                if (!tab->virt[lane] && !on) {
                     const long long grow = vrow0 + tab->row[lane];
                     rec->flush[lane] = FlushCmd{lane, 0, grow < p.capacity ? (int)grow : -1, (float)tab->weight[lane]};
+                } else if (tab->virt[lane] && tab->weight[lane] == 0 && !on) {
+                    empty = 1u << lane;             // came in from the frame before the item and got no member here
                 } else {
                     const int pc = it.item * kPieceSlots + 16 + lane;
                     rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
                     p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
                 }
             }
-            if (lane == 0) rec->flush_mask = active_slots;
+            empty = __reduce_or_sync(full, empty);
+            if (lane == 0) rec->flush_mask = active_slots & ~empty;
         } else {
             const int lv = packed & 3, link_local = (packed >> 8) - 1;
             const int t = it.tstart + j;
@@ -340,8 +355,11 @@ k_flow_chain(const __grid_constant__ FlowParams p) {
             const int wint = p.weight_mode ? __popc(cells) : 1;
             const long long gc = (long long)it.b * p.N + (long long)t * p.HW + lg.cell;
             // chains that ended: lane s looks at slot s (before the slot is given away again)
+            uint32_t empty = 0;
             if (low && ((dead >> lane) & 1u)) {
-                if (tab->virt[lane]) {
+                if (tab->virt[lane] && tab->weight[lane] == 0) {
+                    empty = 1u << lane;             // a node of the frame before the item that nothing was linked to: no piece
+                } else if (tab->virt[lane]) {
                     const int pc = it.item * kPieceSlots + tab->cell[lane];
                     rec->flush[lane] = FlushCmd{lane, 1, pc, 0.f};
                     p.piece_meta[pc] = make_int2(tab->key[lane], tab->weight[lane]);
@@ -368,7 +386,8 @@ k_flow_chain(const __grid_constant__ FlowParams p) {
                 const float wc = (lv == 0 ? 1.f : (lv == 1 ? w1 : w2)) * (float)wnode;
                 rec->wmat[cur_slot * 16 + c] = __bfloat16_as_ushort(__float2bfloat16_rn(wc));
             }
-            if (lane == 0) rec->flush_mask = dead;
+            empty = __reduce_or_sync(full, empty);
+            if (lane == 0) rec->flush_mask = dead & ~empty;
             if (!is_halo && low && valid) p.chain_key[gc] = tab->key[cur_slot] - it.b * p.N;
             active_slots = memb | __reduce_or_sync(full, fresh ? 1u << slot_fresh : 0u);
             prev_slot = cur_slot;

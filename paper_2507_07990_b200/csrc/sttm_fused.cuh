@@ -1137,24 +1137,44 @@ k_resolve_roots(Geo g, int max_hops, const int32_t* __restrict__ chain_key, int3
 }
 
 // ---------------------------------------------------------------------------------
-// After the ordering: chains cut by item borders.  One thread per piece: find the row of
-// the piece's chain, add its weight, push it on the row's list.
+// After the ordering: chains cut by item borders.  A row that is put together from pieces is
+// named by its smallest piece index, the leader.  k_piece_link (one thread per piece) finds the
+// piece's row, adds its weight and proposes itself as the row's leader; k_piece_group (after it)
+// enters every piece in its leader's list.
 // ---------------------------------------------------------------------------------
+constexpr int kRowPieces = 64;          // pieces listed per row; a row with more is found by a scan of all pieces
+
 __global__ void __launch_bounds__(256)
 k_piece_link(Geo g, int npieces, const int2* __restrict__ piece_meta, const int32_t* __restrict__ root,
              const int32_t* __restrict__ row_at_root, const long long* __restrict__ vid_off,
-             int32_t* __restrict__ row_head, int32_t* __restrict__ piece_next, int32_t* __restrict__ row_weight) {
+             int32_t* __restrict__ row_head, int32_t* __restrict__ piece_row, int32_t* __restrict__ lead_n,
+             int32_t* __restrict__ row_weight) {
     wait_for_prior_kernel();
     const int pc = blockIdx.x * blockDim.x + threadIdx.x;
     if (pc >= npieces) return;
+    lead_n[pc] = 0;
     const int2 m = piece_meta[pc];
-    if (m.x < 0) return;
+    if (m.x < 0) { piece_row[pc] = -1; return; }
     const int b = m.x / g.N;
     const long long vb = (long long)b * g.N;
     const int r = root[vb + (m.x - b * g.N)];
     const long long row = vid_off[b] + row_at_root[vb + r];
-    piece_next[pc] = atomicExch(row_head + row, pc);
+    piece_row[pc] = (int32_t)row;
+    atomicMin(reinterpret_cast<unsigned int*>(row_head) + row, (unsigned int)pc);      // (no leader yet: all bits set)
     atomicAdd(row_weight + row, m.y);
+}
+
+__global__ void __launch_bounds__(256)
+k_piece_group(int npieces, const int32_t* __restrict__ piece_row, const int32_t* __restrict__ row_head,
+              int32_t* __restrict__ lead_n, int32_t* __restrict__ lead_ids) {
+    wait_for_prior_kernel();
+    const int pc = blockIdx.x * blockDim.x + threadIdx.x;
+    if (pc >= npieces) return;
+    const int row = piece_row[pc];
+    if (row < 0) return;
+    const int leader = row_head[row];
+    const int at = atomicAdd(lead_n + leader, 1);
+    if (at < kRowPieces) lead_ids[(long long)leader * kRowPieces + at] = pc;
 }
 
 // Gather: kGatherParts warps per output row, each a contiguous share of the channels.  Two
@@ -1216,87 +1236,87 @@ k_gather_rows(Geo g, const long long* __restrict__ vid_off, const int32_t* __res
     }
 }
 
+// Rows put together from pieces: kPieceParts warps per such row, found through its leader piece.
+// The pieces are added in the order of their index (a fixed order, so the result does not depend
+// on scheduling); such a row is bound by the latency of its loads, so four pieces' loads are issued
+// before anything is added.
+constexpr int kPieceParts = 8;
 template <typename OutT>
 __global__ void __launch_bounds__(256)
-k_gather_pieces(Geo g, const long long* __restrict__ vid_off, const int32_t* __restrict__ row_head,
-                const int32_t* __restrict__ piece_next, const int32_t* __restrict__ row_weight,
-                const float* __restrict__ pieces, OutT* __restrict__ out, long long capacity, int max_pieces) {
+k_gather_pieces(Geo g, int npieces, const int32_t* __restrict__ piece_row, const int32_t* __restrict__ lead_n,
+                const int32_t* __restrict__ lead_ids, const int32_t* __restrict__ row_weight,
+                const float* __restrict__ pieces, OutT* __restrict__ out, long long capacity) {
     wait_for_prior_kernel();
+    __shared__ int s_ids[8][2 * kRowPieces];
     const int lane = threadIdx.x & 31;
-    const long long nunits = min(vid_off[g.B], capacity) * kGatherParts;
+    const long long nunits = (long long)npieces * kPieceParts;
     const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
     const int nf4 = g.D / VEC;                                      // 4-channel groups of a row
+    int* ids = s_ids[threadIdx.x >> 5];
+    int* sorted = ids + kRowPieces;
     for (long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); unit < nunits; unit += nwarps) {
-        const long long r = unit / kGatherParts;
-        const int part = (int)(unit % kGatherParts);
-        const int head = row_head[r];
-        if (head < 0) continue;                         // a finished staging row
-        // the row's pieces in increasing index order; lists are short (a few per item border):
-        // one walk that keeps the first eight sorted in registers (the walk also stops after as
-        // many steps as there are pieces at all, whatever the list holds)
-        constexpr int kMaxList = 8;
-        int ids[kMaxList];
-        int n = 0, steps = 0;
-        bool longer = false;
-        for (int pc = head; pc >= 0 && steps < max_pieces; pc = piece_next[pc], steps++) {
-            if (n == kMaxList) { longer = true; break; }
-            int v = pc;
-#pragma unroll
-            for (int k = 0; k < kMaxList; k++) {
-                if (k < n) {
-                    const int lo = min(ids[k], v);
-                    v = max(ids[k], v);
-                    ids[k] = lo;
-                } else if (k == n) {
-                    ids[k] = v;
-                }
-            }
-            n++;
+        const int leader = (int)(unit / kPieceParts), part = (int)(unit % kPieceParts);
+        const int n_all = lead_n[leader];
+        if (n_all == 0) continue;                       // not a leader
+        const long long r = piece_row[leader];
+        if (r >= capacity) continue;
+        const int n = min(n_all, kRowPieces);
+        __syncwarp();
+        for (int i = lane; i < n; i += 32) ids[i] = lead_ids[(long long)leader * kRowPieces + i];
+        __syncwarp();
+        for (int i = lane; i < n; i += 32) {
+            const int mine = ids[i];
+            int rank = 0;
+            for (int k = 0; k < n; k++) rank += ids[k] < mine ? 1 : 0;
+            sorted[rank] = mine;
         }
+        __syncwarp();
         const float wsum = (float)row_weight[r];
-        const int lo = (int)((long long)nf4 * part / kGatherParts), hi = (int)((long long)nf4 * (part + 1) / kGatherParts);
-        // eight groups per trip (a quarter of a 3584-channel row is seven): 8 x n loads in flight
-        for (int f0 = lo + lane; f0 < hi; f0 += 8 * 32) {
-            float sum[8][VEC];
+        const int lo = (int)((long long)nf4 * part / kPieceParts), hi = (int)((long long)nf4 * (part + 1) / kPieceParts);
+        for (int f0 = lo + lane; f0 < hi; f0 += 4 * 32) {
+            float sum[4][VEC];
 #pragma unroll
-            for (int u = 0; u < 8; u++)
+            for (int u = 0; u < 4; u++)
 #pragma unroll
                 for (int v = 0; v < VEC; v++) sum[u][v] = 0.f;
-            if (!longer) {
+            if (n_all <= kRowPieces) {
+                for (int k0 = 0; k0 < n; k0 += 4) {
+                    float4 v[4][4];
 #pragma unroll
-                for (int k = 0; k < kMaxList; k++) {
-                    if (k < n) {
-                        const float4* src = reinterpret_cast<const float4*>(pieces + (long long)ids[k] * g.D);
-                        float4 v[8];
+                    for (int k = 0; k < 4; k++) {
+                        if (k0 + k < n) {
+                            const float4* src = reinterpret_cast<const float4*>(pieces + (long long)sorted[k0 + k] * g.D);
 #pragma unroll
-                        for (int u = 0; u < 8; u++)
-                            if (f0 + u * 32 < hi) v[u] = __ldcs(src + f0 + u * 32);
+                            for (int u = 0; u < 4; u++)
+                                if (f0 + u * 32 < hi) v[k][u] = __ldcs(src + f0 + u * 32);
+                        }
+                    }
 #pragma unroll
-                        for (int u = 0; u < 8; u++)
-                            if (f0 + u * 32 < hi) {
-                                sum[u][0] += v[u].x; sum[u][1] += v[u].y; sum[u][2] += v[u].z; sum[u][3] += v[u].w;
-                            }
+                    for (int k = 0; k < 4; k++) {
+                        if (k0 + k < n) {
+#pragma unroll
+                            for (int u = 0; u < 4; u++)
+                                if (f0 + u * 32 < hi) {
+                                    sum[u][0] += v[k][u].x; sum[u][1] += v[k][u].y; sum[u][2] += v[k][u].z; sum[u][3] += v[k][u].w;
+                                }
+                        }
                     }
                 }
             } else {
-                int lst = -1;
-                for (int round = 0; round < max_pieces; round++) {
-                    int best = 0x7fffffff, hops = 0;
-                    for (int pc = head; pc >= 0 && hops < max_pieces; pc = piece_next[pc], hops++)
-                        if (pc > lst && pc < best) best = pc;
-                    if (best == 0x7fffffff) break;
-                    const float4* src = reinterpret_cast<const float4*>(pieces + (long long)best * g.D);
+                // more pieces than a list holds: all pieces are looked through, in index order
+                for (int q = leader; q < npieces; q++) {
+                    if (piece_row[q] != (int32_t)r) continue;
+                    const float4* src = reinterpret_cast<const float4*>(pieces + (long long)q * g.D);
 #pragma unroll
-                    for (int u = 0; u < 8; u++)
+                    for (int u = 0; u < 4; u++)
                         if (f0 + u * 32 < hi) {
                             const float4 v = src[f0 + u * 32];
                             sum[u][0] += v.x; sum[u][1] += v.y; sum[u][2] += v.z; sum[u][3] += v.w;
                         }
-                    lst = best;
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 8; u++)
+            for (int u = 0; u < 4; u++)
                 if (f0 + u * 32 < hi) {
 #pragma unroll
                     for (int v = 0; v < VEC; v++) sum[u][v] = sum[u][v] / wsum;

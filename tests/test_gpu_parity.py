@@ -225,10 +225,15 @@ def test_bad_arguments_are_rejected_on_the_host():
 # Shapes of the paper's other set-ups at their real feature widths: the 14x14 grid of
 # LLaVA-Video (Section 3.2), a non-square dynamic-resolution grid (three levels: grids up to 16 cells a side), and D = 8192 of the 72B
 # model (eight CTAs per cluster, eight sum warps per CTA).
-@pytest.mark.parametrize("shape", [(6, 14, 14, 3584), (4, 16, 12, 3584), (5, 13, 13, 8192), (3, 16, 16, 8192)],
+@pytest.mark.parametrize("path", [1, 3], ids=["singlepass", "twostream"])
+@pytest.mark.parametrize("shape", [(6, 14, 14, 3584), (4, 16, 12, 3584), (5, 13, 13, 8192), (3, 16, 16, 8192),
+                                   (5, 9, 5, 3584), (4, 13, 5, 1024)],
                          ids=lambda s: "T%dH%dW%dD%d" % s)
-def test_other_workload_shapes_full_width(shape):
+def test_other_workload_shapes_full_width(shape, path):
+    # (9x5 and 13x5: grids one cell higher and wider than a multiple of four, whose last row and
+    # column the two-stream kernels load as strips of 16 cells)
     T, H, W, D = shape
+    lib = binding.load_library()
     done = 0
     for seed in range(3):
         spec = helpers.small_spec(300 + seed, T, H, W, D, sigma=0.05)
@@ -236,9 +241,13 @@ def test_other_workload_shapes_full_width(shape):
         taus = helpers.safe_thresholds(video, 0.5, 0.5)
         if taus is None:
             continue
-        for out_dtype in (torch.float32, torch.bfloat16):
-            run_and_compare(video, taus[0], taus[1], out_dtype=out_dtype)
-        assert binding.load_library().sttm_last_path() == 1          # the single-pass kernel took it
+        lib.sttm_set_tuning(5 if path == 3 else 0, 0, 2 if path == 3 else 0)
+        try:
+            for out_dtype in (torch.float32, torch.bfloat16):
+                run_and_compare(video, taus[0], taus[1], out_dtype=out_dtype)
+            assert lib.sttm_last_path() == path
+        finally:
+            lib.sttm_set_tuning(0, 0, 0)
         done += 1
         break
     assert done >= 1, "no seed gave thresholds with a margin"

@@ -107,6 +107,7 @@ struct Plan {
 int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0, g_tune_pack = 0, g_tune_sum_slots = 0, g_tune_lead = 0;
 
 constexpr size_t kMaxSmem = 232448;   // 227 KB per CTA on sm_100
+constexpr double kFlowMinBytes = 512e6;                    // input size from which the two-stream kernels are the default
 constexpr size_t kFlowSmemMax = (233472 - 2 * 1024) / 2;   // per CTA when two share an SM
 
 // Cuts the grid into the kernel's tiles.  Full 4x4 tiles map one to one.  The partial tiles of
@@ -225,8 +226,11 @@ bool build_flow_tiles(const Geo& g, FlowPlan* f) {
 // Two-stream kernels: bf16 input, channels a multiple of 64, slices of up to eight 64-channel blocks.
 void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
     f->ok = false;
-    // on request, and for the budget mode (its second pass reuses the first pass's Gram stage)
-    if (!(g_tune_path == 5 || (g_tune_path == 0 && budget))) return;
+    // On request, for the budget mode (its second pass reuses the first pass's Gram stage), and for
+    // large inputs: measured on B200, the two-stream kernels overtake the single-pass kernel between
+    // 0.25 GB (qwen: 0.23 against 0.21 ms) and 1.2 GB (long: 0.68 against 0.71 ms) of features.
+    const bool large = (double)g.B * g.N * g.D * 2.0 >= kFlowMinBytes;
+    if (!(g_tune_path == 5 || (g_tune_path == 0 && (budget || large)))) return;
     if (p->in_dtype != STTM_BF16 || g.D % 64 != 0) return;
     if (!build_flow_tiles(g, f)) return;
     const int nblk = g.D / 64;
@@ -247,7 +251,24 @@ void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
     if (R == 0) return;
     f->R = R;
     f->smem = (size_t)f->R * f->slot_bytes + flow_fixed_smem(f->R);
-    f->F = std::min(g.T, g_tune_seg > 0 ? std::min(g_tune_seg, kFlowMaxF) : 32);
+    // Frames per item: the tasks (item x slice) are dealt round robin to two CTAs per SM, so the
+    // stages take rounds x (frames of an item + the frame before it + what starting a task costs);
+    // the shortest such product over the admissible item lengths (long items mean few pieces, short
+    // items mean enough tasks for a short video to fill the GPU).
+    if (g_tune_seg > 0) {
+        f->F = std::min(g.T, std::min(g_tune_seg, kFlowMaxF));
+    } else {
+        const long long ctas = 2ll * sm_count();
+        long long best_cost = -1;
+        int best_F = std::min(g.T, 32);
+        for (int F = std::min(g.T, kFlowMaxF); F >= std::min(g.T, 8); F--) {
+            const long long nseg = (g.T + F - 1) / F;
+            const long long tasks = (long long)g.B * f->ntiles * nseg * f->NS;
+            const long long cost = ((tasks + ctas - 1) / ctas) * (F + 1 + 3);
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_F = F; }
+        }
+        f->F = best_F;
+    }
     f->nseg = (g.T + f->F - 1) / f->F;
     f->nitems = g.B * f->ntiles * f->nseg;
     f->ok = true;

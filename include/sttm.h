@@ -250,9 +250,12 @@ sttm_status sttm_merge_host(const void* h_feats, const sttm_params* p,
  * tau_t}; the threshold returned is the middle of the gap between the k-th and the (k+1)-th largest
  * best cosine, k = nodes - budget (2.0 when the spatial stage alone meets the budget; -2.0, and
  * more rows than asked for, when even linking every node that has a candidate does not).  Equal
- * best cosines at the cut leave the count off by their number.  Runs the fused kernel twice
- * (once to collect the best cosines, once to merge); only for shapes the fused kernel covers
- * (STTM_ERR_UNSUPPORTED otherwise); tau_t / tau_t_per_video of *p are ignored.
+ * best cosines at the cut leave the count off by their number.  The features are streamed once
+ * for all similarities (whose sums are kept), the decisions are taken twice (once without links to
+ * collect the best cosines, once with the chosen thresholds), then the averages are formed: about
+ * 1.4 times the cost of a call with given thresholds.  Only for quadtrees of up to three levels,
+ * bf16 input and D a multiple of 16 (STTM_ERR_UNSUPPORTED otherwise); tau_t / tau_t_per_video of
+ * *p are ignored.
  *   budget_rows  host, [B]: rows allowed per video (>= 1)
  *   ws           at least sttm_budget_workspace_bytes(p) bytes, 256-byte aligned
  *   tau_t_out    [B] float32, may be NULL: the thresholds chosen
@@ -305,12 +308,15 @@ void sttm_set_stage_events(void** events);
 
 /*
  * Benchmark and test knobs; 0 leaves a choice to the library.
- *   path             1: always the three-pass kernels, 2 or 0: the fused single-read kernel
+ *   path             0: the library's choice (the two-stream kernels from 0.5 GB of features on
+ *                    and for the budget mode, else the single-pass kernel, else the three-pass
+ *                    kernels), 1: always the three-pass kernels, 2: the single-pass kernel
  *                    wherever it applies (bf16 input, D a multiple of 16, at most 64 tiles of
  *                    4x4 cells per frame, D / cluster_size <= 1024), 3: the same without
- *                    packing the partial border tiles of a frame together
- *   cluster_size     CTAs that share one tile's channels (1, 2, 4 or 8)
- *   frames_per_item  frames of one tile that one cluster processes in a row
+ *                    packing the partial border tiles of a frame together, 5: the two-stream
+ *                    kernels wherever they apply (bf16 input, D a multiple of 64)
+ *   cluster_size     single-pass kernel: CTAs that share one tile's channels (1, 2, 4 or 8)
+ *   frames_per_item  frames of one tile that are processed in a row (two-stream kernels: at most 64)
  * Not thread safe; affects later calls of every entry point.
  */
 void sttm_set_tuning(int path, int cluster_size, int frames_per_item);
@@ -328,8 +334,8 @@ void sttm_set_tuning(int path, int cluster_size, int frames_per_item);
  */
 void sttm_set_ring_split(int sum_slots, int lead_frames);
 
-/* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 fused, 2 the
- * general kernels for quadtrees of more than three levels. */
+/* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 single-pass (fused),
+ * 2 the general kernels for quadtrees of more than three levels, 3 two-stream. */
 int sttm_last_path(void);
 
 /*

@@ -3,6 +3,7 @@
 #include "../../include/sttm.h"
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cmath>
@@ -53,8 +54,20 @@ const char* const kStageNames[4][kStageCount] = {
     {"gram", "decide+ordering+chain", "sum", "roots+pieces", "-"}};
 thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: single-pass kernel, 2: general kernels, 3: two-stream kernels
 
+// Stage boundary `boundary` (before stage `boundary`, after the one before it): an event for the
+// benchmark when it asked for them, and an NVTX range named after the stage around the launches
+// of the stage, so that a timeline shows the path's stages (costs nothing without a profiler).
+thread_local bool g_range_open = false;
+inline void close_stage_range() {
+    if (g_range_open) { nvtxRangePop(); g_range_open = false; }
+}
 inline void mark_stage(int boundary, cudaStream_t st) {
     if (g_stage_events != nullptr) cudaEventRecord(g_stage_events[boundary], st);
+    close_stage_range();
+    if (boundary < kStageCount && kStageNames[g_last_path][boundary][0] != '-') {
+        nvtxRangePushA(kStageNames[g_last_path][boundary]);
+        g_range_open = true;
+    }
 }
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
@@ -1104,8 +1117,10 @@ sttm_status sttm_temporal(const void* feats, const sttm_params* p, void* ws, siz
 sttm_status sttm_merge_ex(const void* feats, const sttm_params* p, void* ws_, size_t ws_bytes, void* out_feats,
                           int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
                           int32_t* device_status, void* stream) {
-    return merge_impl(feats, p, ws_, ws_bytes, out_feats, out_pos, merge_map, out_count, out_offsets, device_status,
-                      Internal(), stream);
+    const sttm_status s = merge_impl(feats, p, ws_, ws_bytes, out_feats, out_pos, merge_map, out_count, out_offsets,
+                                     device_status, Internal(), stream);
+    close_stage_range();
+    return s;
 }
 
 }  // extern "C"
@@ -1308,6 +1323,7 @@ sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const lon
     first.tmax = tmax;
     s = merge_impl(feats, &q, ws, main_bytes, out_feats, out_pos, nullptr, out_count, out_offsets, device_status, first,
                    stream);
+    close_stage_range();
     if (s != STTM_OK) return s;
     Budgets bd = {};
     for (int b = 0; b < p->B; b++) bd.rows[b] = budget_rows[b];
@@ -1321,6 +1337,7 @@ sttm_status sttm_merge_budget(const void* feats, const sttm_params* p, const lon
     second.second_pass = pl.fl.ok;      // the two-stream kernels keep the first pass's Gram stage
     s = merge_impl(feats, p, ws, main_bytes, out_feats, out_pos, merge_map, out_count, out_offsets, device_status, second,
                    stream);
+    close_stage_range();
     if (s != STTM_OK) return s;
     if (tau_t_out != nullptr)
         STTM_CUDA_TRY(cudaMemcpyAsync(tau_t_out, tau_dev, sizeof(float) * p->B, cudaMemcpyDeviceToDevice, st));

@@ -36,19 +36,24 @@ from paper_2507_07990_b200 import inputs  # noqa: E402
 METRIC = "input visual tokens/sec merged on 1 B200; achieved HBM GB/s vs peak"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-PROFILE_SUMMARY = os.path.join(ROOT, "profiles", "fused_kernel_long_and_qwen.md")
+PROFILE_DIR = os.path.join(ROOT, "profiles")
 
 
 def ncu_traffic_ratio(kernel: str):
-    """DRAM traffic of a kernel as a multiple of its algorithmic bytes, as the ncu summary under
-    profiles/ states it (a line `dram_traffic_ratio <kernel> = <number>`); None when the summary
-    has no such line, i.e. there is no capture of the kernel as it stands."""
+    """DRAM traffic of a kernel as a multiple of its algorithmic bytes, as an ncu summary under
+    profiles/ states it (a line `dram_traffic_ratio <kernel> = <number>`); None when no summary
+    has such a line, i.e. there is no capture of the kernel as it stands."""
     try:
-        with open(PROFILE_SUMMARY) as f:
-            m = re.search(r"dram_traffic_ratio\s+%s\s*=\s*([0-9.]+)" % re.escape(kernel), f.read())
-        return float(m.group(1)) if m else None
+        for name in sorted(os.listdir(PROFILE_DIR)):
+            if not name.endswith((".md", ".txt")):
+                continue
+            with open(os.path.join(PROFILE_DIR, name)) as f:
+                m = re.search(r"dram_traffic_ratio\s+%s\s*=\s*([0-9.]+)" % re.escape(kernel), f.read())
+            if m:
+                return float(m.group(1))
     except OSError:
-        return None
+        pass
+    return None
 
 
 def workload_setup(name: str, budget=None):

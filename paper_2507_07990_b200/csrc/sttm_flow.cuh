@@ -14,8 +14,8 @@
 //   chain stage   one warp per (tile, run of frames) follows the chains through the run and
 //                 leaves one command record per frame: a 16 x 16 matrix W (chain slot x cell)
 //                 and the list of chains that ended, each with its final output row.
-//   sum stage     streams the features a second time (out of L2 where the two streams run close
-//                 together) and forms the chain averages of Section 3.3 as running sums
+//   sum stage     streams the features a second time and forms the chain averages of Section 3.3
+//                 as running sums
 //                 sums[16 chain slots x channels] += W X on the tensor cores.  A chain that ends
 //                 is divided by its weight and written straight to its output row.  Chains that
 //                 cross the border between two runs of frames leave fp32 pieces that a small

@@ -703,15 +703,41 @@ sttm_status launch_after_smem(void (*kernel)(KArgs...), unsigned grid, unsigned 
     return e == cudaSuccess ? STTM_OK : STTM_ERR_CUDA;
 }
 
+// Ordering: rows of the surviving tokens from the per-frame counts.  Up to kRowsScanFrames frames every
+// block of the row kernel adds up the counts before its own frame itself; beyond that the counts are
+// scanned once by a kernel of their own.
+constexpr long long kRowsScanFrames = 4096;
+sttm_status launch_ordering(const Plan& pl, const sttm_params* p, char* ws, const int8_t* cover, const int32_t* link,
+                            int32_t* out_pos, int32_t* out_count, int64_t* out_offsets, int32_t* device_status,
+                            cudaStream_t st) {
+    const Geo g = pl.g;
+    const int32_t* frame_roots = (const int32_t*)(ws + pl.frame_counts);
+    int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
+    long long* vid_off = (long long*)(ws + pl.vid_off);
+    int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
+    int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
+    if ((long long)g.B * g.T <= kRowsScanFrames)
+        return launch_after(k_rows_scan, (unsigned)(g.B * g.T), 256, st, g, cover, link, frame_roots, out_count, vid_off,
+                            out_offsets, row_at_root, row_anchor, out_pos, (long long)p->out_capacity_rows, (int)p->pos,
+                            device_status);
+    sttm_status s = launch_after(k_scan_frames, 1u, 1024, st, g, frame_roots, frame_base, out_count, vid_off, out_offsets);
+    if (s != STTM_OK) return s;
+    return launch_after(k_rows, (unsigned)(g.B * g.T), 256, st, g, cover, link, (const int32_t*)frame_base,
+                        (const long long*)vid_off, row_at_root, row_anchor, out_pos, (long long)p->out_capacity_rows,
+                        (int)p->pos, device_status);
+}
+
 // Chains cut by item borders: rows, leaders and lists of the pieces, then the rows themselves.
 template <typename OutT>
-sttm_status launch_pieces(const Plan& pl, int npieces, char* ws, void* out, long long capacity, cudaStream_t st) {
+sttm_status launch_pieces(const Plan& pl, int npieces, char* ws, void* out, long long capacity, int32_t* status,
+                          cudaStream_t st) {
     const Geo g = pl.g;
     sttm_status s = launch_after(k_piece_link, blocks_for(npieces, 256), 256, st, g, npieces,
-                                 (const int2*)(ws + pl.piece_meta), (const int32_t*)(ws + pl.root),
+                                 (pl.fl.ok ? pl.fl.nseg : pl.f.nseg) + 1,
+                                 (const int2*)(ws + pl.piece_meta), (const int32_t*)(ws + pl.cell_row),
                                  (const int32_t*)(ws + pl.row_at_root), (const long long*)(ws + pl.vid_off),
                                  (int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.piece_row), (int32_t*)(ws + pl.lead_n),
-                                 (int32_t*)(ws + pl.row_weight));
+                                 (int32_t*)(ws + pl.row_weight), status);
     if (s != STTM_OK) return s;
     s = launch_after(k_piece_group, blocks_for(npieces, 256), 256, st, npieces, (const int32_t*)(ws + pl.piece_row),
                      (const int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.lead_n), (int32_t*)(ws + pl.lead_ids));
@@ -812,19 +838,13 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     const int pairs = (f.F + 2) / 2;
     s = launch_after(k_flow_decide, blocks_for((long long)f.nitems * pairs, 8), 256, st, fp, taus);
     if (s != STTM_OK) return s;
-    int32_t* frame_roots = (int32_t*)(ws + pl.frame_counts);
-    int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
-    long long* vid_off = (long long*)(ws + pl.vid_off);
     int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
-    int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
     int32_t* root = (int32_t*)(ws + pl.root);
-    s = launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)frame_roots, frame_base, out_count, vid_off,
-                     out_offsets);
-    if (s != STTM_OK) return s;
-    if (in.tmax != nullptr) return STTM_OK;            // first pass of the budget mode: only the node counts are needed
-    s = launch_after(k_rows, (unsigned)(g.B * g.T), 256, st, g, (const int8_t*)fp.cover, (const int32_t*)fp.link,
-                     (const int32_t*)frame_base, (const long long*)vid_off, row_at_root, row_anchor, out_pos,
-                     (long long)p->out_capacity_rows, (int)p->pos, device_status);
+    if (in.tmax != nullptr)                            // first pass of the budget mode: only the node counts are needed
+        return launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)(ws + pl.frame_counts),
+                            (int32_t*)(ws + pl.frame_base), out_count, (long long*)(ws + pl.vid_off), out_offsets);
+    s = launch_ordering(pl, p, ws, (const int8_t*)fp.cover, (const int32_t*)fp.link, out_pos, out_count, out_offsets,
+                        device_status, st);
     if (s != STTM_OK) return s;
     s = launch_after(k_flow_chain, blocks_for(f.nitems, kChainWarps), kChainWarps * 32, st, fp);
     if (s != STTM_OK) return s;
@@ -832,24 +852,24 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     s = launch_after_smem(k_flow<true>, grid, kFlowThreads, f.smem, true, st, fp, maps);
     if (s != STTM_OK) return s;
     mark_stage(3, st);
-    s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, f.nseg + 1,
-                     (const int32_t*)(ws + pl.cell_row), root, device_status);
-    if (s != STTM_OK) return s;
     if (merge_map != nullptr) {
+        s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, f.nseg + 1,
+                         (const int32_t*)(ws + pl.cell_row), root, device_status);
+        if (s != STTM_OK) return s;
         s = launch_after(k_merge_map, blocks_for(pl.cells, 256), 256, st, g, (const int32_t*)root,
                          (const int32_t*)row_at_root, merge_map);
         if (s != STTM_OK) return s;
     }
     const int npieces = f.nitems * kPieceSlots;
-    s = p->out_dtype == STTM_BF16 ? launch_pieces<__nv_bfloat16>(pl, npieces, ws, out_feats, p->out_capacity_rows, st)
-                                  : launch_pieces<float>(pl, npieces, ws, out_feats, p->out_capacity_rows, st);
+    s = p->out_dtype == STTM_BF16 ? launch_pieces<__nv_bfloat16>(pl, npieces, ws, out_feats, p->out_capacity_rows, device_status, st)
+                                  : launch_pieces<float>(pl, npieces, ws, out_feats, p->out_capacity_rows, device_status, st);
     mark_stage(4, st);
     mark_stage(5, st);
     return s;
 }
 
 template <typename OutT>
-sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacity, cudaStream_t st) {
+sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacity, int32_t* status, cudaStream_t st) {
     const Geo g = pl.g;
     // kGatherParts warps per row, striding; the row count is only known on the device, so the grid
     // covers the most rows there can be, up to a few waves of blocks (most tokens merge: few rows,
@@ -857,7 +877,7 @@ sttm_status launch_gather(const Plan& pl, char* ws, void* out, long long capacit
     const long long max_rows = std::min<long long>(pl.cells, std::max<long long>(capacity, 1));
     const unsigned blocks = std::min<unsigned>(blocks_for(max_rows * kGatherParts, 8), sm_count() * 16);
     // (first the rows made of pieces: the copy below leaves out the rows that have a leader piece)
-    sttm_status s = launch_pieces<OutT>(pl, pl.f.nitems * kPieceSlots, ws, out, capacity, st);
+    sttm_status s = launch_pieces<OutT>(pl, pl.f.nitems * kPieceSlots, ws, out, capacity, status, st);
     if (s != STTM_OK) return s;
     s = launch_after(k_gather_rows<OutT>, blocks, 256, st, g, (const long long*)(ws + pl.vid_off),
                                  (const int32_t*)(ws + pl.row_anchor), (const int32_t*)(ws + pl.row_head),
@@ -1182,30 +1202,21 @@ sttm_status merge_impl(const void* feats, const sttm_params* p, void* ws_, size_
             return launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)(ws + pl.frame_counts),
                                 (int32_t*)(ws + pl.frame_base), out_count, (long long*)(ws + pl.vid_off), out_offsets);
         }
-        s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, pl.f.nseg + 1,
-                         (const int32_t*)(ws + pl.cell_row), root, device_status);
-        if (s != STTM_OK) return s;
         mark_stage(2, st);
-        int32_t* frame_roots = (int32_t*)(ws + pl.frame_counts);     // counted by the fused kernel
-        int32_t* frame_base = (int32_t*)(ws + pl.frame_base);
-        long long* vid_off = (long long*)(ws + pl.vid_off);
-        int32_t* row_at_root = (int32_t*)(ws + pl.row_at_root);
-        int32_t* row_anchor = (int32_t*)(ws + pl.row_anchor);
-        s = launch_after(k_scan_frames, 1u, 1024, st, g, (const int32_t*)frame_roots, frame_base, out_count, vid_off,
-                         out_offsets);
-        if (s != STTM_OK) return s;
-        s = launch_after(k_rows, (unsigned)(g.B * g.T), 256, st, g, (const int8_t*)cover, (const int32_t*)link,
-                         (const int32_t*)frame_base, (const long long*)vid_off, row_at_root, row_anchor, out_pos,
-                         (long long)p->out_capacity_rows, (int)p->pos, device_status);
+        s = launch_ordering(pl, p, ws, (const int8_t*)cover, (const int32_t*)link, out_pos, out_count, out_offsets,
+                            device_status, st);
         if (s != STTM_OK) return s;
         if (merge_map != nullptr) {
+            s = launch_after(k_resolve_roots, blocks_for(pl.cells, 256), 256, st, g, pl.f.nseg + 1,
+                             (const int32_t*)(ws + pl.cell_row), root, device_status);
+            if (s != STTM_OK) return s;
             s = launch_after(k_merge_map, blocks_for(pl.cells, 256), 256, st, g, (const int32_t*)root,
-                             (const int32_t*)row_at_root, merge_map);
+                             (const int32_t*)(ws + pl.row_at_root), merge_map);
             if (s != STTM_OK) return s;
         }
         mark_stage(3, st);
-        s = p->out_dtype == STTM_BF16 ? launch_gather<__nv_bfloat16>(pl, ws, out_feats, p->out_capacity_rows, st)
-                                      : launch_gather<float>(pl, ws, out_feats, p->out_capacity_rows, st);
+        s = p->out_dtype == STTM_BF16 ? launch_gather<__nv_bfloat16>(pl, ws, out_feats, p->out_capacity_rows, device_status, st)
+                                      : launch_gather<float>(pl, ws, out_feats, p->out_capacity_rows, device_status, st);
         mark_stage(4, st);
         mark_stage(5, st);
         return s;

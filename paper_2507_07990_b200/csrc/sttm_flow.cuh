@@ -123,6 +123,10 @@ __device__ __forceinline__ bool mbar_wait_sleep(uint32_t bar, int use, bool& tim
     }
     return true;
 }
+// The k-th task a kernel takes up.  The Gram stage goes through the video forwards, the sum stage
+// backwards: what the Gram stage read last is what L2 still holds when the sum stage begins.
+__device__ __forceinline__ int flow_task(bool sum_stage, int k, int ntasks) { return sum_stage ? ntasks - 1 - k : k; }
+
 // bounded wait whose outcome is the same in every lane of the warp
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, int use, bool& timed_out) {
     const bool ok = mbar_wait_sleep(bar, use, timed_out);
@@ -465,8 +469,9 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
         const int nthr = kFlowWorkers * 32;
         const uint32_t redsum_a = smem_u32(redsum), W2s = smem_u32(wtab);
         for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
-            const FlowItem it = flow_item(p, task / p.NS);
-            const int slice = task % p.NS;
+            const int tk = flow_task(kSum, task, ntasks);
+            const FlowItem it = flow_item(p, tk / p.NS);
+            const int slice = tk % p.NS;
             const LaneGeo lg = lane_geo(p.tiles[it.tile], tid & 15, p.L, p.W);
             named_sync(1, nthr);                       // the previous task's weights are not read any more
             if (tid < 16) wtab[tid] = lg.w2;
@@ -550,8 +555,9 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
             const uint32_t woff = 16 + 256 + lrow * 32 + (lane >> 4) * 16;
             const int ntmax = 2 * warp + 1 < p.NB ? 16 : 8;     // an odd block count leaves the last warp one block
             for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
-                const FlowItem it = flow_item(p, task / p.NS);
-                const int slice = task % p.NS;
+                const int tk = flow_task(kSum, task, ntasks);
+                const FlowItem it = flow_item(p, tk / p.NS);
+                const int slice = tk % p.NS;
                 const long long chan0 = ((long long)slice * p.NB + 2 * warp) * 64;
                 // one record per frame, and a closing one that writes out what the item leaves
                 for (int j = 0; j <= it.n; j++, q++) {
@@ -619,8 +625,9 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
         // One tensor copy per frame (and, in the sum stage, one plain bulk copy of the frame's
         // record), all on the slot's barrier.
         for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
-            const FlowItem it = flow_item(p, task / p.NS);
-            const int slice = task % p.NS;
+            const int tk = flow_task(kSum, task, ntasks);
+            const FlowItem it = flow_item(p, tk / p.NS);
+            const int slice = tk % p.NS;
             const TileBox bx = p.boxes[it.tile];
             const int nslots = it.n + (kSum ? 1 : 0);
             for (int j = 0; j < nslots; j++, q++) {

@@ -1145,10 +1145,10 @@ k_resolve_roots(Geo g, int max_hops, const int32_t* __restrict__ chain_key, int3
 constexpr int kRowPieces = 64;          // pieces listed per row; a row with more is found by a scan of all pieces
 
 __global__ void __launch_bounds__(256)
-k_piece_link(Geo g, int npieces, const int2* __restrict__ piece_meta, const int32_t* __restrict__ root,
+k_piece_link(Geo g, int npieces, int max_hops, const int2* __restrict__ piece_meta, const int32_t* __restrict__ chain_key,
              const int32_t* __restrict__ row_at_root, const long long* __restrict__ vid_off,
              int32_t* __restrict__ row_head, int32_t* __restrict__ piece_row, int32_t* __restrict__ lead_n,
-             int32_t* __restrict__ row_weight) {
+             int32_t* __restrict__ row_weight, int32_t* status) {
     wait_for_prior_kernel();
     const int pc = blockIdx.x * blockDim.x + threadIdx.x;
     if (pc >= npieces) return;
@@ -1157,7 +1157,18 @@ k_piece_link(Geo g, int npieces, const int2* __restrict__ piece_meta, const int3
     if (m.x < 0) { piece_row[pc] = -1; return; }
     const int b = m.x / g.N;
     const long long vb = (long long)b * g.N;
-    const int r = root[vb + (m.x - b * g.N)];
+    // the root of the piece's chain: the hand-over walk of k_resolve_roots, for this one cell
+    int r = chain_key[m.x];
+    int hops = 0;
+    while (true) {
+        const int up = chain_key[vb + r];
+        if (up == r) break;
+        r = up;
+        if (++hops > max_hops) {
+            if (status != nullptr) atomicOr(status, kStatusNotConverged);
+            break;
+        }
+    }
     const long long row = vid_off[b] + row_at_root[vb + r];
     piece_row[pc] = (int32_t)row;
     atomicMin(reinterpret_cast<unsigned int*>(row_head) + row, (unsigned int)pc);      // (no leader yet: all bits set)

@@ -422,6 +422,59 @@ k_rows(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__ link
     }
 }
 
+// The same with the scan folded in (one launch less): every block adds up the root counts of the
+// frames before its own (all frames of the earlier videos, the earlier frames of its video); the
+// first block of a video also writes the video's count and offset.
+__global__ void __launch_bounds__(256)
+k_rows_scan(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__ link,
+            const int32_t* __restrict__ frame_roots, int32_t* __restrict__ out_count, long long* __restrict__ vid_off,
+            int64_t* out_offsets, int32_t* __restrict__ row_at_root, int32_t* __restrict__ row_anchor,
+            int32_t* __restrict__ out_pos, long long capacity, int pos_mode, int32_t* status) {
+    wait_for_prior_kernel();
+    __shared__ int sm[33];
+    const long long bt = blockIdx.x;
+    const int b = (int)(bt / g.T), t = (int)(bt % g.T);
+    int before_videos = 0, before_frames = 0, after_frames = 0;
+    for (int i = threadIdx.x; i < b * g.T; i += blockDim.x) before_videos += frame_roots[i];
+    for (int i = threadIdx.x; i < g.T; i += blockDim.x) {
+        const int v = frame_roots[(long long)b * g.T + i];
+        if (i < t) before_frames += v; else after_frames += v;
+    }
+    int off_i, carry, rest;
+    block_exclusive_scan(before_videos, off_i, sm);
+    __syncthreads();
+    block_exclusive_scan(before_frames, carry, sm);
+    __syncthreads();
+    block_exclusive_scan(after_frames, rest, sm);
+    __syncthreads();
+    const long long off = off_i;
+    if (t == 0 && threadIdx.x == 0) {
+        out_count[b] = carry + rest;
+        vid_off[b] = off;
+        if (out_offsets != nullptr) out_offsets[b] = off;
+        if (b == g.B - 1) {
+            vid_off[g.B] = off + carry + rest;
+            if (out_offsets != nullptr) out_offsets[g.B] = off + carry + rest;
+        }
+    }
+    for (int c0 = 0; c0 < g.HW; c0 += blockDim.x) {
+        const int cell = c0 + threadIdx.x;
+        const int flag = cell < g.HW && is_root_anchor(g, cell, cover[bt * g.HW + cell], link[bt * g.HW + cell]);
+        int total;
+        const int ex = block_exclusive_scan(flag, total, sm);
+        if (flag) {
+            const int row = carry + ex;
+            const long long grow = off + row;
+            row_at_root[bt * g.HW + cell] = row;
+            row_anchor[grow] = t * g.HW + cell;
+            if (grow < capacity) out_pos[grow] = pos_mode ? row : t * g.HW + cell;
+            else if (status != nullptr) atomicOr(status, kStatusCapacity);
+        }
+        carry += total;
+        __syncthreads();
+    }
+}
+
 // one thread per cell: row of the cell's root; per row: total weight and last frame
 __global__ void __launch_bounds__(256)
 k_members(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__ root,

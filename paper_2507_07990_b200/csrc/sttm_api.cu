@@ -112,7 +112,7 @@ struct Plan {
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
         frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
-        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_row, lead_n, lead_ids, flow_partial,
+        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_row, lead_n, lead_ids, lead_list, flow_partial,
         flow_hand, flow_recs, total;
 };
 
@@ -444,7 +444,7 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         if (!pl->fl.ok) plan_fused(p, g, &pl->f);
     }
     pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = o;
-    pl->piece_row = pl->lead_n = pl->lead_ids = o;
+    pl->piece_row = pl->lead_n = pl->lead_ids = pl->lead_list = o;
     pl->flow_partial = pl->flow_hand = pl->flow_recs = o;
     if (pl->fl.ok) {
         const FlowPlan& f = pl->fl;
@@ -454,7 +454,8 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         pl->pieces = take((size_t)f.nitems * kPieceSlots * g.D * sizeof(float));
         pl->piece_meta = take((size_t)f.nitems * kPieceSlots * sizeof(int2));
         pl->piece_row = take((size_t)f.nitems * kPieceSlots * 4);
-        pl->lead_n = take((size_t)f.nitems * kPieceSlots * 4);
+        pl->lead_n = take(((size_t)f.nitems * kPieceSlots + 1) * 4);
+        pl->lead_list = take((size_t)f.nitems * kPieceSlots * 4);
         pl->lead_ids = take((size_t)f.nitems * kPieceSlots * kRowPieces * 4);
         pl->flow_partial = take((size_t)f.nitems * (f.F + 1) * f.NS * kSumVals * sizeof(float));
         pl->flow_hand = take((size_t)f.nitems * (f.F + 1) * 16 * 4);
@@ -469,7 +470,8 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         pl->pieces = take((size_t)pl->f.nitems * kPieceSlots * g.D * sizeof(float));
         pl->piece_meta = take((size_t)pl->f.nitems * kPieceSlots * sizeof(int2));
         pl->piece_row = take((size_t)pl->f.nitems * kPieceSlots * 4);
-        pl->lead_n = take((size_t)pl->f.nitems * kPieceSlots * 4);
+        pl->lead_n = take(((size_t)pl->f.nitems * kPieceSlots + 1) * 4);
+        pl->lead_list = take((size_t)pl->f.nitems * kPieceSlots * 4);
         pl->lead_ids = take((size_t)pl->f.nitems * kPieceSlots * kRowPieces * 4);
     }
     pl->total = o;
@@ -740,11 +742,13 @@ sttm_status launch_pieces(const Plan& pl, int npieces, char* ws, void* out, long
                                  (int32_t*)(ws + pl.row_weight), status);
     if (s != STTM_OK) return s;
     s = launch_after(k_piece_group, blocks_for(npieces, 256), 256, st, npieces, (const int32_t*)(ws + pl.piece_row),
-                     (const int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.lead_n), (int32_t*)(ws + pl.lead_ids));
+                     (const int32_t*)(ws + pl.row_head), (int32_t*)(ws + pl.lead_n), (int32_t*)(ws + pl.lead_ids),
+                     (int32_t*)(ws + pl.lead_list));
     if (s != STTM_OK) return s;
-    const unsigned blocks = std::min<unsigned>(blocks_for((long long)npieces * kPieceParts, 8), sm_count() * 8);
+    const unsigned blocks = std::min<unsigned>(blocks_for((long long)npieces * kPieceParts, 8), sm_count() * 3);
     return launch_after(k_gather_pieces<OutT>, blocks, 256, st, g, npieces, (const int32_t*)(ws + pl.piece_row),
                         (const int32_t*)(ws + pl.lead_n), (const int32_t*)(ws + pl.lead_ids),
+                        (const int32_t*)(ws + pl.lead_list),
                         (const int32_t*)(ws + pl.row_weight), (const float*)(ws + pl.pieces), (OutT*)out, capacity);
 }
 

@@ -1153,6 +1153,7 @@ k_piece_link(Geo g, int npieces, int max_hops, const int2* __restrict__ piece_me
     const int pc = blockIdx.x * blockDim.x + threadIdx.x;
     if (pc >= npieces) return;
     lead_n[pc] = 0;
+    if (pc == 0) lead_n[npieces] = 0;                   // number of leaders, counted by k_piece_group
     const int2 m = piece_meta[pc];
     if (m.x < 0) { piece_row[pc] = -1; return; }
     const int b = m.x / g.N;
@@ -1177,7 +1178,7 @@ k_piece_link(Geo g, int npieces, int max_hops, const int2* __restrict__ piece_me
 
 __global__ void __launch_bounds__(256)
 k_piece_group(int npieces, const int32_t* __restrict__ piece_row, const int32_t* __restrict__ row_head,
-              int32_t* __restrict__ lead_n, int32_t* __restrict__ lead_ids) {
+              int32_t* __restrict__ lead_n, int32_t* __restrict__ lead_ids, int32_t* __restrict__ lead_list) {
     wait_for_prior_kernel();
     const int pc = blockIdx.x * blockDim.x + threadIdx.x;
     if (pc >= npieces) return;
@@ -1186,6 +1187,8 @@ k_piece_group(int npieces, const int32_t* __restrict__ piece_row, const int32_t*
     const int leader = row_head[row];
     const int at = atomicAdd(lead_n + leader, 1);
     if (at < kRowPieces) lead_ids[(long long)leader * kRowPieces + at] = pc;
+    // the leaders, in any order (every row is added up on its own): the gather walks this list only
+    if (pc == leader) lead_list[atomicAdd(lead_n + npieces, 1)] = pc;
 }
 
 // Gather: kGatherParts warps per output row, each a contiguous share of the channels.  Two
@@ -1247,33 +1250,35 @@ k_gather_rows(Geo g, const long long* __restrict__ vid_off, const int32_t* __res
     }
 }
 
-// Rows put together from pieces: kPieceParts warps per such row, found through its leader piece.
-// The pieces are added in the order of their index (a fixed order, so the result does not depend
-// on scheduling); such a row is bound by the latency of its loads, so four pieces' loads are issued
-// before anything is added.
+// Rows put together from pieces: kPieceParts warps per such row, the rows taken from the list of
+// leader pieces.  The pieces are added in the order of their index (a fixed order, so the result
+// does not depend on scheduling); such a row is bound by the latency of its dependent loads
+// (leader -> list -> data), so the grid holds as many warps as the GPU keeps resident and two pieces'
+// loads are issued before anything is added.
 constexpr int kPieceParts = 8;
 template <typename OutT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 k_gather_pieces(Geo g, int npieces, const int32_t* __restrict__ piece_row, const int32_t* __restrict__ lead_n,
-                const int32_t* __restrict__ lead_ids, const int32_t* __restrict__ row_weight,
-                const float* __restrict__ pieces, OutT* __restrict__ out, long long capacity) {
+                const int32_t* __restrict__ lead_ids, const int32_t* __restrict__ lead_list,
+                const int32_t* __restrict__ row_weight, const float* __restrict__ pieces, OutT* __restrict__ out,
+                long long capacity) {
     wait_for_prior_kernel();
     __shared__ int s_ids[8][2 * kRowPieces];
     const int lane = threadIdx.x & 31;
-    const long long nunits = (long long)npieces * kPieceParts;
+    const long long nunits = (long long)lead_n[npieces] * kPieceParts;
     const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
     const int nf4 = g.D / VEC;                                      // 4-channel groups of a row
     int* ids = s_ids[threadIdx.x >> 5];
     int* sorted = ids + kRowPieces;
     for (long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); unit < nunits; unit += nwarps) {
-        const int leader = (int)(unit / kPieceParts), part = (int)(unit % kPieceParts);
+        const int leader = lead_list[unit / kPieceParts], part = (int)(unit % kPieceParts);
         const int n_all = lead_n[leader];
-        if (n_all == 0) continue;                       // not a leader
         const long long r = piece_row[leader];
         if (r >= capacity) continue;
         const int n = min(n_all, kRowPieces);
         __syncwarp();
         for (int i = lane; i < n; i += 32) ids[i] = lead_ids[(long long)leader * kRowPieces + i];
+        const float wsum = (float)row_weight[r];
         __syncwarp();
         for (int i = lane; i < n; i += 32) {
             const int mine = ids[i];
@@ -1282,7 +1287,6 @@ k_gather_pieces(Geo g, int npieces, const int32_t* __restrict__ piece_row, const
             sorted[rank] = mine;
         }
         __syncwarp();
-        const float wsum = (float)row_weight[r];
         const int lo = (int)((long long)nf4 * part / kPieceParts), hi = (int)((long long)nf4 * (part + 1) / kPieceParts);
         for (int f0 = lo + lane; f0 < hi; f0 += 4 * 32) {
             float sum[4][VEC];
@@ -1291,10 +1295,10 @@ k_gather_pieces(Geo g, int npieces, const int32_t* __restrict__ piece_row, const
 #pragma unroll
                 for (int v = 0; v < VEC; v++) sum[u][v] = 0.f;
             if (n_all <= kRowPieces) {
-                for (int k0 = 0; k0 < n; k0 += 4) {
-                    float4 v[4][4];
+                for (int k0 = 0; k0 < n; k0 += 2) {
+                    float4 v[2][4];
 #pragma unroll
-                    for (int k = 0; k < 4; k++) {
+                    for (int k = 0; k < 2; k++) {
                         if (k0 + k < n) {
                             const float4* src = reinterpret_cast<const float4*>(pieces + (long long)sorted[k0 + k] * g.D);
 #pragma unroll
@@ -1303,7 +1307,7 @@ k_gather_pieces(Geo g, int npieces, const int32_t* __restrict__ piece_row, const
                         }
                     }
 #pragma unroll
-                    for (int k = 0; k < 4; k++) {
+                    for (int k = 0; k < 2; k++) {
                         if (k0 + k < n) {
 #pragma unroll
                             for (int u = 0; u < 4; u++)

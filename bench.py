@@ -229,7 +229,7 @@ def _spawned(rank, world, port, argv):
     args = parse_args()
     if args.selftest_spawn:
         return spawn_selftest(rank, world, port)
-    run_ours(args)
+    (run_segments if args.mode == "segments" else run_ours)(args)
 
 
 def spawn_ranks(args):
@@ -440,6 +440,110 @@ def run_ours(args):
     return 0
 
 
+def run_segments(args):
+    """`--mode segments`: ONE video cut into runs of consecutive frames, one run per rank
+    (segments.SegmentMerge + DistLink: every rank merges its frames with the last frame of the rank
+    before in front, then one message per cut travels from the last rank to the first).  The ranks'
+    rows and ids, put together, are checked against the merge of the whole video on rank 0's GPU."""
+    import torch
+    import torch.distributed as dist
+    from paper_2507_07990_b200 import binding, segments
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if "MASTER_ADDR" in os.environ:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        import socket
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % port, rank=0, world_size=1,
+                                device_id=torch.device("cuda", local))
+    lib = binding.load_library()
+    cfg, specs, ths, key = workload_setup(args.workload, args.budget)
+    if len(specs) != 1:
+        raise SystemExit("--mode segments cuts one video; workload %s holds %d" % (args.workload, len(specs)))
+    spec, th = specs[0], ths[0]
+    if spec.dtype != "bf16":
+        raise SystemExit("--mode segments runs the bf16 workloads")
+    HW = spec.H * spec.W
+    video = inputs.make_video(spec)                     # every rank generates the video and keeps its own frames
+    cuts = segments.cut_frames(spec.T, world)
+    a, b = cuts[rank], cuts[rank + 1]
+    halo = 1 if rank > 0 else 0
+    mine = torch.from_numpy(video[a - halo:b].view(np.int16)).view(torch.bfloat16).cuda()
+    part = segments.SegmentMerge(mine, bool(halo), a, th["tau_s"], th["tau_t"], out_dtype=torch.bfloat16)
+    link = segments.DistLink()
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    out = None
+    for _ in range(max(args.warmup, 3)):
+        part.merge_local()
+        out = part.finish(link)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        part.merge_local()
+        out = part.finish(link)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop() if sampler is not None else None
+    # kernels per step: the merge of the segment, of its halo frame, and the fold / emit / finish kernels
+    launches = args.steps * (part.res.launches + (part.halo.launches + 1 if halo else 0) + (1 if rank + 1 < world else 0) + 1)
+    total_ms = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device="cuda")
+    dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
+    total_ms = float(total_ms.item())
+    if int(out.device_status.item()) != 0:
+        raise RuntimeError("device status %d on rank %d" % (int(out.device_status.item()), rank))
+
+    # the packed result: counts and ids of every rank, in rank order
+    owned = torch.tensor([out.owned_count], dtype=torch.int64, device="cuda")
+    every = [torch.zeros_like(owned) for _ in range(world)]
+    dist.all_gather(every, owned)
+    counts = [int(c.item()) for c in every]
+    ids = torch.full((max(counts + [1]),), -1, dtype=torch.int32, device="cuda")
+    ids[:out.owned_count] = out.out_pos[:out.owned_count]
+    all_ids = [torch.empty_like(ids) for _ in range(world)]
+    dist.all_gather(all_ids, ids)
+    check = None
+    if rank == 0:
+        whole = torch.from_numpy(video.view(np.int16)).view(torch.bfloat16).cuda().unsqueeze(0)
+        plan = binding.MergePlan(tuple(whole.shape), torch.bfloat16, th["tau_s"], th["tau_t"], out_dtype=torch.bfloat16,
+                                 want_map=False)
+        ref = plan.run(whole)
+        n = int(ref.out_count[0].item())
+        got = torch.cat([t[:c] for t, c in zip(all_ids, counts)])
+        check = {"rows": sum(counts), "rows_single_gpu": n, "rows_calibrated": th["count"],
+                 "ids_equal": bool(got.numel() == n and torch.equal(got, ref.out_pos[:n]))}
+        if not (check["ids_equal"] and n == th["count"]):
+            raise RuntimeError("segments disagree with the whole video: %s" % check)
+        in_bytes = spec.tokens * spec.D * 2
+        line = {"metric": METRIC, "value": spec.tokens * args.steps / (total_ms / 1e3), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+                "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": dict(workload_config(args.workload, specs, ths, key), mode="segments",
+                               frames_per_rank=[cuts[r + 1] - cuts[r] for r in range(world)],
+                               message="per cut at most %d rows of %d fp32 sums, weights and ids, last rank first"
+                                       % (HW, spec.D)),
+                "out_rows": sum(counts), "rows_per_rank": counts, "check": check,
+                "roofline": None, "e2e": None, "gpu_launches": launches, "clocks": clocks,
+                "path": {"algorithmic_bytes": in_bytes + sum(counts) * (spec.D * 2 + 4),
+                         "achieved": (in_bytes + sum(counts) * (spec.D * 2 + 4)) / (total_ms / args.steps / 1e3) / 1e9}}
+        print(json.dumps(line))
+    dist.destroy_process_group()
+    return 0
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -462,6 +566,9 @@ def parse_args():
     ap.add_argument("--tuning", default="0,0,0",
                     help="path,cluster_size,frames_per_item for sttm_set_tuning (path 5: the two-stream kernels), "
                          "optionally followed by sum_slots,lead_frames for sttm_set_ring_split (0 = library's choice)")
+    ap.add_argument("--mode", default="videos", choices=["videos", "segments"],
+                    help="videos: every rank merges its own videos (the default); segments: one video cut by frames "
+                         "over the ranks, checked against the merge of the whole video")
     ap.add_argument("--selftest-spawn", action="store_true", help=argparse.SUPPRESS)
     return ap.parse_args()
 
@@ -472,7 +579,7 @@ def main():
         return run_reference(args)
     if "WORLD_SIZE" not in os.environ and (args.gpus > 1 or args.selftest_spawn):
         return spawn_ranks(args)
-    return run_ours(args)
+    return (run_segments if args.mode == "segments" else run_ours)(args)
 
 
 if __name__ == "__main__":

@@ -36,9 +36,9 @@
  *     c = t*H*W + y*W + x.  A quadtree node is named by the cell id of its top-left
  *     (anchor) cell.  Quadtrees of up to 3 levels (coarsest node at most 4 cells wide) run on
  *     the tuned kernels; deeper ones (up to 8 levels) only through sttm_merge_ex / sttm_merge /
- *     sttm_merge_host, on plain general kernels whose chain sums use floating-point atomics
- *     (last bits may differ between runs); the stage calls and the budget mode report them
- *     as STTM_ERR_UNSUPPORTED.
+ *     sttm_merge_host, on plain general kernels (same results, a row's members added in index
+ *     order, several times slower); the stage calls and the budget mode report them as
+ *     STTM_ERR_UNSUPPORTED.  On every path the output bits do not depend on scheduling.
  */
 #ifndef STTM_H
 #define STTM_H

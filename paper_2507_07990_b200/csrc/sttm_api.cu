@@ -107,7 +107,7 @@ struct Plan {
     FlowPlan fl;
     bool generic;             // more than three quadtree levels: the plain kernels of sttm_generic.cuh
     Pyr py;
-    size_t gen_pooled, gen_norms, gen_dots, gen_allpass, gen_acc;
+    size_t gen_pooled, gen_norms, gen_dots, gen_allpass, gen_cnt, gen_start, gen_list, gen_sorted;
     size_t norms_bytes;       // the spatial stage's only scratch: one squared norm per quadtree node
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
@@ -430,15 +430,18 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
     pl->partial = take((size_t)pl->partial_slots * g.D * sizeof(float));
     pl->f.ok = false;
     pl->fl.ok = false;
-    pl->gen_pooled = pl->gen_norms = pl->gen_dots = pl->gen_allpass = pl->gen_acc = o;
+    pl->gen_pooled = pl->gen_norms = pl->gen_dots = pl->gen_allpass = o;
+    pl->gen_cnt = pl->gen_start = pl->gen_list = pl->gen_sorted = o;
     if (pl->generic) {
         const long long frames = (long long)g.B * g.T;
-        const long long rows = std::min<long long>(pl->cells, std::max<long long>(p->out_capacity_rows, 1));
         pl->gen_pooled = take((size_t)frames * pl->py.upper * g.D * sizeof(float));
         pl->gen_norms = take((size_t)frames * pl->py.nodes * sizeof(float));
         pl->gen_dots = take((size_t)frames * pl->py.nodes * sizeof(float));
         pl->gen_allpass = take((size_t)frames * pl->py.nodes);
-        pl->gen_acc = take((size_t)rows * g.D * sizeof(float));
+        pl->gen_cnt = take((size_t)pl->cells * 4);
+        pl->gen_start = take(((size_t)pl->cells + 1) * 4);
+        pl->gen_list = take((size_t)pl->cells * 4);
+        pl->gen_sorted = take((size_t)pl->cells * 4);
     } else {
         plan_flow(p, g, &pl->fl, budget);
         if (!pl->fl.ok) plan_fused(p, g, &pl->f);
@@ -901,7 +904,10 @@ sttm_status run_generic(const T* feats, const sttm_params* p, const Plan& pl, ch
     float* norms = (float*)(ws + pl.gen_norms);
     float* dots = (float*)(ws + pl.gen_dots);
     int8_t* allpass = (int8_t*)(ws + pl.gen_allpass);
-    float* acc = (float*)(ws + pl.gen_acc);
+    int32_t* cnt = (int32_t*)(ws + pl.gen_cnt);
+    int32_t* start = (int32_t*)(ws + pl.gen_start);
+    int32_t* list = (int32_t*)(ws + pl.gen_list);
+    int32_t* sorted = (int32_t*)(ws + pl.gen_sorted);
     int8_t* cover = (int8_t*)(ws + pl.cover);
     int32_t* link = (int32_t*)(ws + pl.link);
     int32_t* root = (int32_t*)(ws + pl.root);
@@ -909,13 +915,12 @@ sttm_status run_generic(const T* feats, const sttm_params* p, const Plan& pl, ch
     const long long rows = std::min<long long>(pl.cells, std::max<long long>(p->out_capacity_rows, 1));
     sttm_status s;
     STTM_CUDA_TRY(cudaMemsetAsync(link, 0xff, (size_t)pl.cells * 4, st));
-    STTM_CUDA_TRY(cudaMemsetAsync(acc, 0, (size_t)rows * g.D * sizeof(float), st));
+    STTM_CUDA_TRY(cudaMemsetAsync(cnt, 0, (size_t)pl.cells * 4, st));
     for (int l = 1; l < py.L; l++) {
-        k_gen_pool<T><<<blocks_for(frames * py.H[l] * py.W[l] * 32, 256), 256, 0, st>>>(feats, pooled, g, py, l);
+        k_gen_pool<T><<<blocks_for(frames * py.H[l] * py.W[l] * 32, 256), 256, 0, st>>>(feats, pooled, g, py, l, norms,
+                                                                                       dots);
         if ((s = launched()) != STTM_OK) return s;
     }
-    k_gen_norm_dot<T><<<blocks_for(frames * py.nodes * 32, 256), 256, 0, st>>>(feats, pooled, g, py, norms, dots);
-    if ((s = launched()) != STTM_OK) return s;
     k_gen_allpass<<<blocks_for(frames * py.nodes, 256), 256, 0, st>>>(g, py, taus, norms, dots, allpass);
     if ((s = launched()) != STTM_OK) return s;
     k_gen_cover<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, py, allpass, cover);
@@ -951,13 +956,19 @@ sttm_status run_generic(const T* feats, const sttm_params* p, const Plan& pl, ch
                                                         (int32_t*)(ws + pl.row_weight),
                                                         (int32_t*)(ws + pl.row_last_t), (int)p->wt);
     if ((s = launched()) != STTM_OK) return s;
-    k_gen_accumulate<T><<<blocks_for(pl.cells * 32, 256), 256, 0, st>>>(feats, pooled, g, py, cover,
-                                                                       (const int32_t*)(ws + pl.cell_row), acc,
-                                                                       p->out_capacity_rows, (int)p->wt);
+    const long long cap = p->out_capacity_rows;
+    const int32_t* cell_row = (const int32_t*)(ws + pl.cell_row);
+    k_gen_count<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, cover, cell_row, cnt, cap);
     if ((s = launched()) != STTM_OK) return s;
-    k_gen_finish<OutT><<<blocks_for(rows * (g.D / VEC), 256), 256, 0, st>>>(g, vid_off, acc,
-                                                                           (const int32_t*)(ws + pl.row_weight),
-                                                                           out_feats, p->out_capacity_rows);
+    k_gen_scan_rows<<<1, 1024, 0, st>>>(g, vid_off, cap, cnt, start);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_fill<<<blocks_for(pl.cells, 256), 256, 0, st>>>(g, cover, cell_row, cnt, start, list, cap);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_sort<<<blocks_for(rows * 32, 256), 256, 0, st>>>(g, vid_off, cap, start, list, sorted);
+    if ((s = launched()) != STTM_OK) return s;
+    k_gen_gather<T, OutT><<<blocks_for(rows * kGenParts * 32, 256), 256, 0, st>>>(
+        feats, pooled, g, py, vid_off, cover, start, sorted, (const int32_t*)(ws + pl.row_weight), out_feats, cap,
+        (int)p->wt);
     return launched();
 }
 

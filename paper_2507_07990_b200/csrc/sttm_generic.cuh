@@ -1,7 +1,7 @@
 // General path for quadtrees of more than three levels (grids of more than 16 cells a side
 // with a 4x4 coarsest map, or the 2x2 coarsest map of the paper's ablation on a 13x13 / 14x14 /
 // 16x16 grid).  Plain kernels, one step of Section 3 each, pooled features kept in fp32 in the
-// workspace; nothing here is tuned: the fused kernel covers the shapes that matter for speed.
+// workspace; nothing here is tuned for speed: the fused kernel covers the shapes that matter there.
 #pragma once
 
 #include "sttm_device.cuh"
@@ -29,10 +29,13 @@ __device__ __forceinline__ void node4(const T* __restrict__ feats, const float* 
 }
 
 // Section 3.2: level l = 2x2 average pooling of level l - 1 (border parents average the children
-// that exist).  One warp per node of level l.
+// that exist).  One warp per node of level l; with the children in registers it also takes what the
+// search needs: the node's squared norm, every child's dot product with it and, at level 1, the
+// children's (the cells') squared norms.
 template <typename T>
 __global__ void __launch_bounds__(256)
-k_gen_pool(const T* __restrict__ feats, float* __restrict__ pooled, Geo g, Pyr py, int l) {
+k_gen_pool(const T* __restrict__ feats, float* __restrict__ pooled, Geo g, Pyr py, int l,
+           float* __restrict__ norms, float* __restrict__ dots) {
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     const int per = py.H[l] * py.W[l];
@@ -45,52 +48,48 @@ k_gen_pool(const T* __restrict__ feats, float* __restrict__ pooled, Geo g, Pyr p
             if (2 * i + a < py.H[l - 1] && 2 * j + b < py.W[l - 1]) child[n++] = (2 * i + a) * py.W[l - 1] + 2 * j + b;
     const float inv = 1.f / (float)n;
     float* dst = pooled + (bt * py.upper + py.uoff[l] + idx) * (long long)g.D;
+    float nn = 0.f, dp[4] = {0.f, 0.f, 0.f, 0.f}, cn[4] = {0.f, 0.f, 0.f, 0.f};
     for (int d = lane * VEC; d < g.D; d += 32 * VEC) {
         float s[VEC] = {0.f, 0.f, 0.f, 0.f};
-        for (int c = 0; c < n; c++) {
-            float x[VEC];
-            node4(feats, pooled, g, py, bt, l - 1, child[c], d, x);
+        float x[4][VEC];
 #pragma unroll
-            for (int v = 0; v < VEC; v++) s[v] += x[v];
+        for (int c = 0; c < 4; c++) {
+            if (c < n) {
+                node4(feats, pooled, g, py, bt, l - 1, child[c], d, x[c]);
+#pragma unroll
+                for (int v = 0; v < VEC; v++) s[v] += x[c][v];
+            }
         }
 #pragma unroll
         for (int v = 0; v < VEC; v++) s[v] *= inv;
         store4(dst + d, s);
-    }
-}
-
-// squared norm of every node and its dot product with its parent.  One warp per node.
-template <typename T>
-__global__ void __launch_bounds__(256)
-k_gen_norm_dot(const T* __restrict__ feats, const float* __restrict__ pooled, Geo g, Pyr py,
-               float* __restrict__ norms, float* __restrict__ dots) {
-    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (warp >= (long long)g.B * g.T * py.nodes) return;
-    const long long bt = warp / py.nodes;
-    const int node = (int)(warp % py.nodes);
-    int l = 0;
-    while (l + 1 < py.L && node >= py.noff[l + 1]) l++;
-    const int idx = node - py.noff[l], i = idx / py.W[l], j = idx % py.W[l];
-    const bool has_parent = l + 1 < py.L;
-    const int pidx = has_parent ? (i >> 1) * py.W[l + 1] + (j >> 1) : 0;
-    float nn = 0.f, dp = 0.f;
-    for (int d = lane * VEC; d < g.D; d += 32 * VEC) {
-        float x[VEC], q[VEC];
-        node4(feats, pooled, g, py, bt, l, idx, d, x);
 #pragma unroll
-        for (int v = 0; v < VEC; v++) nn = fmaf(x[v], x[v], nn);
-        if (has_parent) {
-            node4(feats, pooled, g, py, bt, l + 1, pidx, d, q);
+        for (int v = 0; v < VEC; v++) nn = fmaf(s[v], s[v], nn);
 #pragma unroll
-            for (int v = 0; v < VEC; v++) dp = fmaf(x[v], q[v], dp);
+        for (int c = 0; c < 4; c++) {
+            if (c < n) {
+#pragma unroll
+                for (int v = 0; v < VEC; v++) {
+                    dp[c] = fmaf(x[c][v], s[v], dp[c]);
+                    cn[c] = fmaf(x[c][v], x[c][v], cn[c]);
+                }
+            }
         }
     }
     nn = warp_sum(nn);
-    dp = warp_sum(dp);
+#pragma unroll
+    for (int c = 0; c < 4; c++) { dp[c] = warp_sum(dp[c]); cn[c] = warp_sum(cn[c]); }
     if (lane == 0) {
-        norms[bt * py.nodes + node] = nn;
-        dots[bt * py.nodes + node] = dp;
+        const long long at = bt * py.nodes;
+        norms[at + py.noff[l] + idx] = nn;
+        if (l + 1 == py.L) dots[at + py.noff[l] + idx] = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; c++) {
+            if (c < n) {
+                dots[at + py.noff[l - 1] + child[c]] = dp[c];
+                if (l == 1) norms[at + child[c]] = cn[c];
+            }
+        }
     }
 }
 
@@ -213,47 +212,124 @@ k_gen_root_fill(Geo g, const int8_t* __restrict__ cover, int32_t* root) {
     root[i0] = root[i0 / g.N * g.N + t * g.HW + (y & ~m) * g.W + (x & ~m)];
 }
 
-// Section 3.3, merge: every kept node adds its weighted feature to its row (fp32 atomics: the
-// order of the additions, hence the last bits, may differ from run to run), then one division.
-template <typename T>
+// Section 3.3, merge.  Every output row gets the list of its kept nodes (counted, placed by a prefix
+// sum over the rows, put into index order), then kGenParts warps per row add the weighted features
+// in that order and divide once: the sums do not depend on scheduling.
+__device__ __forceinline__ bool gen_kept_anchor(const Geo& g, long long i0, int lv) {
+    const int cell = (int)(i0 % g.HW), y0 = cell / g.W, x0 = cell % g.W, m = (1 << lv) - 1;
+    return ((y0 & m) | (x0 & m)) == 0;
+}
 __global__ void __launch_bounds__(256)
-k_gen_accumulate(const T* __restrict__ feats, const float* __restrict__ pooled, Geo g, Pyr py,
-                 const int8_t* __restrict__ cover, const int32_t* __restrict__ cell_row, float* __restrict__ acc,
-                 long long capacity, int weight_mode) {
-    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (warp >= (long long)g.B * g.N) return;
-    const long long bt = warp / g.HW;
-    const int cell = (int)(warp % g.HW), y0 = cell / g.W, x0 = cell % g.W;
-    const int lv = cover[warp], m = (1 << lv) - 1;
-    if (((y0 & m) | (x0 & m)) != 0) return;
-    const long long row = cell_row[warp];
+k_gen_count(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__ cell_row, int32_t* __restrict__ cnt,
+            long long capacity) {
+    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i0 >= (long long)g.B * g.N || !gen_kept_anchor(g, i0, cover[i0])) return;
+    const long long row = cell_row[i0];
+    if (row < capacity) atomicAdd(cnt + row, 1);
+}
+// one block: start[r] = number of list entries before row r, start[rows] = their total
+__global__ void __launch_bounds__(1024)
+k_gen_scan_rows(Geo g, const long long* __restrict__ vid_off, long long capacity, const int32_t* __restrict__ cnt,
+                int32_t* __restrict__ start) {
+    __shared__ int sm[33];
+    const long long rows = min(vid_off[g.B], capacity);
+    int carry = 0;
+    for (long long r0 = 0; r0 < rows; r0 += blockDim.x) {
+        const long long r = r0 + threadIdx.x;
+        const int v = r < rows ? cnt[r] : 0;
+        int total;
+        const int ex = block_exclusive_scan(v, total, sm);
+        if (r < rows) start[r] = carry + ex;
+        carry += total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) start[rows] = carry;
+}
+// (the counts are used up as cursors: a row's entries land in any order and are put in order next)
+__global__ void __launch_bounds__(256)
+k_gen_fill(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__ cell_row, int32_t* __restrict__ cnt,
+           const int32_t* __restrict__ start, int32_t* __restrict__ list, long long capacity) {
+    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i0 >= (long long)g.B * g.N || !gen_kept_anchor(g, i0, cover[i0])) return;
+    const long long row = cell_row[i0];
     if (row >= capacity) return;
-    const float w = weight_mode ? (float)(min(1 << lv, g.H - y0) * min(1 << lv, g.W - x0)) : 1.f;
-    const int vidx = (y0 >> lv) * py.W[lv] + (x0 >> lv);
-    for (int d = lane * VEC; d < g.D; d += 32 * VEC) {
-        float x[VEC];
-        node4(feats, pooled, g, py, bt, lv, vidx, d, x);
-#pragma unroll
-        for (int v = 0; v < VEC; v++) atomicAdd(acc + row * g.D + d + v, w * x[v]);
+    const int at = atomicSub(cnt + row, 1) - 1;
+    list[start[row] + at] = (int32_t)i0;
+}
+// one warp per row: its entries in increasing order (rank by counting; rows are short)
+__global__ void __launch_bounds__(256)
+k_gen_sort(Geo g, const long long* __restrict__ vid_off, long long capacity, const int32_t* __restrict__ start,
+           const int32_t* __restrict__ list, int32_t* __restrict__ sorted) {
+    const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= min(vid_off[g.B], capacity)) return;
+    const int base = start[row], n = start[row + 1] - base;
+    for (int i = lane; i < n; i += 32) {
+        const int mine = list[base + i];
+        int rank = 0;
+        for (int k = 0; k < n; k++) rank += list[base + k] < mine ? 1 : 0;
+        sorted[base + rank] = mine;
     }
 }
-template <typename OutT>
+constexpr int kGenParts = 8;
+template <typename T, typename OutT>
 __global__ void __launch_bounds__(256)
-k_gen_finish(Geo g, const long long* __restrict__ vid_off, const float* __restrict__ acc,
-             const int32_t* __restrict__ row_weight, OutT* __restrict__ out, long long capacity) {
-    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long rows = min(vid_off[g.B], capacity);
-    const int per = g.D / VEC;
-    if (i0 >= rows * per) return;
-    const long long row = i0 / per;
-    const int d = (int)(i0 % per) * VEC;
+k_gen_gather(const T* __restrict__ feats, const float* __restrict__ pooled, Geo g, Pyr py,
+             const long long* __restrict__ vid_off, const int8_t* __restrict__ cover,
+             const int32_t* __restrict__ start, const int32_t* __restrict__ sorted,
+             const int32_t* __restrict__ row_weight, OutT* __restrict__ out, long long capacity, int weight_mode) {
+    const long long unit = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const long long row = unit / kGenParts;
+    const int part = (int)(unit % kGenParts);
+    if (row >= min(vid_off[g.B], capacity)) return;
+    const int base = start[row], n = start[row + 1] - base;
     const float inv = 1.f / (float)row_weight[row];
-    float x[VEC];
-    load4(acc + row * g.D + d, x);
+    const int nf4 = g.D / VEC;
+    const int lo = (int)((long long)nf4 * part / kGenParts), hi = (int)((long long)nf4 * (part + 1) / kGenParts);
+    for (int f0 = lo + lane; f0 < hi; f0 += 4 * 32) {
+        float sum[4][VEC];
 #pragma unroll
-    for (int v = 0; v < VEC; v++) x[v] *= inv;
-    store4(out + row * g.D + d, x);
+        for (int u = 0; u < 4; u++)
+#pragma unroll
+            for (int v = 0; v < VEC; v++) sum[u][v] = 0.f;
+        // two members' loads are issued before anything is added; the additions keep the list's order
+        for (int k0 = 0; k0 < n; k0 += 2) {
+            float x[2][4][VEC], w[2];
+#pragma unroll
+            for (int k = 0; k < 2; k++) {
+                if (k0 + k < n) {
+                    const long long i0 = sorted[base + k0 + k];
+                    const long long bt = i0 / g.HW;
+                    const int cell = (int)(i0 % g.HW), y0 = cell / g.W, x0 = cell % g.W;
+                    const int lv = cover[i0];
+                    w[k] = weight_mode ? (float)(min(1 << lv, g.H - y0) * min(1 << lv, g.W - x0)) : 1.f;
+                    const int vidx = (y0 >> lv) * py.W[lv] + (x0 >> lv);
+#pragma unroll
+                    for (int u = 0; u < 4; u++)
+                        if (f0 + u * 32 < hi) node4(feats, pooled, g, py, bt, lv, vidx, (f0 + u * 32) * VEC, x[k][u]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 2; k++) {
+                if (k0 + k < n) {
+#pragma unroll
+                    for (int u = 0; u < 4; u++)
+                        if (f0 + u * 32 < hi) {
+#pragma unroll
+                            for (int v = 0; v < VEC; v++) sum[u][v] = fmaf(w[k], x[k][u][v], sum[u][v]);
+                        }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; u++)
+            if (f0 + u * 32 < hi) {
+#pragma unroll
+                for (int v = 0; v < VEC; v++) sum[u][v] *= inv;
+                store4(out + row * g.D + (long long)(f0 + u * 32) * VEC, sum[u]);
+            }
+    }
 }
 
 }  // namespace sttm

@@ -388,6 +388,21 @@ def test_deeper_quadtrees(shape):
     assert done >= 1, "no seed gave thresholds with a margin"
 
 
+def test_deeper_quadtrees_features_do_not_depend_on_scheduling():
+    """The general kernels add a row's members in index order: two runs give the same bits."""
+    spec = helpers.small_spec(871, 24, 13, 13, 256, dtype="bf16", sigma=0.05, depth_max=4, p_static=0.9)
+    dev = helpers.to_torch(inputs.make_video(spec)[None])
+    outs = []
+    for _ in range(3):
+        out = binding.sttm_merge_ex(dev, 0.6, 0.6, lv1=2, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        assert int(out.device_status.item()) == 0 and binding.load_library().sttm_last_path() == 2
+        n = int(out.out_count[0])
+        outs.append(out.out_feats[:n].clone())
+    assert n < spec.tokens                       # something was merged
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+
+
 def test_deeper_quadtrees_batch_capacity_and_host_entry():
     specs = [helpers.small_spec(840 + v, 5, 18, 20, 64, dtype="bf16", sigma=0.3, depth_max=4, p_static=p)
              for v, p in enumerate((0.9, 0.4))]

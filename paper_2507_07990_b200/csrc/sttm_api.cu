@@ -112,7 +112,7 @@ struct Plan {
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
         frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
-        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_row, lead_n, lead_ids, lead_list, flow_partial,
+        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_row, lead_n, lead_ids, lead_list, flow_progress, flow_partial,
         flow_hand, flow_recs, total;
 };
 
@@ -448,11 +448,12 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
     }
     pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = o;
     pl->piece_row = pl->lead_n = pl->lead_ids = pl->lead_list = o;
-    pl->flow_partial = pl->flow_hand = pl->flow_recs = o;
+    pl->flow_partial = pl->flow_hand = pl->flow_recs = pl->flow_progress = o;
     if (pl->fl.ok) {
         const FlowPlan& f = pl->fl;
         pl->ones_begin = o;
         pl->row_head = take((size_t)pl->cells * 4);
+        pl->flow_progress = take((size_t)f.nitems * 4);
         pl->ones_end = o;
         pl->pieces = take((size_t)f.nitems * kPieceSlots * g.D * sizeof(float));
         pl->piece_meta = take((size_t)f.nitems * kPieceSlots * sizeof(int2));
@@ -822,6 +823,7 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     fp.partial = (float*)(ws + pl.flow_partial);
     fp.hand = (int32_t*)(ws + pl.flow_hand);
     fp.recs = (FrameRec*)(ws + pl.flow_recs);
+    fp.progress = (int32_t*)(ws + pl.flow_progress);
     fp.row_at_root = (const int32_t*)(ws + pl.row_at_root);
     fp.vid_off = (const long long*)(ws + pl.vid_off);
     fp.out = out_feats;

@@ -62,6 +62,18 @@ struct Col {
 // (its blocks may become resident while the kernel before it in the stream still runs): waits
 // until that kernel has completed and its writes are visible.  Returns at once otherwise.
 __device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the kernel launched after this one (with the same attribute) become resident now instead of
+// when this kernel ends.  That kernel still sees this one's writes only after its own
+// wait_for_prior_kernel(), or through flags written with store_release() and read with load_acquire().
+__device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void store_release(int32_t* p, int32_t v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int32_t load_acquire(const int32_t* p) {
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -62,6 +62,7 @@ struct FlowParams {
     float* partial;          // [nitems][F+1][NS][128]: the Gram stage's numbers, [number][cell]
     int32_t* hand;           // [nitems][F+1][16]: cover level | (link lane + 1) << 8 of every tile row
     FrameRec* recs;          // [nitems][F+2]: the chain stage's records, one per frame and a closing one
+    int32_t* progress;       // [nitems]: index of the last record the chain stage has written (-1: none yet)
     const int32_t* row_at_root;   // [B*N] row (inside its video) of every surviving token
     const long long* vid_off;     // [B+1] first row of every video
     void* out;               // [rows][D] output rows
@@ -282,6 +283,9 @@ constexpr int kChainWarps = 4;
 __global__ void __launch_bounds__(kChainWarps * 32)
 k_flow_chain(const __grid_constant__ FlowParams p) {
     wait_for_prior_kernel();
+    // The sum stage may become resident now: it takes a frame's record only after this kernel has
+    // published it (`progress`), so its stream of features starts while the records are still written.
+    let_next_kernel_start();
     __shared__ __align__(16) FrameRec s_rec[kChainWarps];
     __shared__ SlotTable s_tab[kChainWarps];
     const unsigned full = 0xffffffffu;
@@ -301,15 +305,16 @@ k_flow_chain(const __grid_constant__ FlowParams p) {
     const int32_t* hand = p.hand + (long long)it.item * (p.F + 1) * 16;
     int prev_slot = 0;
     uint32_t active_slots = 0;
-    // (the next frame's decisions and row numbers are fetched while this frame is worked on)
-    int packed_next = hand[c];
-    int row_next = valid ? p.row_at_root[(long long)it.b * p.N + (long long)it.tstart * p.HW + lg.cell] : -1;
+    // The run's decisions and row numbers, fetched at once: the frames are worked on one after the other,
+    // and a load per frame would put the memory's latency (long while the sum stage streams) into every step.
+    __shared__ int32_t s_hand[kChainWarps][(kFlowMaxF + 1) * 16], s_rows[kChainWarps][(kFlowMaxF + 1) * 16];
+    for (int i = lane; i < it.n * 16; i += 32) {
+        s_hand[wib][i] = hand[i];
+        s_rows[wib][i] = valid ? p.row_at_root[(long long)it.b * p.N + (long long)(it.tstart + (i >> 4)) * p.HW + lg.cell] : -1;
+    }
+    __syncwarp();
     for (int j = 0; j <= it.n; j++) {
-        const int packed = packed_next, my_row = row_next;
-        if (j + 1 < it.n) {
-            packed_next = hand[(j + 1) * 16 + c];
-            row_next = valid ? p.row_at_root[(long long)it.b * p.N + (long long)(it.tstart + j + 1) * p.HW + lg.cell] : -1;
-        }
+        const int packed = j < it.n ? s_hand[wib][j * 16 + c] : 0, my_row = j < it.n ? s_rows[wib][j * 16 + c] : -1;
         if (j == it.n) {
             // Closing record: everything still running is written out.  A chain goes on into the next
             // item iff a node of that item's first frame is linked to its node of this frame; the
@@ -403,6 +408,8 @@ k_flow_chain(const __grid_constant__ FlowParams p) {
             for (int i = lane; i < kRecBytes / 16; i += 32) d4[i] = src[i];
         }
         __syncwarp();
+        // (published every eighth record and at the end: the release costs about as much as a record)
+        if (lane == 0 && ((j & 7) == 7 || j == it.n)) store_release(p.progress + it.item, j);
     }
 }
 
@@ -450,7 +457,7 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if constexpr (kSum) wait_for_prior_kernel();
+    // (the sum stage does not wait for the chain stage as a whole: its producer waits per record)
 
     bool timed_out = false;
     int q = 0;                      // slots used so far by this CTA's tasks: slot q % R, filled q / R times before
@@ -630,10 +637,26 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
             const int slice = tk % p.NS;
             const TileBox bx = p.boxes[it.tile];
             const int nslots = it.n + (kSum ? 1 : 0);
+            int seen = -1;
             for (int j = 0; j < nslots; j++, q++) {
                 const int s = q % p.R;
                 const uint32_t bar = full_bar + 8 * s;
                 if (q >= p.R && !mbar_wait_warp(empty_bar + 8 * s, q / p.R - 1, timed_out)) break;
+                if (kSum && seen < j) {
+                    // the record of this frame exists?  (bounded like every wait; the chain stage's blocks
+                    // are all resident before this kernel's first block is)
+                    bool late = false;
+                    if (lane == 0) {
+                        const unsigned long long t0 = global_timer_ns();
+                        while ((seen = load_acquire(p.progress + it.item)) < j) {
+                            __nanosleep(100);
+                            if (global_timer_ns() - t0 > kWaitLimitNs) { late = true; break; }
+                        }
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                    }
+                    seen = __shfl_sync(0xffffffffu, seen, 0);
+                    if (__any_sync(0xffffffffu, late)) { timed_out = true; break; }
+                }
                 if (lane == 0) {
                     const bool frame = j < it.n;
                     mbar_expect_tx(bar, (uint32_t)((frame ? p.slot_bytes : 0) + (kSum ? kRecBytes : 0)));

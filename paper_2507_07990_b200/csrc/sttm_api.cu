@@ -112,7 +112,7 @@ struct Plan {
     // byte offsets into the workspace
     size_t norms, cover, link, root, row_at_root, cell_row, row_anchor, span_off, frame_roots,
         frame_base, vid_off, zero_begin, frame_counts, row_weight, row_last_t, span_total, status, queue,
-        zero_end, partial, ones_begin, row_head, ones_end, staging, pieces, piece_meta, piece_row, lead_n, lead_ids, lead_list, flow_progress, flow_partial,
+        zero_end, partial, row_head, staging, pieces, piece_meta, piece_row, lead_n, lead_ids, lead_list, flow_progress, flow_partial,
         flow_hand, flow_recs, total;
 };
 
@@ -419,6 +419,14 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
     pl->frame_roots = take((size_t)g.B * g.T * 4);
     pl->frame_base = take((size_t)g.B * g.T * 4);
     pl->vid_off = take((size_t)(g.B + 1) * 8);
+    pl->f.ok = false;
+    pl->fl.ok = false;
+    if (!pl->generic) {
+        plan_flow(p, g, &pl->fl, budget);
+        if (!pl->fl.ok) plan_fused(p, g, &pl->f);
+    }
+    const bool tiled = pl->fl.ok || pl->f.ok;
+    // (one memset per call: everything that starts from zero lies together)
     pl->zero_begin = o;
     pl->frame_counts = take((size_t)g.B * g.T * 4);
     pl->row_weight = take((size_t)pl->cells * 4);
@@ -426,10 +434,11 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
     pl->span_total = take(4);
     pl->status = take(4);
     pl->queue = take(4);
+    pl->row_head = pl->flow_progress = o;
+    if (tiled) pl->row_head = take((size_t)pl->cells * 4);
+    if (pl->fl.ok) pl->flow_progress = take((size_t)pl->fl.nitems * 4);
     pl->zero_end = o;
-    pl->partial = take((size_t)pl->partial_slots * g.D * sizeof(float));
-    pl->f.ok = false;
-    pl->fl.ok = false;
+    pl->partial = take(tiled ? 0 : (size_t)pl->partial_slots * g.D * sizeof(float));
     pl->gen_pooled = pl->gen_norms = pl->gen_dots = pl->gen_allpass = o;
     pl->gen_cnt = pl->gen_start = pl->gen_list = pl->gen_sorted = o;
     if (pl->generic) {
@@ -442,19 +451,12 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         pl->gen_start = take(((size_t)pl->cells + 1) * 4);
         pl->gen_list = take((size_t)pl->cells * 4);
         pl->gen_sorted = take((size_t)pl->cells * 4);
-    } else {
-        plan_flow(p, g, &pl->fl, budget);
-        if (!pl->fl.ok) plan_fused(p, g, &pl->f);
     }
-    pl->ones_begin = pl->ones_end = pl->row_head = pl->staging = pl->pieces = pl->piece_meta = o;
+    pl->staging = pl->pieces = pl->piece_meta = o;
     pl->piece_row = pl->lead_n = pl->lead_ids = pl->lead_list = o;
-    pl->flow_partial = pl->flow_hand = pl->flow_recs = pl->flow_progress = o;
+    pl->flow_partial = pl->flow_hand = pl->flow_recs = o;
     if (pl->fl.ok) {
         const FlowPlan& f = pl->fl;
-        pl->ones_begin = o;
-        pl->row_head = take((size_t)pl->cells * 4);
-        pl->flow_progress = take((size_t)f.nitems * 4);
-        pl->ones_end = o;
         pl->pieces = take((size_t)f.nitems * kPieceSlots * g.D * sizeof(float));
         pl->piece_meta = take((size_t)f.nitems * kPieceSlots * sizeof(int2));
         pl->piece_row = take((size_t)f.nitems * kPieceSlots * 4);
@@ -467,9 +469,6 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
     }
     if (pl->f.ok) {
         const size_t out_elt = p->out_dtype == STTM_BF16 ? 2 : 4;
-        pl->ones_begin = o;
-        pl->row_head = take((size_t)pl->cells * 4);
-        pl->ones_end = o;
         pl->staging = take((size_t)pl->cells * g.D * out_elt);
         pl->pieces = take((size_t)pl->f.nitems * kPieceSlots * g.D * sizeof(float));
         pl->piece_meta = take((size_t)pl->f.nitems * kPieceSlots * sizeof(int2));
@@ -1204,12 +1203,10 @@ sttm_status merge_impl(const void* feats, const sttm_params* p, void* ws_, size_
         return s;
     }
     if (pl.fl.ok) {
-        STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.ones_begin, 0xff, pl.ones_end - pl.ones_begin, st));
         return run_flow(feats, p, pl, ws, out_feats, out_pos, merge_map, out_count, out_offsets, device_status, in, st);
     }
     if (pl.f.ok) {
         // single-read path: fused kernel, roots, ordering, gather
-        STTM_CUDA_TRY(cudaMemsetAsync(ws + pl.ones_begin, 0xff, pl.ones_end - pl.ones_begin, st));
         mark_stage(0, st);
         s = run_fused(feats, p, pl, ws, device_status, in, st);
         if (s != STTM_OK) return s;

@@ -62,7 +62,7 @@ struct FlowParams {
     float* partial;          // [nitems][F+1][NS][128]: the Gram stage's numbers, [number][cell]
     int32_t* hand;           // [nitems][F+1][16]: cover level | (link lane + 1) << 8 of every tile row
     FrameRec* recs;          // [nitems][F+2]: the chain stage's records, one per frame and a closing one
-    int32_t* progress;       // [nitems]: index of the last record the chain stage has written (-1: none yet)
+    int32_t* progress;       // [nitems]: number of records the chain stage has published (zero before the call)
     const int32_t* row_at_root;   // [B*N] row (inside its video) of every surviving token
     const long long* vid_off;     // [B+1] first row of every video
     void* out;               // [rows][D] output rows
@@ -409,7 +409,7 @@ k_flow_chain(const __grid_constant__ FlowParams p) {
         }
         __syncwarp();
         // (published every eighth record and at the end: the release costs about as much as a record)
-        if (lane == 0 && ((j & 7) == 7 || j == it.n)) store_release(p.progress + it.item, j);
+        if (lane == 0 && ((j & 7) == 7 || j == it.n)) store_release(p.progress + it.item, j + 1);
     }
 }
 
@@ -637,18 +637,18 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
             const int slice = tk % p.NS;
             const TileBox bx = p.boxes[it.tile];
             const int nslots = it.n + (kSum ? 1 : 0);
-            int seen = -1;
+            int seen = 0;                               // records of this run known to exist
             for (int j = 0; j < nslots; j++, q++) {
                 const int s = q % p.R;
                 const uint32_t bar = full_bar + 8 * s;
                 if (q >= p.R && !mbar_wait_warp(empty_bar + 8 * s, q / p.R - 1, timed_out)) break;
-                if (kSum && seen < j) {
+                if (kSum && seen <= j) {
                     // the record of this frame exists?  (bounded like every wait; the chain stage's blocks
                     // are all resident before this kernel's first block is)
                     bool late = false;
                     if (lane == 0) {
                         const unsigned long long t0 = global_timer_ns();
-                        while ((seen = load_acquire(p.progress + it.item)) < j) {
+                        while ((seen = load_acquire(p.progress + it.item)) <= j) {
                             __nanosleep(100);
                             if (global_timer_ns() - t0 > kWaitLimitNs) { late = true; break; }
                         }

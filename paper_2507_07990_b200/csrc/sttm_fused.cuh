@@ -1172,7 +1172,7 @@ k_piece_link(Geo g, int npieces, int max_hops, const int2* __restrict__ piece_me
     }
     const long long row = vid_off[b] + row_at_root[vb + r];
     piece_row[pc] = (int32_t)row;
-    atomicMin(reinterpret_cast<unsigned int*>(row_head) + row, (unsigned int)pc);      // (no leader yet: all bits set)
+    atomicMax(row_head + row, npieces - pc);           // (0: no piece yet; the smallest index gives the largest entry)
     atomicAdd(row_weight + row, m.y);
 }
 
@@ -1184,7 +1184,7 @@ k_piece_group(int npieces, const int32_t* __restrict__ piece_row, const int32_t*
     if (pc >= npieces) return;
     const int row = piece_row[pc];
     if (row < 0) return;
-    const int leader = row_head[row];
+    const int leader = npieces - row_head[row];
     const int at = atomicAdd(lead_n + leader, 1);
     if (at < kRowPieces) lead_ids[(long long)leader * kRowPieces + at] = pc;
     // the leaders, in any order (every row is added up on its own): the gather walks this list only
@@ -1212,7 +1212,7 @@ k_gather_rows(Geo g, const long long* __restrict__ vid_off, const int32_t* __res
     for (long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); unit < nunits; unit += nwarps) {
         const long long r = unit / kGatherParts;
         const int part = (int)(unit % kGatherParts);
-        if (row_head[r] >= 0) continue;                 // a row of pieces
+        if (row_head[r] != 0) continue;                 // a row of pieces
         int b = 0;                                      // video of the row: vid_off is short, walk it
         while (b + 1 < g.B && vid_off[b + 1] <= r) b++;
         const long long src = (long long)b * g.N + row_anchor[r];

@@ -253,6 +253,39 @@ def test_other_workload_shapes_full_width(shape, path):
     assert done >= 1, "no seed gave thresholds with a margin"
 
 
+@pytest.mark.parametrize("path", [1, 3], ids=["singlepass", "twostream"])
+def test_many_frames_take_the_separate_count_scan(path):
+    """More than 4096 frames in a call: the per-frame root counts are scanned by a kernel of their
+    own instead of inside the row kernel; two videos, so that the video offsets are in play."""
+    lib = binding.load_library()
+    T, H, W, D = 2100, 5, 5, 256
+    videos, taus, refs = [], [], []
+    for v in range(2):
+        for seed in range(4):
+            spec = helpers.small_spec(930 + 10 * v + seed, T, H, W, D, sigma=0.05, p_static=0.8)
+            video = inputs.make_video(spec)
+            t = helpers.safe_thresholds(video, 0.5, 0.5)
+            if t is not None:
+                break
+        assert t is not None, "no seed gave thresholds with a margin"
+        videos.append(video); taus.append(t); refs.append(oracle.merge(video, t[0], t[1]))
+    dev = helpers.to_torch(np.stack(videos))
+    lib.sttm_set_tuning(5 if path == 3 else 0, 0, 0)
+    try:
+        out = binding.sttm_merge_ex(dev, [t[0] for t in taus], [t[1] for t in taus], out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        assert lib.sttm_last_path() == path
+    finally:
+        lib.sttm_set_tuning(0, 0, 0)
+    assert int(out.device_status.item()) == 0
+    offs = out.out_offsets.tolist()
+    for b, ref in enumerate(refs):
+        assert int(out.out_count[b]) == ref.count and offs[b + 1] - offs[b] == ref.count
+        np.testing.assert_array_equal(out.merge_map[b].cpu().numpy(), ref.merge_map)
+        np.testing.assert_array_equal(out.out_pos[offs[b]:offs[b + 1]].cpu().numpy(), ref.out_pos)
+        helpers.assert_features_close(out.out_feats[offs[b]:offs[b + 1]].cpu().numpy(), ref.out_feats, False)
+
+
 def test_most_similar_destination(tuning):
     """Section 3.3's other destination rule: among the overlapping nodes above tau_t the most
     similar one instead of the top-left one.  Both sides pick a maximum, so the inputs are

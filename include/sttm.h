@@ -314,7 +314,8 @@ void sttm_set_stage_events(void** events);
  *                    wherever it applies (bf16 input, D a multiple of 16, at most 64 tiles of
  *                    4x4 cells per frame, D / cluster_size <= 1024), 3: the same without
  *                    packing the partial border tiles of a frame together, 5: the two-stream
- *                    kernels wherever they apply (bf16 input, D a multiple of 64)
+ *                    kernels wherever they apply (bf16 input, D a multiple of 64), 6: the same
+ *                    with the Gram stage on mma.sync instead of tcgen05
  *   cluster_size     single-pass kernel: CTAs that share one tile's channels (1, 2, 4 or 8)
  *   frames_per_item  frames of one tile that are processed in a row (two-stream kernels: at most 64)
  * Not thread safe; affects later calls of every entry point.

@@ -15,6 +15,7 @@
 #include "sttm_fused.cuh"
 #include "sttm_flow.cuh"
 #include "sttm_generic.cuh"
+#include "sttm_gram_tc.cuh"
 #include "sttm_segments.cuh"
 
 namespace {
@@ -93,7 +94,9 @@ struct FusedPlan {
 struct FlowPlan {
     bool ok;
     int NS, NB, R, slot_bytes, F, nseg, nitems, ntiles;
-    size_t smem;
+    int NSg, NBg;                   // slices and blocks per slice of the Gram stage
+    bool tc;                        // Gram stage on tcgen05 (else on mma.sync, with the sum stage's slices)
+    size_t smem, smem_tc;
     TileDesc tiles[kMaxTiles];
     TileBox boxes[kMaxTiles];
 };
@@ -243,7 +246,7 @@ void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
     // large inputs: measured on B200, the two-stream kernels overtake the single-pass kernel between
     // 0.25 GB (qwen: 0.23 against 0.21 ms) and 1.2 GB (long: 0.68 against 0.71 ms) of features.
     const bool large = (double)g.B * g.N * g.D * 2.0 >= kFlowMinBytes;
-    if (!(g_tune_path == 5 || (g_tune_path == 0 && (budget || large)))) return;
+    if (!(g_tune_path == 5 || g_tune_path == 6 || (g_tune_path == 0 && (budget || large)))) return;
     if (p->in_dtype != STTM_BF16 || g.D % 64 != 0) return;
     if (!build_flow_tiles(g, f)) return;
     const int nblk = g.D / 64;
@@ -284,6 +287,23 @@ void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
     }
     f->nseg = (g.T + f->F - 1) / f->F;
     f->nitems = g.B * f->ntiles * f->nseg;
+    // Gram stage on tcgen05: slices of up to seven blocks (a ring slot holds five frames of a slice)
+    f->tc = g_tune_path != 6;
+    f->NBg = f->NB;
+    f->NSg = f->NS;
+    f->smem_tc = 0;
+    if (f->tc) {
+        int nb = 0;
+        for (int n = std::min(nblk, kTcMaxNB); n >= 1 && nb == 0; n--)
+            if (nblk % n == 0) nb = n;
+        if (nblk / nb > 64) {
+            f->tc = false;
+        } else {
+            f->NBg = nb;
+            f->NSg = nblk / nb;
+            f->smem_tc = tc_smem_bytes(nb);
+        }
+    }
     f->ok = true;
 }
 
@@ -463,7 +483,7 @@ sttm_status make_plan(const sttm_params* p, Plan* pl, bool budget = false) {
         pl->lead_n = take(((size_t)f.nitems * kPieceSlots + 1) * 4);
         pl->lead_list = take((size_t)f.nitems * kPieceSlots * 4);
         pl->lead_ids = take((size_t)f.nitems * kPieceSlots * kRowPieces * 4);
-        pl->flow_partial = take((size_t)f.nitems * (f.F + 1) * f.NS * kSumVals * sizeof(float));
+        pl->flow_partial = take((size_t)f.nitems * (f.F + 1) * f.NSg * kSumVals * sizeof(float));
         pl->flow_hand = take((size_t)f.nitems * (f.F + 1) * 16 * 4);
         pl->flow_recs = take((size_t)f.nitems * (f.F + 2) * sizeof(FrameRec));
     }
@@ -786,6 +806,32 @@ sttm_status make_flow_maps(const void* feats, const Geo& g, int NB, FlowMaps* ma
     return STTM_OK;
 }
 
+// The same tensor with the frame axis inside the block axis: a box of five frames and NB blocks lands as
+// [block][frame][cell][64 channels], 80 rows of 128 bytes per block (the operand layout of k_flow_gram_tc).
+sttm_status make_gram_tc_maps(const void* feats, const Geo& g, int NB, FlowMaps* maps) {
+    static EncodeTiledFn encode = nullptr;
+    if (encode == nullptr) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || fn == nullptr)
+            return STTM_ERR_CUDA;
+        encode = (EncodeTiledFn)fn;
+    }
+    const cuuint64_t dims[5] = {64, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B * g.T, (cuuint64_t)(g.D / 64)};
+    const cuuint64_t strides[4] = {(cuuint64_t)g.D * 2, (cuuint64_t)g.W * g.D * 2, (cuuint64_t)g.HW * g.D * 2, 128};
+    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    const cuuint32_t fr = kTcBoxFrames;
+    const cuuint32_t boxes[3][5] = {{64, 4, 4, fr, (cuuint32_t)NB}, {64, 1, 16, fr, (cuuint32_t)NB}, {64, 16, 1, fr, (cuuint32_t)NB}};
+    for (int k = 0; k < 3; k++) {
+        const CUresult r = encode(&maps->m[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(feats), dims, strides,
+                                  boxes[k], ones, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return STTM_ERR_CUDA;
+    }
+    return STTM_OK;
+}
+
 // The two-stream path: Gram stage, decisions, ordering, chain stage, sum stage, pieces.
 sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, char* ws, void* out_feats,
                      int32_t* out_pos, int32_t* merge_map, int32_t* out_count, int64_t* out_offsets,
@@ -798,6 +844,8 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     if (!configured[dev]) {
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFlowSmemMax));
         STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFlowSmemMax));
+        STTM_CUDA_TRY(cudaFuncSetAttribute(k_flow_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)tc_smem_bytes(kTcMaxNB)));
         configured[dev] = true;
     }
     FlowMaps maps;
@@ -808,6 +856,7 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     fp.HW = g.HW; fp.N = g.N;
     fp.ntiles = f.ntiles;
     fp.NS = f.NS; fp.NB = f.NB;
+    fp.NSg = f.NSg; fp.NBg = f.NBg;
     fp.slot_bytes = f.slot_bytes; fp.R = f.R;
     fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
     fp.weight_mode = (int)p->wt;
@@ -838,7 +887,14 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     const int ntasks = f.nitems * f.NS;
     const unsigned grid = (unsigned)std::min(ntasks, 2 * sm_count());
     mark_stage(0, st);
-    if (!in.second_pass) {
+    if (!in.second_pass && f.tc) {
+        FlowMaps gmaps;
+        s = make_gram_tc_maps(feats, g, f.NBg, &gmaps);
+        if (s != STTM_OK) return s;
+        const unsigned ggrid = (unsigned)std::min(f.nitems * f.NSg, sm_count());
+        s = launch_after_smem(k_flow_gram_tc, ggrid, kTcThreads, f.smem_tc, false, st, fp, gmaps);
+        if (s != STTM_OK) return s;
+    } else if (!in.second_pass) {
         s = launch_after_smem(k_flow<false>, grid, kFlowThreads, f.smem, false, st, fp, maps);
         if (s != STTM_OK) return s;
     }

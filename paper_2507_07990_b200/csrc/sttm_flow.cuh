@@ -49,7 +49,8 @@ struct FlowParams {
     int B, T, H, W, D, L;
     int HW, N;
     int ntiles;
-    int NS, NB;              // channel slices, 64-channel blocks per slice
+    int NS, NB;              // channel slices, 64-channel blocks per slice (sum stage)
+    int NSg, NBg;            // the same for the Gram stage: `partial` holds NSg slices per frame
     int slot_bytes, R;
     int F, nseg, nitems;     // frames per item, items per (video, tile), items
     int weight_mode, out_f32, match_best;
@@ -59,7 +60,7 @@ struct FlowParams {
     int32_t* frame_roots;    // [B*T] chains that start in a frame (= its output rows), zero on entry
     float* tmax;             // budget mode, may be null (see FusedParams::tmax)
     const float* tau_t_dev;  // budget mode, may be null: [B] temporal thresholds in device memory
-    float* partial;          // [nitems][F+1][NS][128]: the Gram stage's numbers, [number][cell]
+    float* partial;          // [nitems][F+1][NSg][128]: the Gram stage's numbers, [cell][number]
     int32_t* hand;           // [nitems][F+1][16]: cover level | (link lane + 1) << 8 of every tile row
     FrameRec* recs;          // [nitems][F+2]: the chain stage's records, one per frame and a closing one
     int32_t* progress;       // [nitems]: number of records the chain stage has published (zero before the call)
@@ -94,6 +95,17 @@ __device__ __forceinline__ FlowItem flow_item(const FlowParams& p, int item) {
     it.n = t1 - it.tstart;
     it.last_seg = t1 == p.T;
     return it;
+}
+
+// Where the Gram stage's numbers of frame j of an item are: [slice][cell][number].  The frame before a
+// run is the last frame of the run before it, and its numbers are taken from there.
+__device__ __forceinline__ const float* flow_numbers(const FlowParams& p, const FlowItem& it, int j) {
+    if (it.halo && j == 0) {
+        const int seg = (it.item / p.ntiles) % p.nseg;
+        const int prev_n = p.F + (seg > 1 ? 1 : 0);         // frames of the run before, its own frame-before included
+        return p.partial + ((long long)(it.item - p.ntiles) * (p.F + 1) + prev_n - 1) * p.NSg * kSumVals;
+    }
+    return p.partial + ((long long)it.item * (p.F + 1) + j) * p.NSg * kSumVals;
 }
 
 // has the phase with this parity completed?  Suspends the thread for a while (the hardware's own
@@ -198,16 +210,17 @@ k_flow_decide(const __grid_constant__ FlowParams p, const __grid_constant__ Taus
     u[0] = u[1] = u[2] = 0.f;
     const bool has_prev = mine && j > 0;
     if (mine && valid) {
-        const float* src = p.partial + ((long long)it.item * (p.F + 1) + j) * p.NS * kSumVals + c;
-        for (int s = 0; s < p.NS; s++) {
-#pragma unroll
-            for (int k = 0; k < 8; k++) v[k] += __ldcg(src + s * kSumVals + k * 16);
+        const float4* src = reinterpret_cast<const float4*>(flow_numbers(p, it, j) + c * 8);
+        for (int s = 0; s < p.NSg; s++) {
+            const float4 a = __ldcg(src + s * (kSumVals / 4)), b = __ldcg(src + s * (kSumVals / 4) + 1);
+            v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+            v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
         }
         if (has_prev) {
-            const float* sp = src - (long long)p.NS * kSumVals;
-            for (int s = 0; s < p.NS; s++) {
-#pragma unroll
-                for (int k = 0; k < 3; k++) u[k] += __ldcg(sp + s * kSumVals + k * 16);
+            const float4* sp = reinterpret_cast<const float4*>(flow_numbers(p, it, j - 1) + c * 8);
+            for (int s = 0; s < p.NSg; s++) {
+                const float4 a = __ldcg(sp + s * (kSumVals / 4));
+                u[0] += a.x; u[1] += a.y; u[2] += a.z;
             }
         }
     }
@@ -534,8 +547,9 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
                     *reinterpret_cast<float2*>(redsum + e) = sum;
                 }
                 named_sync(1, nthr);
-                // contract to 8 numbers per cell: thread = (number, cell), stored [number][cell]
-                if (tid < kSumVals) dst[(long long)j * p.NS * kSumVals + tid] = combine_sums(redsum_a, tid & 15, tid >> 4, lg, W2s);
+                // contract to 8 numbers per cell: thread = (number, cell), stored [cell][number]
+                if (tid < kSumVals)
+                    dst[(long long)j * p.NS * kSumVals + (tid & 15) * 8 + (tid >> 4)] = combine_sums(redsum_a, tid & 15, tid >> 4, lg, W2s);
 #pragma unroll
                 for (int i = 0; i < kFlowMaxKs; i++) {
                     prv[i][0] = cur[i][0]; prv[i][1] = cur[i][1]; prv[i][2] = cur[i][2]; prv[i][3] = cur[i][3];

@@ -16,9 +16,10 @@ pytestmark = pytest.mark.gpu
 # (path, cluster size, frames per item) for sttm_set_tuning, then (sum slots, lead frames) for
 # sttm_set_ring_split: the library's own choice (the two-stream kernels), the same with item
 # borders every frame / every three / every seven frames, the three-pass kernels, single-pass
-# launches that force clusters and many item borders, the single-pass kernel without packing of
+# launches that force clusters and many item borders, the two-stream kernels with either Gram stage, the single-pass kernel without packing of
 # partial border tiles, and two other ways to share out its shared-memory slots
 TUNINGS = {"auto": (0, 0, 0, 0, 0), "flowf1": (5, 0, 1, 0, 0), "flowf3": (5, 0, 3, 0, 0), "flowf7": (5, 0, 7, 0, 0),
+           "gramsyncf3": (6, 0, 3, 0, 0), "gramsyncf6": (6, 0, 6, 0, 0),
            "threepass": (1, 0, 0, 0, 0), "c1f3": (2, 1, 3, 0, 0), "c2f2": (2, 2, 2, 0, 0),
            "c4f5": (2, 4, 5, 0, 0), "c8f1": (2, 8, 1, 0, 0), "nopack": (3, 0, 0, 0, 0), "sum2lead2": (2, 0, 0, 2, 2),
            "sum4": (2, 0, 7, 4, 1)}

@@ -45,12 +45,16 @@ __device__ __forceinline__ uint64_t tc_operand(uint32_t smem_addr) {
     return (uint64_t)((smem_addr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
            (2ull << 61);
 }
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t accumulate) {
+// (the two descriptors differ from product to product only in their address field, the low word:
+// the one thread that issues the products should have little else to do per product)
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(a), "l"(b), "r"(kTcIdesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(kTcIdesc), "r"(accumulate)
         : "memory");
 }
 // the mbarrier gets one arrival when every product issued so far by this thread has completed
@@ -170,11 +174,12 @@ k_flow_gram_tc(const __grid_constant__ FlowParams p, const __grid_constant__ Flo
                 tc_fence_after();
                 if (lane == 0) {
                     const uint32_t d = tmem_base + b * kTcAccStride;
-                    for (int blk = 0; blk < p.NBg; blk++) {
-                        const uint32_t rows = ring_base + s * slot_bytes + blk * kTcBlkBytes;
+                    const uint64_t b0 = tc_operand(ring_base + s * slot_bytes);
+                    const uint32_t hi = (uint32_t)(b0 >> 32);
+                    uint32_t b_lo = (uint32_t)b0, a_lo = b_lo + (kBlkBytes >> 4);       // A: without the frame before
+                    for (int blk = 0; blk < p.NBg; blk++, a_lo += kTcBlkBytes >> 4, b_lo += kTcBlkBytes >> 4) {
 #pragma unroll
-                        for (int k = 0; k < 4; k++)
-                            tc_mma(d, tc_operand(rows + kBlkBytes + k * 32), tc_operand(rows + k * 32), (blk | k) != 0);
+                        for (int k = 0; k < 4; k++) tc_mma(d, a_lo + 2 * k, b_lo + 2 * k, hi, (blk | k) != 0);
                     }
                     tc_commit(empty_bar + 8 * s);           // the slot has been read
                     tc_commit(acc_full + 8 * b);            // the sums are complete
@@ -205,7 +210,7 @@ k_flow_gram_tc(const __grid_constant__ FlowParams p, const __grid_constant__ Flo
             const int ngroups = tc_groups(it);
             for (int g = 0; g < ngroups; g++, q++) {
                 const int b = q & 1;
-                if (!mbar_wait_warp(acc_full + 8 * b, q >> 1, timed_out)) break;
+                if (!mbar_wait(acc_full + 8 * b, q >> 1, timed_out)) break;
                 tc_fence_after();
                 // columns 16 fq ... 16 fq + 15: the frame before (C); the next 16: the frame itself (G)
                 uint32_t v[32];

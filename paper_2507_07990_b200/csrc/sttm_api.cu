@@ -123,7 +123,7 @@ struct Plan {
 int g_tune_path = 0, g_tune_cluster = 0, g_tune_seg = 0, g_tune_pack = 0, g_tune_sum_slots = 0, g_tune_lead = 0;
 
 constexpr size_t kMaxSmem = 232448;   // 227 KB per CTA on sm_100
-constexpr double kFlowMinBytes = 512e6;                    // input size from which the two-stream kernels are the default
+constexpr double kFlowMinBytes = 200e6;                    // input size from which the two-stream kernels are the default
 constexpr size_t kFlowSmemMax = (233472 - 2 * 1024) / 2;   // per CTA when two share an SM
 
 // Cuts the grid into the kernel's tiles.  Full 4x4 tiles map one to one.  The partial tiles of
@@ -244,7 +244,7 @@ void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
     f->ok = false;
     // On request, for the budget mode (its second pass reuses the first pass's Gram stage), and for
     // large inputs: measured on B200, the two-stream kernels overtake the single-pass kernel between
-    // 0.25 GB (qwen: 0.23 against 0.21 ms) and 1.2 GB (long: 0.68 against 0.71 ms) of features.
+    // 0.08 GB (llava: 0.094 against 0.077 ms) and 0.23 GB (qwen: 0.163 against 0.172 ms) of features.
     const bool large = (double)g.B * g.N * g.D * 2.0 >= kFlowMinBytes;
     if (!(g_tune_path == 5 || g_tune_path == 6 || (g_tune_path == 0 && (budget || large)))) return;
     if (p->in_dtype != STTM_BF16 || g.D % 64 != 0) return;
@@ -280,7 +280,9 @@ void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
         for (int F = std::min(g.T, kFlowMaxF); F >= std::min(g.T, 8); F--) {
             const long long nseg = (g.T + F - 1) / F;
             const long long tasks = (long long)g.B * f->ntiles * nseg * f->NS;
-            const long long cost = ((tasks + ctas - 1) / ctas) * (F + 1 + 3);
+            // (two streams of that length, and the chain stage, one warp per run, a third of a frame's
+            // streaming time per frame of the run)
+            const long long cost = 20 * ((tasks + ctas - 1) / ctas) * (F + 1 + 3) + 6 * F;
             if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_F = F; }
         }
         f->F = best_F;

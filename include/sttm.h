@@ -308,7 +308,7 @@ void sttm_set_stage_events(void** events);
 
 /*
  * Benchmark and test knobs; 0 leaves a choice to the library.
- *   path             0: the library's choice (the two-stream kernels from 0.5 GB of features on
+ *   path             0: the library's choice (the two-stream kernels from 0.2 GB of features on
  *                    and for the budget mode, else the single-pass kernel, else the three-pass
  *                    kernels), 1: always the three-pass kernels, 2: the single-pass kernel
  *                    wherever it applies (bf16 input, D a multiple of 16, at most 64 tiles of

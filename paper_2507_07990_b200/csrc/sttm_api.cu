@@ -94,7 +94,7 @@ struct FusedPlan {
 struct FlowPlan {
     bool ok;
     int NS, NB, R, slot_bytes, F, nseg, nitems, ntiles;
-    int NSg, NBg;                   // slices and blocks per slice of the Gram stage
+    int NSg, NBg, NCg;              // Gram stage: slices, blocks per copy, copies per slice
     bool tc;                        // Gram stage on tcgen05 (else on mma.sync, with the sum stage's slices)
     size_t smem, smem_tc;
     TileDesc tiles[kMaxTiles];
@@ -293,16 +293,32 @@ void plan_flow(const sttm_params* p, const Geo& g, FlowPlan* f, bool budget) {
     f->tc = g_tune_path != 6;
     f->NBg = f->NB;
     f->NSg = f->NS;
+    f->NCg = 1;
     f->smem_tc = 0;
     if (f->tc) {
         int nb = 0;
         for (int n = std::min(nblk, kTcMaxNB); n >= 1 && nb == 0; n--)
             if (nblk % n == 0) nb = n;
-        if (nblk / nb > 64) {
+        // Slices: a slice's channels come in copies of nb blocks that are added in tensor memory, so the
+        // number of slices is free among the divisors of the copy count.  Few slices: little to write, read
+        // out and add up in the decision stage (about 1 % of the stage per slice, measured on `long`); many: even
+        // task counts and short tasks (a CTA's last task ends about a fifth of a task after the average).
+        const int ncopies = nblk / nb;
+        int best_ns = 0;
+        long long best_cost = 0;
+        for (int ns = 1; ns <= std::min(ncopies, 64); ns++) {
+            if (ncopies % ns != 0) continue;
+            const long long tasks = (long long)f->nitems * ns;
+            const long long rounds = (tasks + sm_count() - 1) / sm_count();
+            const long long cost = (rounds * 1000 + 180) / ns + 11ll * ns * f->nitems / sm_count();
+            if (best_ns == 0 || cost < best_cost) { best_ns = ns; best_cost = cost; }
+        }
+        if (best_ns == 0) {
             f->tc = false;
         } else {
             f->NBg = nb;
-            f->NSg = nblk / nb;
+            f->NSg = best_ns;
+            f->NCg = ncopies / best_ns;
             f->smem_tc = tc_smem_bytes(nb);
         }
     }
@@ -858,7 +874,7 @@ sttm_status run_flow(const void* feats, const sttm_params* p, const Plan& pl, ch
     fp.HW = g.HW; fp.N = g.N;
     fp.ntiles = f.ntiles;
     fp.NS = f.NS; fp.NB = f.NB;
-    fp.NSg = f.NSg; fp.NBg = f.NBg;
+    fp.NSg = f.NSg; fp.NBg = f.NBg; fp.NCg = f.NCg;
     fp.slot_bytes = f.slot_bytes; fp.R = f.R;
     fp.F = f.F; fp.nseg = f.nseg; fp.nitems = f.nitems;
     fp.weight_mode = (int)p->wt;

@@ -50,7 +50,7 @@ struct FlowParams {
     int HW, N;
     int ntiles;
     int NS, NB;              // channel slices, 64-channel blocks per slice (sum stage)
-    int NSg, NBg;            // the same for the Gram stage: `partial` holds NSg slices per frame
+    int NSg, NBg, NCg;       // Gram stage: slices (`partial` holds NSg per frame), blocks per copy, copies per slice
     int slot_bytes, R;
     int F, nseg, nitems;     // frames per item, items per (video, tile), items
     int weight_mode, out_f32, match_best;

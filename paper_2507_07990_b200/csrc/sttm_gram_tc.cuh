@@ -96,7 +96,7 @@ __host__ __device__ inline size_t tc_smem_bytes(int NBg) {
            (2 * kTcRing + 4) * 8 + 1024;
 }
 
-// p.NBg blocks per slice, p.NSg slices; tasks = (item, slice); partial is [nitems][F+1][NSg][128]
+// p.NSg slices of p.NCg x p.NBg blocks; tasks = (item, slice); partial is [nitems][F+1][NSg][128]
 __global__ void __launch_bounds__(kTcThreads, 1)
 k_flow_gram_tc(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps maps) {
     extern __shared__ unsigned char smem_raw[];
@@ -134,7 +134,7 @@ k_flow_gram_tc(const __grid_constant__ FlowParams p, const __grid_constant__ Flo
 
     const int ntasks = p.nitems * p.NSg;
     bool timed_out = false;
-    int q = 0;                      // groups taken up so far by this CTA: ring slot q % kTcRing, accumulator q % 2
+    int q = 0, qc = 0;              // groups (copies) taken up so far by this CTA, see the roles
 
     if (warp == 0) {
         // ------------------------------------- producer -------------------------------------
@@ -143,7 +143,9 @@ k_flow_gram_tc(const __grid_constant__ FlowParams p, const __grid_constant__ Flo
             const int slice = task % p.NSg;
             const TileBox bx = p.boxes[it.tile];
             const int ngroups = tc_groups(it);
-            for (int g = 0; g < ngroups; g++, q++) {
+            // one copy per group and part of the slice's channels: q counts copies here
+            for (int gh = 0; gh < ngroups * p.NCg && !timed_out; gh++, q++) {
+                const int g = gh / p.NCg, h = gh % p.NCg;
                 const int s = q % kTcRing;
                 // (this warp and the next have nothing else to do: they poll, which sees a completed phase
                 // sooner than a suspended wait is woken, and a slot that waits is bandwidth lost)
@@ -151,7 +153,8 @@ k_flow_gram_tc(const __grid_constant__ FlowParams p, const __grid_constant__ Flo
                 if (lane == 0) {
                     mbar_expect_tx(full_bar + 8 * s, slot_bytes);
                     tc_load_group(ring_base + s * slot_bytes, &maps.m[bx.kind], bx.x0, bx.y0,
-                                  it.b * p.T + it.tstart + it.halo + g * kTcFrames - 1, slice * p.NBg, full_bar + 8 * s);
+                                  it.b * p.T + it.tstart + it.halo + g * kTcFrames - 1, (slice * p.NCg + h) * p.NBg,
+                                  full_bar + 8 * s);
                 }
                 __syncwarp();
             }
@@ -167,24 +170,29 @@ k_flow_gram_tc(const __grid_constant__ FlowParams p, const __grid_constant__ Flo
         for (int task = blockIdx.x; task < ntasks && !timed_out; task += gridDim.x) {
             const FlowItem it = flow_item(p, task / p.NSg);
             const int ngroups = tc_groups(it);
-            for (int g = 0; g < ngroups; g++, q++) {
-                const int s = q % kTcRing, b = q & 1;
-                if (!mbar_wait(full_bar + 8 * s, q / kTcRing, timed_out)) break;
+            // q counts groups (accumulator q % 2), qc copies (ring slot qc % kTcRing): the parts of a
+            // slice's channels arrive in NCg copies and are added into the same accumulator
+            for (int g = 0; g < ngroups && !timed_out; g++, q++) {
+                const int b = q & 1;
                 if (q >= 2 && !mbar_wait(acc_empty + 8 * b, (q >> 1) - 1, timed_out)) break;
-                tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t d = tmem_base + b * kTcAccStride;
-                    const uint64_t b0 = tc_operand(ring_base + s * slot_bytes);
-                    const uint32_t hi = (uint32_t)(b0 >> 32);
-                    uint32_t b_lo = (uint32_t)b0, a_lo = b_lo + (kBlkBytes >> 4);       // A: without the frame before
-                    for (int blk = 0; blk < p.NBg; blk++, a_lo += kTcBlkBytes >> 4, b_lo += kTcBlkBytes >> 4) {
+                for (int h = 0; h < p.NCg; h++, qc++) {
+                    const int s = qc % kTcRing;
+                    if (!mbar_wait(full_bar + 8 * s, qc / kTcRing, timed_out)) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t d = tmem_base + b * kTcAccStride;
+                        const uint64_t b0 = tc_operand(ring_base + s * slot_bytes);
+                        const uint32_t hi = (uint32_t)(b0 >> 32);
+                        uint32_t b_lo = (uint32_t)b0, a_lo = b_lo + (kBlkBytes >> 4);   // A: without the frame before
+                        for (int blk = 0; blk < p.NBg; blk++, a_lo += kTcBlkBytes >> 4, b_lo += kTcBlkBytes >> 4) {
 #pragma unroll
-                        for (int k = 0; k < 4; k++) tc_mma(d, a_lo + 2 * k, b_lo + 2 * k, hi, (blk | k) != 0);
+                            for (int k = 0; k < 4; k++) tc_mma(d, a_lo + 2 * k, b_lo + 2 * k, hi, (h | blk | k) != 0);
+                        }
+                        tc_commit(empty_bar + 8 * s);                           // the slot has been read
+                        if (h + 1 == p.NCg) tc_commit(acc_full + 8 * b);        // the sums are complete
                     }
-                    tc_commit(empty_bar + 8 * s);           // the slot has been read
-                    tc_commit(acc_full + 8 * b);            // the sums are complete
+                    __syncwarp();
                 }
-                __syncwarp();
             }
         }
         // (the last products have completed before the tensor memory is given back)

@@ -801,16 +801,22 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-sttm_status make_flow_maps(const void* feats, const Geo& g, int NB, FlowMaps* maps) {
+// the driver's tensor-map encoder, through the runtime (no link against libcuda); null when it is not there
+EncodeTiledFn tensor_map_encoder() {
     static EncodeTiledFn encode = nullptr;
     if (encode == nullptr) {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess || fn == nullptr)
-            return STTM_ERR_CUDA;
-        encode = (EncodeTiledFn)fn;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            encode = (EncodeTiledFn)fn;
     }
+    return encode;
+}
+
+sttm_status make_flow_maps(const void* feats, const Geo& g, int NB, FlowMaps* maps) {
+    const EncodeTiledFn encode = tensor_map_encoder();
+    if (encode == nullptr) return STTM_ERR_CUDA;
     const cuuint64_t dims[5] = {64, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)(g.D / 64), (cuuint64_t)g.B * g.T};
     const cuuint64_t strides[4] = {(cuuint64_t)g.D * 2, (cuuint64_t)g.W * g.D * 2, 128, (cuuint64_t)g.HW * g.D * 2};
     const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
@@ -827,15 +833,8 @@ sttm_status make_flow_maps(const void* feats, const Geo& g, int NB, FlowMaps* ma
 // The same tensor with the frame axis inside the block axis: a box of five frames and NB blocks lands as
 // [block][frame][cell][64 channels], 80 rows of 128 bytes per block (the operand layout of k_flow_gram_tc).
 sttm_status make_gram_tc_maps(const void* feats, const Geo& g, int NB, FlowMaps* maps) {
-    static EncodeTiledFn encode = nullptr;
-    if (encode == nullptr) {
-        void* fn = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess || fn == nullptr)
-            return STTM_ERR_CUDA;
-        encode = (EncodeTiledFn)fn;
-    }
+    const EncodeTiledFn encode = tensor_map_encoder();
+    if (encode == nullptr) return STTM_ERR_CUDA;
     const cuuint64_t dims[5] = {64, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B * g.T, (cuuint64_t)(g.D / 64)};
     const cuuint64_t strides[4] = {(cuuint64_t)g.D * 2, (cuuint64_t)g.W * g.D * 2, (cuuint64_t)g.HW * g.D * 2, 128};
     const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
@@ -991,7 +990,10 @@ sttm_status run_generic(const T* feats, const sttm_params* p, const Plan& pl, ch
     sttm_status s;
     STTM_CUDA_TRY(cudaMemsetAsync(link, 0xff, (size_t)pl.cells * 4, st));
     STTM_CUDA_TRY(cudaMemsetAsync(cnt, 0, (size_t)pl.cells * 4, st));
-    for (int l = 1; l < py.L; l++) {
+    // (the general kernels serve quadtrees of four levels and more: levels 1 and 2 come from one pass)
+    k_gen_pool2<T><<<blocks_for(frames * py.H[2] * py.W[2] * 32, 128), 128, 0, st>>>(feats, pooled, g, py, norms, dots);
+    if ((s = launched()) != STTM_OK) return s;
+    for (int l = 3; l < py.L; l++) {
         k_gen_pool<T><<<blocks_for(frames * py.H[l] * py.W[l] * 32, 256), 256, 0, st>>>(feats, pooled, g, py, l, norms,
                                                                                        dots);
         if ((s = launched()) != STTM_OK) return s;

@@ -93,6 +93,119 @@ k_gen_pool(const T* __restrict__ feats, float* __restrict__ pooled, Geo g, Pyr p
     }
 }
 
+// Levels 1 and 2 in one pass over the cells: one warp per node of level 2 holds its (up to) 4 x 4 cells,
+// forms its level-1 children and itself, and takes all the norms and dot products of the three levels
+// (same sums in the same order as two passes of k_gen_pool; level 1 is not read back).
+template <typename T>
+__global__ void __launch_bounds__(128)
+k_gen_pool2(const T* __restrict__ feats, float* __restrict__ pooled, Geo g, Pyr py, float* __restrict__ norms,
+            float* __restrict__ dots) {
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int per = py.H[2] * py.W[2];
+    if (warp >= (long long)g.B * g.T * per) return;
+    const long long bt = warp / per;
+    const int idx2 = (int)(warp % per), i2 = idx2 / py.W[2], j2 = idx2 % py.W[2];
+    int kid[4], nk = 0;                 // level-1 children of the node
+    int cell[4][4], nc[4];              // their cells
+    for (int a = 0; a < 2; a++)
+        for (int b = 0; b < 2; b++) {
+            const int i1 = 2 * i2 + a, j1 = 2 * j2 + b;
+            if (i1 >= py.H[1] || j1 >= py.W[1]) continue;
+            kid[nk] = i1 * py.W[1] + j1;
+            nc[nk] = 0;
+            for (int a0 = 0; a0 < 2; a0++)
+                for (int b0 = 0; b0 < 2; b0++)
+                    if (2 * i1 + a0 < py.H[0] && 2 * j1 + b0 < py.W[0]) cell[nk][nc[nk]++] = (2 * i1 + a0) * py.W[0] + 2 * j1 + b0;
+            nk++;
+        }
+    float n2 = 0.f, n1[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+    float cn[4][4], d0[4][4];
+#pragma unroll
+    for (int k = 0; k < 4; k++)
+#pragma unroll
+        for (int c = 0; c < 4; c++) cn[k][c] = d0[k][c] = 0.f;
+    float* dst2 = pooled + (bt * py.upper + py.uoff[2] + idx2) * (long long)g.D;
+    for (int d = lane * VEC; d < g.D; d += 32 * VEC) {
+        float s2[VEC] = {0.f, 0.f, 0.f, 0.f};
+        float s1[4][VEC];
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            if (k < nk) {
+                float x[4][VEC];
+#pragma unroll
+                for (int v = 0; v < VEC; v++) s1[k][v] = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; c++) {
+                    if (c < nc[k]) {
+                        load4(feats + ((bt * g.HW + cell[k][c]) * (long long)g.D + d), x[c]);
+#pragma unroll
+                        for (int v = 0; v < VEC; v++) s1[k][v] += x[c][v];
+                    }
+                }
+                const float inv1 = 1.f / (float)nc[k];
+#pragma unroll
+                for (int v = 0; v < VEC; v++) s1[k][v] *= inv1;
+                store4(pooled + ((bt * py.upper + py.uoff[1] + kid[k]) * (long long)g.D + d), s1[k]);
+#pragma unroll
+                for (int v = 0; v < VEC; v++) n1[k] = fmaf(s1[k][v], s1[k][v], n1[k]);
+#pragma unroll
+                for (int c = 0; c < 4; c++) {
+                    if (c < nc[k]) {
+#pragma unroll
+                        for (int v = 0; v < VEC; v++) {
+                            d0[k][c] = fmaf(x[c][v], s1[k][v], d0[k][c]);
+                            cn[k][c] = fmaf(x[c][v], x[c][v], cn[k][c]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int v = 0; v < VEC; v++) s2[v] += s1[k][v];
+            }
+        }
+        const float inv2 = 1.f / (float)nk;
+#pragma unroll
+        for (int v = 0; v < VEC; v++) s2[v] *= inv2;
+        store4(dst2 + d, s2);
+#pragma unroll
+        for (int v = 0; v < VEC; v++) n2 = fmaf(s2[v], s2[v], n2);
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            if (k < nk) {
+#pragma unroll
+                for (int v = 0; v < VEC; v++) d1[k] = fmaf(s1[k][v], s2[v], d1[k]);
+            }
+        }
+    }
+    n2 = warp_sum(n2);
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        n1[k] = warp_sum(n1[k]);
+        d1[k] = warp_sum(d1[k]);
+#pragma unroll
+        for (int c = 0; c < 4; c++) { cn[k][c] = warp_sum(cn[k][c]); d0[k][c] = warp_sum(d0[k][c]); }
+    }
+    if (lane == 0) {
+        const long long at = bt * py.nodes;
+        norms[at + py.noff[2] + idx2] = n2;
+        if (py.L == 3) dots[at + py.noff[2] + idx2] = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            if (k < nk) {
+                norms[at + py.noff[1] + kid[k]] = n1[k];
+                dots[at + py.noff[1] + kid[k]] = d1[k];
+#pragma unroll
+                for (int c = 0; c < 4; c++) {
+                    if (c < nc[k]) {
+                        norms[at + cell[k][c]] = cn[k][c];
+                        dots[at + cell[k][c]] = d0[k][c];
+                    }
+                }
+            }
+        }
+    }
+}
+
 // does every existing child of a node exceed tau_s in cosine to it?  One thread per node of a
 // level >= 1.
 __global__ void __launch_bounds__(256)

@@ -287,6 +287,32 @@ def test_many_frames_take_the_separate_count_scan(path):
         helpers.assert_features_close(out.out_feats[offs[b]:offs[b + 1]].cpu().numpy(), ref.out_feats, False)
 
 
+# Channel counts that give the tensor-memory Gram stage other copy widths and copy counts per slice
+# (D / 64 = 3, 7, 15, 64 blocks: copies of 3, 7, 5 and 4 blocks), on grids with clipped tiles and strips,
+# runs of frames that are not a multiple of four, both Gram stages of the two-stream kernels.
+@pytest.mark.parametrize("gram", [5, 6], ids=["tensormemory", "mmasync"])
+@pytest.mark.parametrize("case", [(5, 13, 9, 192, 3), (9, 7, 5, 448, 2), (7, 16, 13, 960, 5), (6, 5, 12, 4096, 0),
+                                  (13, 4, 4, 320, 8), (2, 14, 3, 1024, 1)],
+                         ids=lambda c: "T%dH%dW%dD%df%d" % c)
+def test_two_stream_other_widths(case, gram):
+    T, H, W, D, F = case
+    lib = binding.load_library()
+    for seed in range(4):
+        spec = helpers.small_spec(7100 + 7 * seed + T, T, H, W, D, sigma=0.05, p_static=0.8)
+        video = inputs.make_video(spec)
+        taus = helpers.safe_thresholds(video, 0.5, 0.5)
+        if taus is not None:
+            break
+    assert taus is not None, "no seed gave thresholds with a margin"
+    lib.sttm_set_tuning(gram, 0, F)
+    try:
+        run_and_compare(video, taus[0], taus[1], out_dtype=torch.float32, stages=False)
+        run_and_compare(video, taus[0], taus[1], out_dtype=torch.bfloat16, stages=False, wt=binding.W_AREA)
+        assert lib.sttm_last_path() == 3
+    finally:
+        lib.sttm_set_tuning(0, 0, 0)
+
+
 def test_most_similar_destination(tuning):
     """Section 3.3's other destination rule: among the overlapping nodes above tau_t the most
     similar one instead of the top-left one.  Both sides pick a maximum, so the inputs are

@@ -582,7 +582,9 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
                 const long long chan0 = ((long long)slice * p.NB + 2 * warp) * 64;
                 // one record per frame, and a closing one that writes out what the item leaves
                 for (int j = 0; j <= it.n; j++, q++) {
-                    const bool frame = j < it.n;
+                    // (the frame before a run only opens the chains that come in from it: its features are not
+                    // added here, so they are not loaded either)
+                    const bool frame = j < it.n && !(it.halo && j == 0);
                     const int s = q % p.R;
                     if (!mbar_wait_warp(full_bar + 8 * s, q / p.R, timed_out)) break;
                     const uint32_t rec = recs_base + s * kRecBytes;
@@ -672,7 +674,7 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
                     if (__any_sync(0xffffffffu, late)) { timed_out = true; break; }
                 }
                 if (lane == 0) {
-                    const bool frame = j < it.n;
+                    const bool frame = j < it.n && !(kSum && it.halo && j == 0);
                     mbar_expect_tx(bar, (uint32_t)((frame ? p.slot_bytes : 0) + (kSum ? kRecBytes : 0)));
                     if (frame)
                         tma_load_tile(ring_base + s * p.slot_bytes, &maps.m[bx.kind], bx.x0, bx.y0, slice * p.NB,

@@ -440,13 +440,26 @@ k_rows_scan(Geo g, const int8_t* __restrict__ cover, const int32_t* __restrict__
         const int v = frame_roots[(long long)b * g.T + i];
         if (i < t) before_frames += v; else after_frames += v;
     }
-    int off_i, carry, rest;
-    block_exclusive_scan(before_videos, off_i, sm);
+    // the three totals in one pass: warp sums, then one thread per total adds the warps' sums
+    __shared__ int tot3[3][8];
+    {
+        int v0 = before_videos, v1 = before_frames, v2 = after_frames;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            v0 += __shfl_xor_sync(0xffffffffu, v0, o);
+            v1 += __shfl_xor_sync(0xffffffffu, v1, o);
+            v2 += __shfl_xor_sync(0xffffffffu, v2, o);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            tot3[0][threadIdx.x >> 5] = v0;
+            tot3[1][threadIdx.x >> 5] = v1;
+            tot3[2][threadIdx.x >> 5] = v2;
+        }
+    }
     __syncthreads();
-    block_exclusive_scan(before_frames, carry, sm);
-    __syncthreads();
-    block_exclusive_scan(after_frames, rest, sm);
-    __syncthreads();
+    int off_i = 0, carry = 0, rest = 0;
+#pragma unroll
+    for (int w = 0; w < 8; w++) { off_i += tot3[0][w]; carry += tot3[1][w]; rest += tot3[2][w]; }
     const long long off = off_i;
     if (t == 0 && threadIdx.x == 0) {
         out_count[b] = carry + rest;

@@ -338,6 +338,9 @@ void sttm_set_ring_split(int sum_slots, int lead_frames);
 /* Which kernels the last sttm_merge_ex on this thread ran: 0 three-pass, 1 single-pass (fused),
  * 2 the general kernels for quadtrees of more than three levels, 3 two-stream. */
 int sttm_last_path(void);
+/* Which Gram stage the last sttm_merge_ex on this thread ran when it took the two-stream kernels:
+ * 2 on tcgen05 with the sums in tensor memory, 1 on mma.sync; 0 when it took other kernels. */
+int sttm_last_gram_stage(void);
 
 /*
  * Launch shape the fused kernel would get for these params (host pointers; queries the

@@ -27,7 +27,7 @@ STATUS_NAMES = ["ok", "bad argument", "unsupported shape", "workspace too small"
 EXPORTS = ["sttm_default_params", "sttm_workspace_bytes", "sttm_sims_per_frame", "sttm_spatial",
            "sttm_temporal", "sttm_merge_ex", "sttm_merge", "sttm_merge_host", "sttm_release_cache",
            "sttm_last_launch_count", "sttm_status_string", "sttm_stage_count", "sttm_stage_name",
-           "sttm_set_stage_events", "sttm_set_tuning", "sttm_set_ring_split", "sttm_last_path",
+           "sttm_set_stage_events", "sttm_set_tuning", "sttm_set_ring_split", "sttm_last_path", "sttm_last_gram_stage",
            "sttm_fused_launch_shape", "sttm_spatial_static", "sttm_merged_positions",
            "sttm_merged_positions_workspace", "sttm_merge_budget", "sttm_budget_workspace_bytes",
            "sttm_row_weights", "sttm_segment_fold", "sttm_segment_emit", "sttm_segment_finish",
@@ -120,6 +120,8 @@ def load_library(path: Optional[str] = None):
     lib.sttm_merge_status.restype = C.c_int
     lib.sttm_last_path.argtypes = []
     lib.sttm_last_path.restype = C.c_int
+    lib.sttm_last_gram_stage.argtypes = []
+    lib.sttm_last_gram_stage.restype = C.c_int
     lib.sttm_fused_launch_shape.argtypes = [pp, C.POINTER(C.c_int)]
     lib.sttm_fused_launch_shape.restype = C.c_int
     lib.sttm_status_string.argtypes = [C.c_int]

@@ -53,6 +53,7 @@ const char* const kStageNames[4][kStageCount] = {
     {"fused", "roots", "ordering", "gather", "-"},
     {"-", "-", "-", "-", "general"},
     {"gram", "decide+ordering+chain", "sum", "roots+pieces", "-"}};
+thread_local int g_last_gram = 0;   // 0: no two-stream kernels, 1: their Gram stage on mma.sync, 2: on tcgen05
 thread_local int g_last_path = 0;   // 0: three-pass kernels, 1: single-pass kernel, 2: general kernels, 3: two-stream kernels
 
 // Stage boundary `boundary` (before stage `boundary`, after the one before it): an event for the
@@ -1151,6 +1152,8 @@ const char* sttm_stage_name(int i) { return i >= 0 && i < kStageCount ? kStageNa
 
 int sttm_last_path(void) { return g_last_path; }
 
+int sttm_last_gram_stage(void) { return g_last_gram; }
+
 int sttm_fused_launch_shape(const sttm_params* p, int* shape) {
     Plan pl;
     if (shape == nullptr || make_plan(p, &pl) != STTM_OK || !pl.f.ok) return 0;
@@ -1260,6 +1263,7 @@ sttm_status merge_impl(const void* feats, const sttm_params* p, void* ws_, size_
     int32_t* link = (int32_t*)(ws + pl.link);
     int32_t* root = (int32_t*)(ws + pl.root);
     g_last_path = pl.generic ? 2 : (pl.fl.ok ? 3 : (pl.f.ok ? 1 : 0));
+    g_last_gram = !pl.generic && pl.fl.ok ? (pl.fl.tc ? 2 : 1) : 0;
     if (pl.generic) {
         // more than three quadtree levels: the plain kernels, no stage breakdown
         for (int i = 0; i <= 4; i++) mark_stage(i, st);

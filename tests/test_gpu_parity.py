@@ -308,7 +308,7 @@ def test_two_stream_other_widths(case, gram):
     try:
         run_and_compare(video, taus[0], taus[1], out_dtype=torch.float32, stages=False)
         run_and_compare(video, taus[0], taus[1], out_dtype=torch.bfloat16, stages=False, wt=binding.W_AREA)
-        assert lib.sttm_last_path() == 3
+        assert lib.sttm_last_path() == 3 and lib.sttm_last_gram_stage() == (2 if gram == 5 else 1)
     finally:
         lib.sttm_set_tuning(0, 0, 0)
 

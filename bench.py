@@ -572,7 +572,7 @@ def parse_args():
     ap.add_argument("--match", default="topleft", choices=["topleft", "best"],
                     help="destination rule of the temporal link (the paper's default, or its most-similar variant)")
     ap.add_argument("--tuning", default="0,0,0",
-                    help="path,cluster_size,frames_per_item for sttm_set_tuning (path 5: the two-stream kernels), "
+                    help="path,cluster_size,frames_per_item for sttm_set_tuning (path 5: the two-stream kernels, 6: the same with the mma.sync Gram stage, 2: the single-pass kernel), "
                          "optionally followed by sum_slots,lead_frames for sttm_set_ring_split (0 = library's choice)")
     ap.add_argument("--mode", default="videos", choices=["videos", "segments"],
                     help="videos: every rank merges its own videos (the default); segments: one video cut by frames "

@@ -600,6 +600,9 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
                         const float inv = mine && fc.y == 0 ? 1.f / __uint_as_float(fc.w) : 1.f;
                         const long long row = (long long)(int)fc.z * p.D + chan0 + 2 * t4;
                         const bool skip = (int)fc.z < 0;                                // a row beyond the capacity
+                        // bf16 rows leave in 16-byte stores: the four lanes of a group first exchange their
+                        // words so that each holds whole 8-channel tiles (the lanes that take part)
+                        const unsigned quads = __ballot_sync(0xffffffffu, mine && fc.y == 0 && !p.out_f32);
 #define STTM_FLOW_FLUSH(I0, I1)                                                                               \
     if (fc.y != 0 || p.out_f32) {                                                                             \
         float* dst = (fc.y != 0 ? p.pieces : reinterpret_cast<float*>(p.out)) + row;                          \
@@ -610,12 +613,21 @@ k_flow(const __grid_constant__ FlowParams p, const __grid_constant__ FlowMaps ma
             if (nt < ntmax && !skip) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x, y);            \
         }                                                                                                     \
     } else {                                                                                                  \
-        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row;                                   \
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (row - 2 * t4);                        \
+        uint32_t w[16];                                                                                       \
         _Pragma("unroll") for (int nt = 0; nt < 16; nt++) {                                                   \
-            const uint32_t w = pack_bf16x2(sums[nt][I0] * inv, sums[nt][I1] * inv);                           \
+            w[nt] = pack_bf16x2(sums[nt][I0] * inv, sums[nt][I1] * inv);                                      \
             sums[nt][I0] = 0.f;                                                                               \
             sums[nt][I1] = 0.f;                                                                               \
-            if (nt < ntmax && !skip) *reinterpret_cast<uint32_t*>(dst + nt * 8) = w;                          \
+        }                                                                                                     \
+        _Pragma("unroll") for (int m = 0; m < 4; m++) {                                                       \
+            uint32_t a0 = w[4 * m], a1 = w[4 * m + 1], a2 = w[4 * m + 2], a3 = w[4 * m + 3], r;               \
+            r = __shfl_xor_sync(quads, (t4 & 1) ? a0 : a1, 1); if (t4 & 1) a0 = r; else a1 = r;               \
+            r = __shfl_xor_sync(quads, (t4 & 1) ? a2 : a3, 1); if (t4 & 1) a2 = r; else a3 = r;               \
+            r = __shfl_xor_sync(quads, (t4 & 2) ? a0 : a2, 2); if (t4 & 2) a0 = r; else a2 = r;               \
+            r = __shfl_xor_sync(quads, (t4 & 2) ? a1 : a3, 2); if (t4 & 2) a1 = r; else a3 = r;               \
+            const int nt = 4 * m + t4;                      /* lane t4 now holds tile 4 m + t4 whole */      \
+            if (nt < ntmax && !skip) *reinterpret_cast<uint4*>(dst + nt * 8) = make_uint4(a0, a1, a2, a3);    \
         }                                                                                                     \
     }
                         if (mine) {
